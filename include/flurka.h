@@ -1,0 +1,139 @@
+/*
+ * flurka.h -- C ABI of the FLuRKA attention forward pass for NVIDIA B200 (sm_100a).
+ *
+ * The operation (arxiv 2306.15799, Section 3, Eq. (2), with the row normalisation that
+ * Appendix D writes out for kernel attention), per batch b and head h, non-causal:
+ *
+ *     K' = E K            V' = F V                  (Section 2.1: E, F are k x N, shared)
+ *     O  = phi(Q) ( phi(K')^T V' )  /  phi(Q) ( phi(K')^T 1_k )          (row-wise division)
+ *
+ * with the feature map phi chosen by `variant` (Section 4's instances):
+ *     FLURKA_PERFORMER  phi(x)_i = exp(w_i . x - |x|^2 / 2) / sqrt(m),  i < m   (positive random
+ *                       features; W = [w_0 .. w_{m-1}] is an input),
+ *     FLURKA_RNN        phi(x)_c = elu(x_c) + 1,  c < d                          (no W, m ignored).
+ * The per-head linear maps W^Q, W^K, W^V of Eq. (2) are applied by the caller ((E K) W^K = E (K W^K)).
+ * No softmax scale is applied: callers pre-scale Q and K.
+ *
+ * Layout.  All tensors are dense, row-major, contiguous:
+ *     Q, K, V, out : [B, H, N, d]      E, F : [k, N]      W : [m, d]
+ * and share one element type per call: bfloat16 (default) or float32 (FLURKA_IO_FP32 or-ed into
+ * `variant`).  Accumulation is fp32 in both cases.
+ *
+ * Ownership.  Every pointer is caller-owned; the library keeps none of them after the call returns.
+ * `out` must not overlap an input.  Scratch memory comes from the workspace (see below).
+ *
+ * Errors.  Every function returns FLURKA_OK (0) or a negative flurka_status; on error NOTHING has been
+ * launched or copied.  No exceptions, no abort, nothing is printed.
+ *
+ * Threads.  One call at a time per process (the workspace and the descriptor cache are shared).
+ */
+#ifndef FLURKA_H_
+#define FLURKA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FLURKA_VERSION 100
+
+typedef enum {
+  FLURKA_PERFORMER = 0, /* Linformer-Performer: FAVOR+ positive random features (Section 2.1, Section 4) */
+  FLURKA_RNN = 1        /* Linformer-RNN: phi(x) = elu(x) + 1 (Section 2.1, Section 4)                  */
+} flurka_kernel_t;
+
+#define FLURKA_IO_BF16 0x000 /* default element type of Q, K, V, E, F, W, out */
+#define FLURKA_IO_FP32 0x100 /* or-ed into `variant`: all of them are float32 */
+
+typedef enum {
+  FLURKA_OK = 0,
+  FLURKA_ERR_NULL = -1,        /* a required pointer is NULL                                        */
+  FLURKA_ERR_VARIANT = -2,     /* unknown kernel, element type or selector                          */
+  FLURKA_ERR_SHAPE = -3,       /* a size is <= 0, d > 128, k > 4096, or the forced path cannot run it */
+  FLURKA_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned                                  */
+  FLURKA_ERR_WORKSPACE = -5,   /* caller workspace too small, or the library could not allocate one */
+  FLURKA_ERR_CUDA = -6,        /* a CUDA call failed; flurka_last_cuda_error() has the cudaError_t  */
+  FLURKA_ERR_DEVICE = -7,      /* no sm_100 device is current                                       */
+  FLURKA_ERR_OVERLAP = -8      /* out overlaps an input                                             */
+} flurka_status;
+
+/* Execution paths, for flurka_set_path().  AUTO picks the tensor-core path when the shape allows. */
+typedef enum {
+  FLURKA_PATH_AUTO = 0,
+  FLURKA_PATH_SIMT = 1,   /* fp32 CUDA-core kernels: any shape within the limits, both element types */
+  FLURKA_PATH_TENSOR = 2  /* tcgen05 / TMEM / TMA kernels: bf16 only, shape rules below; else error  */
+} flurka_path_t;
+
+/*
+ * flurka_forward -- the whole forward pass of Eq. (2) on DEVICE buffers, asynchronous on `stream`.
+ *
+ *   Q, K, V   device, [B,H,N,d]          E, F   device, [k,N]          W   device, [m,d] (NULL for RNN)
+ *   variant   flurka_kernel_t | FLURKA_IO_BF16 / FLURKA_IO_FP32
+ *   out       device, [B,H,N,d], same element type
+ *   stream    a cudaStream_t passed as void*; NULL is the default stream
+ *
+ * Shape limits: B, H, N >= 1, B*H <= 65535; 1 <= d <= 128; 1 <= k <= 4096; PERFORMER: m >= 1.
+ * Pointers 16-byte aligned.  The tensor-core path additionally needs bf16, d in {64, 128},
+ * N % 128 == 0, k % 64 == 0 with k <= 512, and (PERFORMER) m in {64, 128, 192, 256}; other shapes run
+ * on the SIMT path.  The call enqueues work and returns; it never synchronises.  Scratch comes from the
+ * workspace set by flurka_set_workspace(), or from one the library allocates (and re-uses) on first need.
+ */
+int flurka_forward(const void* Q, const void* K, const void* V, const void* E, const void* F,
+                   const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
+                   void* stream);
+
+/*
+ * flurka_forward_host -- the same operation (Eq. (2)) on HOST buffers (same shapes and element types).
+ * Copies the inputs to the device (cudaMemcpyAsync; pinned host memory makes them asynchronous),
+ * runs flurka_forward, copies `out` back and synchronises `stream` before returning.  Device staging
+ * buffers are allocated by the library on first use and re-used while they are large enough.
+ */
+int flurka_forward_host(const void* Q, const void* K, const void* V, const void* E, const void* F,
+                        const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
+                        void* stream);
+
+/* Bytes of device scratch flurka_forward needs for this problem (0 on invalid arguments). Holds the
+ * fp32 projections K', V' (Eq. (2)'s E K and F V), the key-side feature summaries and a status word. */
+size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m);
+
+/* Hands the library a caller-owned device workspace (256-byte aligned). NULL/0 returns to the
+ * library-owned one. The caller keeps it alive until the last call using it has finished. */
+int flurka_set_workspace(void* dev_ptr, size_t bytes);
+
+/* Forces an execution path for later calls (flurka_path_t); returns the previous one. */
+int flurka_set_path(int path);
+
+/* The path the most recent successful flurka_forward took (FLURKA_PATH_SIMT or FLURKA_PATH_TENSOR). */
+int flurka_last_path(void);
+
+/* Number of kernels the most recent successful flurka_forward launched. */
+int flurka_last_launches(void);
+
+/*
+ * Copies an intermediate of the most recent flurka_forward to a DEVICE buffer, asynchronously on
+ * `stream` (order it after the forward).  `which`: 0 = K' [B,H,k,d] fp32, 1 = V' [B,H,k,d] fp32
+ * (Eq. (2)'s E K, F V), 2 = key-side summary a [B,H,p,d] fp32 (a_i = sum_j phi(k'_j)_i v'_j / z_i,
+ * p = m or d; SIMT path only), 3 = per-feature weights [B,H,p] fp32 (PERFORMER: log z_i with the
+ * exponent maximum added back; RNN: z_i), 4 = status words (4 x int32).  `bytes` must equal the
+ * intermediate's size.
+ */
+int flurka_debug_copy(int which, void* dev_dst, size_t bytes, void* stream);
+
+/* Synchronises the device and returns the status word the kernels of the last call left behind:
+ * 0 = clean; bit 0 = a bounded wait gave up (results invalid); bit 1 = an index check failed. */
+int flurka_last_status(void);
+
+/* cudaError_t (as int) behind the most recent FLURKA_ERR_CUDA. */
+int flurka_last_cuda_error(void);
+
+/* Static, human-readable text for a flurka_status. */
+const char* flurka_strerror(int code);
+
+/* FLURKA_VERSION of the loaded library. */
+int flurka_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLURKA_H_ */

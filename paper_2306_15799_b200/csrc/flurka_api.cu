@@ -1,0 +1,414 @@
+// Host side of the FLuRKA forward library: argument checks, workspace, path selection, launches.
+// The C ABI is declared and documented in include/flurka.h.
+#include "flurka.h"
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "simt_kernels.cuh"
+#include "tensor_path.cuh"
+
+namespace {
+
+using namespace flurka;
+
+struct Problem {
+  int kernel;      // FLURKA_PERFORMER / FLURKA_RNN
+  bool fp32;       // element type of the I/O tensors
+  int B, H, N, d, k, m;
+  int BH() const { return B * H; }
+  int p() const { return kernel == FLURKA_PERFORMER ? m : d; }   // feature dimension
+  size_t esize() const { return fp32 ? 4 : 2; }
+  size_t qkv_elems() const { return (size_t)B * H * N * d; }
+  size_t ef_elems() const { return (size_t)k * N; }
+  size_t w_elems() const { return kernel == FLURKA_PERFORMER ? (size_t)m * d : 0; }
+};
+
+// Workspace layout (all offsets 256-byte aligned):
+//   kpvp    fp32 [2][BH][k][d]     K' then V'
+//   weight  fp32 [BH][p]           b_i (PERFORMER) or z_i (RNN)
+//   a32     fp32 [BH][p][d]        key-side summary, feature-major
+//   aT16    fp16 [BH][d][p]        the same, transposed, as the tensor-core B operand
+//   status  int32[4]
+struct Layout {
+  size_t kpvp, weight, a32, aT16, status, total;
+};
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+Layout make_layout(const Problem& pr) {
+  Layout L;
+  size_t off = 0;
+  L.kpvp = off;   off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
+  L.weight = off; off = align256(off + (size_t)pr.BH() * pr.p() * 4);
+  L.a32 = off;    off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 4);
+  L.aT16 = off;   off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 2);
+  L.status = off; off = align256(off + 16);
+  L.total = off;
+  return L;
+}
+
+struct State {
+  void* user_ws = nullptr;
+  size_t user_ws_bytes = 0;
+  void* own_ws = nullptr;
+  size_t own_ws_bytes = 0;
+  int path = FLURKA_PATH_AUTO;
+  int last_path = 0;
+  int last_launches = 0;
+  int last_cuda_error = 0;
+  // most recent forward (for flurka_debug_copy / flurka_last_status)
+  bool have_last = false;
+  Problem last_problem{};
+  char* last_ws = nullptr;
+  // host-buffer entry point: device staging
+  void* stage = nullptr;
+  size_t stage_bytes = 0;
+};
+
+State g;
+
+int cuda_fail(cudaError_t e) {
+  g.last_cuda_error = (int)e;
+  (void)cudaGetLastError();
+  return FLURKA_ERR_CUDA;
+}
+
+int parse_problem(int variant, int B, int H, int N, int d, int k, int m, Problem* pr) {
+  const int kernel = variant & 0xff;
+  const int io = variant & ~0xff;
+  if (kernel != FLURKA_PERFORMER && kernel != FLURKA_RNN) return FLURKA_ERR_VARIANT;
+  if (io != FLURKA_IO_BF16 && io != FLURKA_IO_FP32) return FLURKA_ERR_VARIANT;
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || k <= 0) return FLURKA_ERR_SHAPE;
+  if (d > 128 || k > 4096) return FLURKA_ERR_SHAPE;
+  if (kernel == FLURKA_PERFORMER && m <= 0) return FLURKA_ERR_SHAPE;
+  if ((long long)B * H > 65535) return FLURKA_ERR_SHAPE;
+  pr->kernel = kernel;
+  pr->fp32 = io == FLURKA_IO_FP32;
+  pr->B = B; pr->H = H; pr->N = N; pr->d = d; pr->k = k;
+  pr->m = kernel == FLURKA_PERFORMER ? m : 0;
+  return FLURKA_OK;
+}
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + nb && y < x + na;
+}
+
+bool tensor_path_ok(const Problem& pr) {
+  if (pr.fp32) return false;
+  if (pr.d != 64 && pr.d != 128) return false;
+  if (pr.N % 128) return false;
+  if (pr.k % 64 || pr.k > 512) return false;
+  if (pr.kernel == FLURKA_PERFORMER && (pr.m % 64 || pr.m > 256)) return false;
+  return tensor_path_built();
+}
+
+int get_workspace(size_t need, char** ws) {
+  if (g.user_ws) {
+    if (g.user_ws_bytes < need) return FLURKA_ERR_WORKSPACE;
+    *ws = (char*)g.user_ws;
+    return FLURKA_OK;
+  }
+  if (g.own_ws_bytes < need) {
+    if (g.own_ws) {
+      cudaError_t e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return cuda_fail(e);
+      cudaFree(g.own_ws);
+      g.own_ws = nullptr;
+      g.own_ws_bytes = 0;
+    }
+    cudaError_t e = cudaMalloc(&g.own_ws, need);
+    if (e != cudaSuccess) { cuda_fail(e); return FLURKA_ERR_WORKSPACE; }
+    g.own_ws_bytes = need;
+  }
+  *ws = (char*)g.own_ws;
+  return FLURKA_OK;
+}
+
+int check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return FLURKA_ERR_DEVICE; }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return FLURKA_ERR_DEVICE;
+  }
+  return major == 10 ? FLURKA_OK : FLURKA_ERR_DEVICE;
+}
+
+template <typename T>
+int launch_simt_down_project(const Problem& pr, const void* K, const void* V, const void* E,
+                             const void* F, float* kpvp, cudaStream_t st, int* launches) {
+  // enough sequence splits to fill the machine; each split is a multiple of the 32-wide tile
+  const int jt = (pr.k + 31) / 32;
+  int nsplit = (4 * 148 + jt * pr.BH() * 2 - 1) / (jt * pr.BH() * 2);
+  const int max_split = (pr.N + 255) / 256;
+  if (nsplit > max_split) nsplit = max_split;
+  if (nsplit < 1) nsplit = 1;
+  if (nsplit > 16384) nsplit = 16384;
+  int chunk = (pr.N + nsplit - 1) / nsplit;
+  chunk = (chunk + 31) / 32 * 32;
+  nsplit = (pr.N + chunk - 1) / chunk;
+  dim3 grid(jt, pr.BH(), 2 * nsplit);
+  simt_down_project<T><<<grid, 256, 0, st>>>((const T*)K, (const T*)V, (const T*)E, (const T*)F, kpvp,
+                                            pr.BH(), pr.N, pr.d, pr.k, nsplit, chunk);
+  ++*launches;
+  return FLURKA_OK;
+}
+
+template <typename T, bool P>
+int launch_simt_key_side(const Problem& pr, const float* kpvp, const void* W, float* weight, float* a32,
+                         __half* aT16, cudaStream_t st, int* launches) {
+  const size_t smem = ((size_t)8 * pr.k + 32 * (pr.d + 1)) * 4;
+  auto fn = simt_key_side<T, P>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  dim3 grid((pr.p() + 7) / 8, pr.BH());
+  fn<<<grid, 256, smem, st>>>(kpvp, (const T*)W, weight, a32, aT16, pr.BH(), pr.d, pr.k, pr.p());
+  ++*launches;
+  return FLURKA_OK;
+}
+
+template <typename T, bool P>
+int launch_simt_query_side(const Problem& pr, const void* Q, const void* W, const float* weight,
+                           const float* a32, void* out, cudaStream_t st, int* launches) {
+  const size_t smem = ((size_t)32 * (pr.d + 1) + 32 * pr.d) * 4;
+  dim3 grid((pr.N + 31) / 32, pr.BH());
+  simt_query_side<T, P><<<grid, 256, smem, st>>>((const T*)Q, (const T*)W, weight, a32, (T*)out, pr.N,
+                                                 pr.d, pr.p());
+  ++*launches;
+  return FLURKA_OK;
+}
+
+template <typename T>
+int key_side_dispatch(const Problem& pr, const float* kpvp, const void* W, float* weight, float* a32,
+                      __half* aT16, cudaStream_t st, int* launches) {
+  return pr.kernel == FLURKA_PERFORMER
+             ? launch_simt_key_side<T, true>(pr, kpvp, W, weight, a32, aT16, st, launches)
+             : launch_simt_key_side<T, false>(pr, kpvp, W, weight, a32, aT16, st, launches);
+}
+
+template <typename T>
+int run_simt(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
+             const void* E, const void* F, const void* W, void* out, cudaStream_t st, int* launches) {
+  float* kpvp = (float*)(ws + L.kpvp);
+  float* weight = (float*)(ws + L.weight);
+  float* a32 = (float*)(ws + L.a32);
+  cudaError_t e = cudaMemsetAsync(kpvp, 0, (size_t)2 * pr.BH() * pr.k * pr.d * 4, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  int rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
+  if (rc) return rc;
+  rc = key_side_dispatch<T>(pr, kpvp, W, weight, a32, nullptr, st, launches);
+  if (rc) return rc;
+  rc = pr.kernel == FLURKA_PERFORMER
+           ? launch_simt_query_side<T, true>(pr, Q, W, weight, a32, out, st, launches)
+           : launch_simt_query_side<T, false>(pr, Q, W, weight, a32, out, st, launches);
+  if (rc) return rc;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  return FLURKA_OK;
+}
+
+int validate_pointers(const Problem& pr, const void* Q, const void* K, const void* V, const void* E,
+                      const void* F, const void* W, const void* out) {
+  if (!Q || !K || !V || !E || !F || !out) return FLURKA_ERR_NULL;
+  if (pr.kernel == FLURKA_PERFORMER && !W) return FLURKA_ERR_NULL;
+  const void* ptrs[7] = {Q, K, V, E, F, W, out};
+  for (const void* ptr : ptrs)
+    if (ptr && ((uintptr_t)ptr & 15)) return FLURKA_ERR_ALIGN;
+  const size_t qb = pr.qkv_elems() * pr.esize(), eb = pr.ef_elems() * pr.esize(),
+               wb = pr.w_elems() * pr.esize();
+  if (overlaps(out, qb, Q, qb) || overlaps(out, qb, K, qb) || overlaps(out, qb, V, qb) ||
+      overlaps(out, qb, E, eb) || overlaps(out, qb, F, eb) || (W && wb && overlaps(out, qb, W, wb)))
+    return FLURKA_ERR_OVERLAP;
+  return FLURKA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int flurka_forward(const void* Q, const void* K, const void* V, const void* E, const void* F,
+                   const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
+                   void* stream) {
+  Problem pr;
+  int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
+  if (rc) return rc;
+  rc = validate_pointers(pr, Q, K, V, E, F, W, out);
+  if (rc) return rc;
+  int path = g.path;
+  const bool tensor_ok = tensor_path_ok(pr);
+  if (path == FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
+  if (path == FLURKA_PATH_AUTO) path = tensor_ok ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
+  rc = check_device();
+  if (rc) return rc;
+  const Layout L = make_layout(pr);
+  char* ws = nullptr;
+  rc = get_workspace(L.total, &ws);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  int launches = 0;
+  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, 16, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+
+  if (path == FLURKA_PATH_TENSOR) {
+    TensorArgs ta;
+    ta.kernel = pr.kernel; ta.B = pr.B; ta.H = pr.H; ta.N = pr.N; ta.d = pr.d; ta.k = pr.k; ta.m = pr.m;
+    ta.Q = Q; ta.K = K; ta.V = V; ta.E = E; ta.F = F; ta.W = W; ta.out = out;
+    ta.kpvp = (float*)(ws + L.kpvp);
+    ta.weight = (float*)(ws + L.weight);
+    ta.a32 = (float*)(ws + L.a32);
+    ta.aT16 = (__half*)(ws + L.aT16);
+    ta.status = (int*)(ws + L.status);
+    int cuda_err = 0;
+    rc = run_tensor_path(ta, st, &launches, &cuda_err);
+    if (rc == FLURKA_ERR_CUDA) g.last_cuda_error = cuda_err;
+  } else if (pr.fp32) {
+    rc = run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
+  } else {
+    rc = run_simt<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
+  }
+  if (rc) return rc;
+  g.last_path = path;
+  g.last_launches = launches;
+  g.have_last = true;
+  g.last_problem = pr;
+  g.last_ws = ws;
+  return FLURKA_OK;
+}
+
+int flurka_forward_host(const void* Q, const void* K, const void* V, const void* E, const void* F,
+                        const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
+                        void* stream) {
+  Problem pr;
+  int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
+  if (rc) return rc;
+  if (!Q || !K || !V || !E || !F || !out) return FLURKA_ERR_NULL;
+  if (pr.kernel == FLURKA_PERFORMER && !W) return FLURKA_ERR_NULL;
+  rc = check_device();
+  if (rc) return rc;
+  const size_t qb = align256(pr.qkv_elems() * pr.esize());
+  const size_t eb = align256(pr.ef_elems() * pr.esize());
+  const size_t wb = align256(pr.w_elems() * pr.esize());
+  const size_t need = 4 * qb + 2 * eb + wb;
+  if (g.stage_bytes < need) {
+    if (g.stage) {
+      cudaError_t e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return cuda_fail(e);
+      cudaFree(g.stage);
+      g.stage = nullptr;
+      g.stage_bytes = 0;
+    }
+    cudaError_t e = cudaMalloc(&g.stage, need);
+    if (e != cudaSuccess) { cuda_fail(e); return FLURKA_ERR_WORKSPACE; }
+    g.stage_bytes = need;
+  }
+  char* base = (char*)g.stage;
+  char* dQ = base;
+  char* dK = dQ + qb;
+  char* dV = dK + qb;
+  char* dO = dV + qb;
+  char* dE = dO + qb;
+  char* dF = dE + eb;
+  char* dW = dF + eb;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t qn = pr.qkv_elems() * pr.esize(), en = pr.ef_elems() * pr.esize(),
+               wn = pr.w_elems() * pr.esize();
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(dQ, Q, qn, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dK, K, qn, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dV, V, qn, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dE, E, en, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(dF, F, en, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if (wn && (e = cudaMemcpyAsync(dW, W, wn, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(e);
+  rc = flurka_forward(dQ, dK, dV, dE, dF, wn ? dW : nullptr, variant, B, H, N, d, k, m, dO, stream);
+  if (rc) {
+    cudaStreamSynchronize(st);
+    return rc;
+  }
+  if ((e = cudaMemcpyAsync(out, dO, qn, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
+  return FLURKA_OK;
+}
+
+size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m) {
+  Problem pr;
+  if (parse_problem(variant, B, H, N, d, k, m, &pr)) return 0;
+  return make_layout(pr).total;
+}
+
+int flurka_set_workspace(void* dev_ptr, size_t bytes) {
+  if (dev_ptr && ((uintptr_t)dev_ptr & 255)) return FLURKA_ERR_ALIGN;
+  if (dev_ptr && bytes == 0) return FLURKA_ERR_WORKSPACE;
+  g.user_ws = dev_ptr;
+  g.user_ws_bytes = dev_ptr ? bytes : 0;
+  g.have_last = false;
+  return FLURKA_OK;
+}
+
+int flurka_set_path(int path) {
+  const int prev = g.path;
+  if (path == FLURKA_PATH_AUTO || path == FLURKA_PATH_SIMT || path == FLURKA_PATH_TENSOR) g.path = path;
+  return prev;
+}
+
+int flurka_last_path(void) { return g.last_path; }
+int flurka_last_launches(void) { return g.last_launches; }
+
+int flurka_debug_copy(int which, void* dev_dst, size_t bytes, void* stream) {
+  if (!dev_dst) return FLURKA_ERR_NULL;
+  if (!g.have_last) return FLURKA_ERR_WORKSPACE;
+  const Problem& pr = g.last_problem;
+  const Layout L = make_layout(pr);
+  const size_t kd = (size_t)pr.BH() * pr.k * pr.d * 4;
+  size_t off = 0, size = 0;
+  switch (which) {
+    case 0: off = L.kpvp; size = kd; break;
+    case 1: off = L.kpvp + kd; size = kd; break;
+    case 2: off = L.a32; size = (size_t)pr.BH() * pr.p() * pr.d * 4; break;
+    case 3: off = L.weight; size = (size_t)pr.BH() * pr.p() * 4; break;
+    case 4: off = L.status; size = 16; break;
+    default: return FLURKA_ERR_VARIANT;
+  }
+  if (bytes != size) return FLURKA_ERR_SHAPE;
+  cudaError_t e = cudaMemcpyAsync(dev_dst, g.last_ws + off, size, cudaMemcpyDeviceToDevice,
+                                  (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return FLURKA_OK;
+}
+
+int flurka_last_status(void) {
+  if (!g.have_last) return 0;
+  const Layout L = make_layout(g.last_problem);
+  int words[4] = {0, 0, 0, 0};
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaMemcpy(words, g.last_ws + L.status, 16, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return words[0];
+}
+
+int flurka_last_cuda_error(void) { return g.last_cuda_error; }
+
+const char* flurka_strerror(int code) {
+  switch (code) {
+    case FLURKA_OK: return "ok";
+    case FLURKA_ERR_NULL: return "a required pointer is NULL";
+    case FLURKA_ERR_VARIANT: return "unknown kernel variant, element type or selector";
+    case FLURKA_ERR_SHAPE: return "unsupported shape";
+    case FLURKA_ERR_ALIGN: return "pointer not sufficiently aligned";
+    case FLURKA_ERR_WORKSPACE: return "workspace missing, too small or not allocatable";
+    case FLURKA_ERR_CUDA: return "a CUDA call failed (see flurka_last_cuda_error)";
+    case FLURKA_ERR_DEVICE: return "no sm_100 device is current";
+    case FLURKA_ERR_OVERLAP: return "out overlaps an input";
+    default: return "unknown flurka status";
+  }
+}
+
+int flurka_version(void) { return FLURKA_VERSION; }
+
+}  // extern "C"
