@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Throughput of the FLuRKA attention forward pass (tokens/s = B*H*N per second) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config c3] [--impl reference]
+
+One step = one whole forward pass (down-projection, key side, query side) over one synthetic batch.
+Under torchrun every rank runs its own batch on its own GPU (the path shards over B*H with no
+collective), timing is the maximum over ranks, and rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2306_15799_b200 import configs, synth  # noqa: E402
+
+METRIC = "flurka_attn_fwd_tokens_per_s"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.tmp = None
+
+    def start(self):
+        try:
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def oracle_sample(w, inputs, heads):
+    """Times the fp64 oracle (as it stands) on `heads` heads of the workload. Returns seconds."""
+    import oracle
+    f64 = lambda t: t.double().numpy()
+    E, F = f64(inputs["E"]), f64(inputs["F"])
+    W = f64(inputs["W"]) if inputs["W"] is not None else None
+    t0 = time.perf_counter()
+    for i in range(heads):
+        b, h = divmod(i % (w.B * w.H), w.H)
+        oracle.head(f64(inputs["Q"][b, h]), f64(inputs["K"][b, h]), f64(inputs["V"][b, h]), E, F, W, w.variant)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle on the machine's host cores, a bounded sample per step."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    small = configs.shrink(w, B=1, H=1)          # one head per step; E, F, W keep their full size
+    inputs = synth.make_inputs(small)
+    for _ in range(args.warmup):
+        oracle_sample(small, inputs, 1)
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_sample(small, inputs, 1)
+    ms = 1e3 * t / max(args.steps, 1)
+    value = small.N / (ms * 1e-3)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": "one head (N=%d tokens) per step" % small.N},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                         "sample": "one head of %s per step, fp64 C + OpenMP" % w.name},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="c3")
+    ap.add_argument("--impl", default="flurka", choices=["flurka", "reference"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = configs.get(args.config)
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2306_15799_b200 import binding, build
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    binding.load()
+    binding.flurka_set_path({"auto": binding.PATH_AUTO, "simt": binding.PATH_SIMT, "tensor": binding.PATH_TENSOR}[args.path])
+
+    # every rank draws its own batch (weak scaling over B*H); same recipe, rank-offset seed
+    wr = configs.shrink(w, seed=w.seed + 7919 * rank)
+    host = synth.make_inputs(wr)
+    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in host.items()}
+    dev = {n: (t.cuda(non_blocking=True) if t is not None else None) for n, t in pinned.items()}
+    out = torch.empty_like(dev["Q"])
+    host_out = torch.empty_like(pinned["Q"]).pin_memory()
+    in_bytes = sum(t.numel() * t.element_size() for t in dev.values() if t is not None)
+    flush = None
+    if in_bytes < 2 * L2_BYTES:
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+
+    def step():
+        binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant,
+                               out=out, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            step()
+    barrier()
+
+    # ---- timed region: K steps, CUDA events on the launch stream around each step
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    with torch.cuda.stream(stream):
+        for i in range(args.steps):
+            if flush is not None:
+                flush.zero_()
+            starts[i].record(stream)
+            step()
+            stops[i].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
+    total_ms = sum(step_ms)
+    launches = binding.flurka_last_launches() * args.steps
+    path_taken = {1: "simt", 2: "tensor"}.get(binding.flurka_last_path(), "?")
+
+    # ---- per-stage durations (same inputs, events inside the library between the stages)
+    binding.flurka_set_stage_timing(True)
+    stage_ms = [0.0, 0.0, 0.0]
+    with torch.cuda.stream(stream):
+        for _ in range(args.steps):
+            if flush is not None:
+                flush.zero_()
+            step()
+            ms3 = binding.flurka_last_stage_ms()
+            stage_ms = [a + b for a, b in zip(stage_ms, ms3)]
+    binding.flurka_set_stage_timing(False)
+    stage_ms = [x / args.steps for x in stage_ms]
+    torch.cuda.synchronize()
+
+    # ---- end to end: host buffers in, host buffer out, through the host entry point
+    e2e_steps = max(1, min(args.steps, 5))
+    binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
+                                w.variant, out=host_out, stream=stream)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
+                                    w.variant, out=host_out, stream=stream)
+    torch.cuda.synchronize()
+    e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
+    status = binding.flurka_last_status()
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+
+    if rank == 0:
+        peaks = measured_peaks()
+        tokens = w.tokens * world
+        value = tokens / (ms_per_step * 1e-3)
+        flops, byts = w.flops(), w.compulsory_bytes()
+        t_tensor = flops / (peaks["bf16_tflops"] * 1e12)
+        t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+        roof_s = max(t_tensor, t_hbm)
+        # dominant stage and its own roofline (algorithmic work of that stage alone)
+        N, d, k, m, BH, s = w.N, w.d, w.k, w.m, w.B * w.H, w.elem_bytes
+        p = m if w.variant == configs.PERFORMER else d
+        stage_flops = [4 * N * k * d * BH,
+                       (2 * k * d * m + 2 * k * m * d) * BH if w.variant == configs.PERFORMER else 2 * k * d * d * BH,
+                       (2 * N * d * m + 2 * N * m * d) * BH if w.variant == configs.PERFORMER else 2 * N * d * d * BH]
+        stage_bytes = [2 * BH * N * d * s + 2 * k * N * s + 2 * BH * k * d * 4,
+                       2 * BH * k * d * 4 + m * d * s + BH * p * (d * 2 + 4),
+                       2 * BH * N * d * s + m * d * s + BH * p * (d * 2 + 4)]
+        names = ["down_projection", "key_side", "query_side"]
+        dom = max(range(3), key=lambda i: stage_ms[i])
+        dt = stage_ms[dom] * 1e-3
+        tf_t = stage_flops[dom] / (peaks["bf16_tflops"] * 1e12)
+        hb_t = stage_bytes[dom] / (peaks["hbm_gbs"] * 1e9)
+        if hb_t >= tf_t:
+            roofline = {"bound": "hbm", "achieved": stage_bytes[dom] / dt / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            roofline = {"bound": "tensor", "achieved": stage_flops[dom] / dt / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline["traffic"] = None
+        roofline["kernel"] = names[dom]
+        roofline["peak_source"] = "of " + peaks["source"]
+        roofline["stage_ms"] = dict(zip(names, stage_ms))
+
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.io == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": w.name, "variant": "performer" if w.variant == configs.PERFORMER else "rnn",
+                       "B": w.B, "H": w.H, "N": w.N, "d": w.d, "k": w.k, "m": w.m, "io": w.io, "path": path_taken,
+                       "parallelism": "replicated batches over B*H, no collective" if world > 1 else "single GPU",
+                       "l2": "inputs (%.0f MB) exceed L2" % (in_bytes / 1e6) if flush is None
+                             else "L2 flushed between steps (252 MiB write)"},
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
+            "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out.numel() * out.element_size()},
+            "gpu_launches": launches,
+            "roofline": roofline,
+            "path_roofline": {"flops": flops, "bytes": byts, "t_tensor_us": t_tensor * 1e6, "t_hbm_us": t_hbm * 1e6,
+                              "frac": roof_s / (ms_per_step * 1e-3 / 1.0), "peak_source": "of " + peaks["source"]},
+            "step_ms_min": min(step_ms), "step_ms_median": statistics.median(step_ms),
+            "device_status": status,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            import oracle
+            oracle.build()
+            t1 = oracle_sample(wr, host, 1)                        # warm + calibrate
+            heads = max(1, min(w.B * w.H, int(15.0 / max(t1, 1e-3))))
+            tt = oracle_sample(wr, host, heads)
+            line["cpu_baseline"] = {"value": heads * w.N / tt, "unit": UNIT, "cores": oracle.threads(),
+                                    "kind": "oracle",
+                                    "sample": "%d of %d heads of %s, all %d rows each, %.1f s" % (heads, w.B * w.H, w.name, w.N, tt)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -127,6 +127,16 @@ int flurka_last_status(void);
 /* cudaError_t (as int) behind the most recent FLURKA_ERR_CUDA. */
 int flurka_last_cuda_error(void);
 
+/*
+ * Per-stage device timing.  With timing on, flurka_forward records CUDA events on its stream before
+ * and after each of the three stages of Eq. (2): 0 = down-projection (E K, F V), 1 = key side
+ * (phi(K'), phi(K')^T V', phi(K')^T 1), 2 = query side (phi(Q), the product, the division).
+ * flurka_last_stage_ms waits for the last forward and writes the three durations in milliseconds;
+ * it returns FLURKA_ERR_WORKSPACE if that forward ran with timing off.
+ */
+int flurka_set_stage_timing(int on);
+int flurka_last_stage_ms(float* ms3);
+
 /* Static, human-readable text for a flurka_status. */
 const char* flurka_strerror(int code);
 

@@ -1,0 +1,205 @@
+"""ctypes binding of libflurka.so: the same names as include/flurka.h, argument marshalling only.
+
+Every step of the forward pass runs inside the CUDA library.  If the library has not been built
+(``python -m paper_2306_15799_b200.build``) loading raises; there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .configs import PERFORMER, RNN
+
+IO_BF16 = 0x000
+IO_FP32 = 0x100
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+
+EXPORTS = [
+    "flurka_forward", "flurka_forward_host", "flurka_workspace_bytes", "flurka_set_workspace",
+    "flurka_set_path", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
+    "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
+    "flurka_strerror", "flurka_version",
+]
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libflurka.so")
+_lib = None
+
+
+class FlurkaError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        detail = ""
+        if code == -6:
+            detail = " (cudaError %d)" % load().flurka_last_cuda_error()
+        super().__init__("%s failed: %d %s%s" % (what, code, strerror(code), detail))
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load() -> ctypes.CDLL:
+    """Loads libflurka.so and declares the prototypes. Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise FileNotFoundError(
+            "%s not found: build it with `python -m paper_2306_15799_b200.build`" % _LIB_PATH)
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    fwd_args = [vp] * 6 + [ci] * 7 + [vp, vp]
+    lib.flurka_forward.restype = ci
+    lib.flurka_forward.argtypes = fwd_args
+    lib.flurka_forward_host.restype = ci
+    lib.flurka_forward_host.argtypes = fwd_args
+    lib.flurka_workspace_bytes.restype = sz
+    lib.flurka_workspace_bytes.argtypes = [ci] * 7
+    lib.flurka_set_workspace.restype = ci
+    lib.flurka_set_workspace.argtypes = [vp, sz]
+    lib.flurka_set_path.restype = ci
+    lib.flurka_set_path.argtypes = [ci]
+    lib.flurka_last_path.restype = ci
+    lib.flurka_last_launches.restype = ci
+    lib.flurka_debug_copy.restype = ci
+    lib.flurka_debug_copy.argtypes = [ci, vp, sz, vp]
+    lib.flurka_last_status.restype = ci
+    lib.flurka_last_cuda_error.restype = ci
+    lib.flurka_set_stage_timing.restype = ci
+    lib.flurka_set_stage_timing.argtypes = [ci]
+    lib.flurka_last_stage_ms.restype = ci
+    lib.flurka_last_stage_ms.argtypes = [ctypes.POINTER(ctypes.c_float)]
+    lib.flurka_strerror.restype = ctypes.c_char_p
+    lib.flurka_strerror.argtypes = [ci]
+    lib.flurka_version.restype = ci
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().flurka_strerror(code).decode()
+
+
+def version() -> int:
+    return load().flurka_version()
+
+
+def _variant_word(variant: int, dtype: torch.dtype) -> int:
+    if dtype == torch.bfloat16:
+        return variant | IO_BF16
+    if dtype == torch.float32:
+        return variant | IO_FP32
+    raise TypeError("flurka: tensors must be bfloat16 or float32, got %s" % dtype)
+
+
+def _check(Q, K, V, E, F, W, variant, out, device_type):
+    for name, t in (("Q", Q), ("K", K), ("V", V), ("E", E), ("F", F), ("out", out)):
+        if t.device.type != device_type:
+            raise ValueError("flurka: %s must live on %s" % (name, device_type))
+        if not t.is_contiguous():
+            raise ValueError("flurka: %s must be contiguous" % name)
+        if t.dtype != Q.dtype:
+            raise TypeError("flurka: %s has dtype %s, Q has %s" % (name, t.dtype, Q.dtype))
+    if Q.dim() != 4 or K.shape != Q.shape or V.shape != Q.shape or out.shape != Q.shape:
+        raise ValueError("flurka: Q, K, V, out must all be [B,H,N,d]")
+    B, H, N, d = Q.shape
+    if E.dim() != 2 or E.shape[1] != N or F.shape != E.shape:
+        raise ValueError("flurka: E, F must be [k,N]")
+    k = E.shape[0]
+    m = 0
+    if variant == PERFORMER:
+        if W is None or W.dim() != 2 or W.shape[1] != d or W.dtype != Q.dtype or not W.is_contiguous() \
+                or W.device.type != device_type:
+            raise ValueError("flurka: W must be a contiguous [m,d] tensor like Q")
+        m = W.shape[0]
+    return B, H, N, d, k, m
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def flurka_forward(Q, K, V, E, F, W, variant, out=None, stream=None):
+    """O = phi(Q)(phi(EK)^T FV) / phi(Q)(phi(EK)^T 1) on device tensors; asynchronous on `stream`."""
+    if out is None:
+        out = torch.empty_like(Q)
+    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cuda")
+    rc = load().flurka_forward(
+        Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype),
+        B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_forward")
+    return out
+
+
+def flurka_forward_host(Q, K, V, E, F, W, variant, out=None, stream=None):
+    """The same on host (ideally pinned) tensors: copies in, computes, copies out, synchronises."""
+    if out is None:
+        out = torch.empty_like(Q, pin_memory=True)
+    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cpu")
+    rc = load().flurka_forward_host(
+        Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype),
+        B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_forward_host")
+    return out
+
+
+def flurka_workspace_bytes(variant, io_dtype, B, H, N, d, k, m) -> int:
+    return int(load().flurka_workspace_bytes(_variant_word(variant, io_dtype), B, H, N, d, k, m))
+
+
+def flurka_set_workspace(buf) -> None:
+    """buf: a uint8 CUDA tensor the caller keeps alive, or None for the library-owned workspace."""
+    if buf is None:
+        rc = load().flurka_set_workspace(None, 0)
+    else:
+        rc = load().flurka_set_workspace(buf.data_ptr(), buf.numel() * buf.element_size())
+    if rc:
+        raise FlurkaError(rc, "flurka_set_workspace")
+
+
+def flurka_set_path(path: int) -> int:
+    return int(load().flurka_set_path(path))
+
+
+def flurka_last_path() -> int:
+    return int(load().flurka_last_path())
+
+
+def flurka_last_launches() -> int:
+    return int(load().flurka_last_launches())
+
+
+def flurka_last_status() -> int:
+    return int(load().flurka_last_status())
+
+
+def flurka_debug_copy(which: int, shape, dtype=torch.float32, stream=None):
+    """Returns a fresh CUDA tensor holding intermediate `which` of the last forward (see flurka.h)."""
+    dst = torch.empty(shape, dtype=dtype, device="cuda")
+    rc = load().flurka_debug_copy(which, dst.data_ptr(), dst.numel() * dst.element_size(), _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_debug_copy")
+    return dst
+
+
+def flurka_set_stage_timing(on: bool) -> None:
+    rc = load().flurka_set_stage_timing(1 if on else 0)
+    if rc:
+        raise FlurkaError(rc, "flurka_set_stage_timing")
+
+
+def flurka_last_stage_ms():
+    """(down-projection, key side, query side) milliseconds of the last forward run with timing on."""
+    ms = (ctypes.c_float * 3)()
+    rc = load().flurka_last_stage_ms(ms)
+    if rc:
+        raise FlurkaError(rc, "flurka_last_stage_ms")
+    return [float(x) for x in ms]

@@ -64,6 +64,7 @@ struct State {
   // host-buffer entry point: device staging
   void* stage = nullptr;
   size_t stage_bytes = 0;
+  StageTimer timer;
 };
 
 State g;
@@ -199,14 +200,18 @@ int run_simt(const Problem& pr, const Layout& L, char* ws, const void* Q, const 
   float* a32 = (float*)(ws + L.a32);
   cudaError_t e = cudaMemsetAsync(kpvp, 0, (size_t)2 * pr.BH() * pr.k * pr.d * 4, st);
   if (e != cudaSuccess) return cuda_fail(e);
+  g.timer.mark(0, st);
   int rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
   if (rc) return rc;
+  g.timer.mark(1, st);
   rc = key_side_dispatch<T>(pr, kpvp, W, weight, a32, nullptr, st, launches);
   if (rc) return rc;
+  g.timer.mark(2, st);
   rc = pr.kernel == FLURKA_PERFORMER
            ? launch_simt_query_side<T, true>(pr, Q, W, weight, a32, out, st, launches)
            : launch_simt_query_side<T, false>(pr, Q, W, weight, a32, out, st, launches);
   if (rc) return rc;
+  g.timer.mark(3, st);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return FLURKA_OK;
@@ -264,7 +269,7 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
     ta.aT16 = (__half*)(ws + L.aT16);
     ta.status = (int*)(ws + L.status);
     int cuda_err = 0;
-    rc = run_tensor_path(ta, st, &launches, &cuda_err);
+    rc = run_tensor_path(ta, st, g.timer, &launches, &cuda_err);
     if (rc == FLURKA_ERR_CUDA) g.last_cuda_error = cuda_err;
   } else if (pr.fp32) {
     rc = run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
@@ -272,6 +277,7 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
     rc = run_simt<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
   }
   if (rc) return rc;
+  g.timer.have = g.timer.on;
   g.last_path = path;
   g.last_launches = launches;
   g.have_last = true;
@@ -393,6 +399,32 @@ int flurka_last_status(void) {
 }
 
 int flurka_last_cuda_error(void) { return g.last_cuda_error; }
+
+int flurka_set_stage_timing(int on) {
+  if (on) {
+    for (int i = 0; i < 4; ++i) {
+      if (!g.timer.ev[i]) {
+        cudaError_t e = cudaEventCreate(&g.timer.ev[i]);
+        if (e != cudaSuccess) return cuda_fail(e);
+      }
+    }
+  }
+  g.timer.on = on != 0;
+  g.timer.have = false;
+  return FLURKA_OK;
+}
+
+int flurka_last_stage_ms(float* ms3) {
+  if (!ms3) return FLURKA_ERR_NULL;
+  if (!g.timer.have) return FLURKA_ERR_WORKSPACE;
+  cudaError_t e = cudaEventSynchronize(g.timer.ev[3]);
+  if (e != cudaSuccess) return cuda_fail(e);
+  for (int i = 0; i < 3; ++i) {
+    e = cudaEventElapsedTime(&ms3[i], g.timer.ev[i], g.timer.ev[i + 1]);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return FLURKA_OK;
+}
 
 const char* flurka_strerror(int code) {
   switch (code) {

@@ -17,9 +17,19 @@ struct TensorArgs {
   int* status;     // 4 words
 };
 
+// Optional per-stage timing: events recorded on the launch stream around the three stages.
+struct StageTimer {
+  bool on = false;
+  bool have = false;
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  void mark(int i, cudaStream_t st) {
+    if (on && ev[i]) cudaEventRecord(ev[i], st);
+  }
+};
+
 // false while the tensor-core kernels are not compiled into this library
 inline bool tensor_path_built() { return false; }
 
-inline int run_tensor_path(const TensorArgs&, cudaStream_t, int*, int*) { return -3; }
+inline int run_tensor_path(const TensorArgs&, cudaStream_t, StageTimer&, int*, int*) { return -3; }
 
 }  // namespace flurka

@@ -1,0 +1,125 @@
+"""CUDA path against the fp64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2306_15799_b200 import binding, build, configs, synth
+from paper_2306_15799_b200.configs import PERFORMER, RNN, Workload
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    binding.load()
+
+
+def _wl(name, variant, io, B, H, N, d, k, m, seed):
+    return Workload(name, variant, io, B, H, N, d, k, m if variant == PERFORMER else 0, seed)
+
+
+def test_c1_fp32_exact_config():
+    pu.check_all_heads(configs.C1)
+    assert binding.flurka_last_path() == binding.PATH_SIMT
+
+
+SIMT_CASES = [
+    # several tiles in every dimension plus ragged tails
+    _wl("simt_perf_fp32_ragged", PERFORMER, "fp32", 2, 3, 333, 48, 40, 72, 11),
+    _wl("simt_rnn_fp32_ragged", RNN, "fp32", 2, 2, 301, 40, 37, 0, 12),
+    _wl("simt_perf_bf16_ragged", PERFORMER, "bf16", 1, 3, 520, 64, 72, 100, 13),
+    _wl("simt_rnn_bf16", RNN, "bf16", 2, 2, 512, 64, 64, 0, 14),
+    _wl("simt_perf_bf16_d128", PERFORMER, "bf16", 1, 2, 384, 128, 128, 256, 15),
+    # degenerate sizes
+    _wl("simt_perf_n1", PERFORMER, "fp32", 1, 2, 1, 8, 1, 1, 16),
+    _wl("simt_rnn_k1", RNN, "fp32", 1, 1, 65, 1, 1, 0, 17),
+    _wl("simt_perf_d1", PERFORMER, "fp32", 1, 1, 40, 1, 3, 5, 18),
+]
+
+
+@pytest.mark.parametrize("w", SIMT_CASES, ids=lambda w: w.name)
+def test_simt_path_matches_oracle(w):
+    pu.check_all_heads(w, path=binding.PATH_SIMT)
+    assert binding.flurka_last_path() == binding.PATH_SIMT
+    assert binding.flurka_last_launches() == 3
+
+
+def test_intermediates_match_oracle():
+    """K' = E K and V' = F V (Eq. (2)) and the per-feature log-weights, stage by stage."""
+    w = _wl("stage_perf_bf16", PERFORMER, "bf16", 1, 2, 640, 64, 64, 128, 21)
+    inputs = synth.make_inputs(w)
+    pu.run_gpu(w, inputs, binding.PATH_SIMT)
+    Kp = binding.flurka_debug_copy(0, (w.B, w.H, w.k, w.d)).cpu().double().numpy()
+    Vp = binding.flurka_debug_copy(1, (w.B, w.H, w.k, w.d)).cpu().double().numpy()
+    a = binding.flurka_debug_copy(2, (w.B, w.H, w.m, w.d)).cpu().double().numpy()
+    bw = binding.flurka_debug_copy(3, (w.B, w.H, w.m)).cpu().double().numpy()
+    torch.cuda.synchronize()
+    for h in range(w.H):
+        _, inter = pu.oracle_head(inputs, w, 0, h, rows=[0], intermediates=True)
+        assert np.abs(Kp[0, h] - inter["Kp"]).max() < 2e-5 * max(1.0, np.abs(inter["Kp"]).max())
+        assert np.abs(Vp[0, h] - inter["Vp"]).max() < 2e-5 * max(1.0, np.abs(inter["Vp"]).max())
+        # oracle: KV_i = sum_j Phi_ji v'_j, z_i = sum_j Phi_ji  =>  a_i = KV_i / z_i and
+        # b_i - b_i' = log z_i - log z_i' (the global stabiliser drops out of differences)
+        a_ref = inter["KV"] / inter["z"][:, None]
+        big = inter["z"] > 1e-30 * inter["z"].max()
+        assert np.abs(a[0, h][big] - a_ref[big]).max() < 5e-3 * max(1.0, np.abs(a_ref[big]).max())
+        lz = np.log(inter["z"][big])
+        assert np.abs((bw[0, h][big] - bw[0, h][big][0]) - (lz - lz[0])).max() < 5e-3
+
+
+def test_v_ones_gives_equal_columns_within_projection_range():
+    """Convexity invariant (rows of the normalised weights sum to one) on a GPU output."""
+    w = _wl("ones_perf_bf16", PERFORMER, "bf16", 1, 2, 512, 64, 64, 64, 31)
+    inputs = synth.make_inputs(w)
+    inputs["V"] = torch.ones_like(inputs["V"])
+    out = pu.run_gpu(w, inputs).float().cpu()
+    s = inputs["F"].double().sum(dim=1)
+    assert float((out - out[..., :1]).abs().max()) <= 2e-2 * float(s.abs().max())
+    assert out.min() >= s.min() - 2e-2 * s.abs().max() and out.max() <= s.max() + 2e-2 * s.abs().max()
+
+
+def test_host_entry_point_matches_device_entry_point():
+    w = _wl("host_perf_bf16", PERFORMER, "bf16", 1, 2, 512, 64, 64, 64, 41)
+    inputs = synth.make_inputs(w)
+    dev_out = pu.run_gpu(w, inputs).cpu()
+    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in inputs.items()}
+    host_out = binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"],
+                                           pinned["W"], w.variant)
+    assert torch.equal(host_out, dev_out) or float((host_out.float() - dev_out.float()).abs().max()) < 2e-2
+
+
+def test_caller_workspace_and_too_small_workspace():
+    w = _wl("ws_rnn_bf16", RNN, "bf16", 1, 2, 256, 64, 64, 0, 51)
+    inputs = synth.make_inputs(w)
+    need = binding.flurka_workspace_bytes(w.variant, torch.bfloat16, w.B, w.H, w.N, w.d, w.k, w.m)
+    assert need > 0
+    dev = pu.to_device(inputs)
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    binding.flurka_set_workspace(small)
+    try:
+        with pytest.raises(binding.FlurkaError) as ei:
+            binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], None, w.variant)
+        assert ei.value.code == -5
+        buf = torch.empty(need, dtype=torch.uint8, device="cuda")
+        binding.flurka_set_workspace(buf)
+        out = binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], None, w.variant)
+        torch.cuda.synchronize()
+    finally:
+        binding.flurka_set_workspace(None)
+    ref = pu.oracle_head(inputs, w, 0, 1)
+    pu.assert_close(out[0, 1].cpu().double().numpy(), ref, "bf16", "caller workspace")
+
+
+def test_repeated_calls_are_independent():
+    """The workspace is re-zeroed every call: a second call on other data is not polluted."""
+    w1 = _wl("rep_a", PERFORMER, "bf16", 1, 2, 256, 64, 64, 64, 61)
+    w2 = _wl("rep_b", PERFORMER, "bf16", 1, 2, 256, 64, 64, 64, 62)
+    i1, i2 = synth.make_inputs(w1), synth.make_inputs(w2)
+    pu.run_gpu(w1, i1)
+    o2 = pu.run_gpu(w2, i2).cpu().double().numpy()
+    o2b = pu.run_gpu(w2, i2).cpu().double().numpy()
+    pu.assert_close(o2[0, 0], pu.oracle_head(i2, w2, 0, 0), "bf16", "second call")
+    assert np.abs(o2 - o2b).max() <= 2e-2
