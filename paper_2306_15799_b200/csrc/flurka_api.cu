@@ -163,7 +163,7 @@ int launch_simt_key_side(const Problem& pr, const float* kpvp, const void* W, fl
                          __half* aT16, cudaStream_t st, int* launches) {
   const size_t smem = ((size_t)8 * pr.k + 32 * (pr.d + 1)) * 4;
   auto fn = simt_key_side<T, P>;
-  if (smem > 48 * 1024) {
+  if (smem > 24 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e);
   }
@@ -178,6 +178,11 @@ int launch_simt_query_side(const Problem& pr, const void* Q, const void* W, cons
                            const float* a32, void* out, cudaStream_t st, int* launches) {
   const size_t smem = ((size_t)32 * (pr.d + 1) + 32 * pr.d) * 4;
   dim3 grid((pr.N + 31) / 32, pr.BH());
+  if (smem > 24 * 1024) {   // static (16.6 KB) + dynamic may pass the 48 KB default limit
+    cudaError_t e = cudaFuncSetAttribute(simt_query_side<T, P>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   simt_query_side<T, P><<<grid, 256, smem, st>>>((const T*)Q, (const T*)W, weight, a32, (T*)out, pr.N,
                                                  pr.d, pr.p());
   ++*launches;
