@@ -55,7 +55,8 @@ typedef enum {
   FLURKA_ERR_WORKSPACE = -5,   /* caller workspace too small, or the library could not allocate one */
   FLURKA_ERR_CUDA = -6,        /* a CUDA call failed; flurka_last_cuda_error() has the cudaError_t  */
   FLURKA_ERR_DEVICE = -7,      /* no sm_100 device is current                                       */
-  FLURKA_ERR_OVERLAP = -8      /* out overlaps an input                                             */
+  FLURKA_ERR_OVERLAP = -8,     /* out overlaps an input                                             */
+  FLURKA_ERR_TOO_LARGE = -9    /* flurka_forward_static_scratch: scratch need exceeds the built-in array */
 } flurka_status;
 
 /* Execution paths, for flurka_set_path().  AUTO picks the tensor-core path when the shape allows. */
@@ -142,6 +143,36 @@ const char* flurka_strerror(int code);
 
 /* FLURKA_VERSION of the loaded library. */
 int flurka_version(void);
+
+/*
+ * flurka_forward_static_scratch -- flurka_forward for callers that are not allowed to allocate.
+ * (A convenience of this library; the paper has no counterpart.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework whose caching
+ * allocator owns all device memory and forbids side allocations, in a latency-critical serving loop
+ * where an allocation would stall the device, or in a sandboxed plug-in that is only handed finished
+ * buffers.  flurka_forward may call cudaMalloc for its workspace on first use (unless the caller set
+ * one); this entry point never calls cudaMalloc, cudaFree or any allocating routine.  Its scratch
+ * (the fp32 projections K', V', the key-side summaries and a status word) sits in a device array of
+ * FLURKA_STATIC_SCRATCH_BYTES that is compiled into the library, so every GPU that loads the
+ * library carries those bytes until the process exits.
+ *
+ * Arguments, layouts, element types and error codes are those of flurka_forward; inputs and `out`
+ * are still the caller's device buffers.  Differences:
+ *   - a problem whose flurka_workspace_bytes() exceeds FLURKA_STATIC_SCRATCH_BYTES is refused with
+ *     FLURKA_ERR_TOO_LARGE and nothing is launched;
+ *   - it always runs the fp32 CUDA-core kernels (flurka_set_path is ignored), and it does not feed
+ *     flurka_debug_copy / flurka_last_status / flurka_last_path;
+ *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current); make that first call outside any stream capture;
+ *   - all calls share the one array and it keeps what the last call left there.  The call itself
+ *     clears what has to start at zero, but two calls that overlap in time on the GPU (different
+ *     streams, or this one next to another thread's) race on it: serialise them.
+ */
+#define FLURKA_STATIC_SCRATCH_BYTES (8u << 20)
+int flurka_forward_static_scratch(const void* Q, const void* K, const void* V, const void* E,
+                                  const void* F, const void* W, int variant, int B, int H, int N,
+                                  int d, int k, int m, void* out, void* stream);
 
 #ifdef __cplusplus
 }

@@ -20,8 +20,10 @@ EXPORTS = [
     "flurka_forward", "flurka_forward_host", "flurka_workspace_bytes", "flurka_set_workspace",
     "flurka_set_path", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
     "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
-    "flurka_strerror", "flurka_version",
+    "flurka_strerror", "flurka_version", "flurka_forward_static_scratch",
 ]
+
+STATIC_SCRATCH_BYTES = 8 << 20
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libflurka.so")
 _lib = None
@@ -55,6 +57,8 @@ def load() -> ctypes.CDLL:
     lib.flurka_forward.argtypes = fwd_args
     lib.flurka_forward_host.restype = ci
     lib.flurka_forward_host.argtypes = fwd_args
+    lib.flurka_forward_static_scratch.restype = ci
+    lib.flurka_forward_static_scratch.argtypes = fwd_args
     lib.flurka_workspace_bytes.restype = sz
     lib.flurka_workspace_bytes.argtypes = [ci] * 7
     lib.flurka_set_workspace.restype = ci
@@ -203,3 +207,21 @@ def flurka_last_stage_ms():
     if rc:
         raise FlurkaError(rc, "flurka_last_stage_ms")
     return [float(x) for x in ms]
+
+
+def flurka_forward_static_scratch(Q, K, V, E, F, W, variant, out, stream=None):
+    """flurka_forward without any allocation inside the library: scratch is a fixed device array.
+
+    For callers that may not allocate device memory themselves (all memory owned by a framework
+    allocator, latency-critical loops, plug-ins that only receive buffers).  `out` must be passed
+    in; problems needing more than STATIC_SCRATCH_BYTES of scratch raise FlurkaError(-9).
+    Calls share the array, so do not let two of them overlap on the GPU.
+    """
+    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cuda")
+    rc = load().flurka_forward_static_scratch(
+        Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype),
+        B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_forward_static_scratch")
+    return out

@@ -442,6 +442,7 @@ const char* flurka_strerror(int code) {
     case FLURKA_ERR_CUDA: return "a CUDA call failed (see flurka_last_cuda_error)";
     case FLURKA_ERR_DEVICE: return "no sm_100 device is current";
     case FLURKA_ERR_OVERLAP: return "out overlaps an input";
+    case FLURKA_ERR_TOO_LARGE: return "problem needs more scratch than the built-in array holds";
     default: return "unknown flurka status";
   }
 }
@@ -449,3 +450,59 @@ const char* flurka_strerror(int code) {
 int flurka_version(void) { return FLURKA_VERSION; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Forward pass for callers that must not allocate: all scratch lives in a fixed device array that
+// is part of the library image.  In host code `g_static_scratch` is only a handle for the symbol,
+// never a device address; the address kernels may use comes from cudaGetSymbolAddress, looked up
+// once per device with that device current.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[FLURKA_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+char* g_static_scratch_addr[kMaxDevices] = {};
+
+int static_scratch_address(char** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return FLURKA_ERR_DEVICE; }
+  if (dev < 0 || dev >= kMaxDevices) return FLURKA_ERR_DEVICE;
+  if (!g_static_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!ptr) return FLURKA_ERR_WORKSPACE;
+    g_static_scratch_addr[dev] = (char*)ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return FLURKA_OK;
+}
+
+}  // namespace
+
+extern "C" int flurka_forward_static_scratch(const void* Q, const void* K, const void* V, const void* E,
+                                             const void* F, const void* W, int variant, int B, int H,
+                                             int N, int d, int k, int m, void* out, void* stream) {
+  Problem pr;
+  int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
+  if (rc) return rc;
+  rc = validate_pointers(pr, Q, K, V, E, F, W, out);
+  if (rc) return rc;
+  const Layout L = make_layout(pr);
+  if (L.total > (size_t)FLURKA_STATIC_SCRATCH_BYTES) return FLURKA_ERR_TOO_LARGE;
+  rc = check_device();
+  if (rc) return rc;
+  char* ws = nullptr;
+  rc = static_scratch_address(&ws);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  // The array still holds the previous call's contents: the status words are cleared here and
+  // run_simt zeroes the K', V' accumulators before the kernels add into them.
+  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, 16, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  int launches = 0;
+  if (pr.fp32) return run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
+  return run_simt<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
+}
