@@ -63,7 +63,9 @@ typedef enum {
 typedef enum {
   FLURKA_PATH_AUTO = 0,
   FLURKA_PATH_SIMT = 1,   /* fp32 CUDA-core kernels: any shape within the limits, both element types */
-  FLURKA_PATH_TENSOR = 2  /* tcgen05 / TMEM / TMA kernels: bf16 only, shape rules below; else error  */
+  FLURKA_PATH_TENSOR = 2, /* tcgen05 / TMEM / TMA kernels: bf16 only, shape rules below; else error  */
+  FLURKA_PATH_TENSOR_STAGE1 = 3, /* for bisecting: tensor-core down-projection, the rest on CUDA cores */
+  FLURKA_PATH_TENSOR_STAGE3 = 4  /* for bisecting: tensor-core query side, the rest on CUDA cores      */
 } flurka_path_t;
 
 /*
@@ -105,7 +107,11 @@ int flurka_set_workspace(void* dev_ptr, size_t bytes);
 /* Forces an execution path for later calls (flurka_path_t); returns the previous one. */
 int flurka_set_path(int path);
 
-/* The path the most recent successful flurka_forward took (FLURKA_PATH_SIMT or FLURKA_PATH_TENSOR). */
+/* Tuning / test knob: the persistent tensor-core kernels use at most `max_ctas` CTAs (0 = one per SM,
+ * the default), so that small problems still exercise several tiles per CTA. Returns the old limit. */
+int flurka_set_cta_limit(int max_ctas);
+
+/* The path the most recent successful flurka_forward took (never FLURKA_PATH_AUTO). */
 int flurka_last_path(void);
 
 /* Number of kernels the most recent successful flurka_forward launched. */

@@ -14,11 +14,11 @@ from .configs import PERFORMER, RNN
 
 IO_BF16 = 0x000
 IO_FP32 = 0x100
-PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_STAGE1, PATH_TENSOR_STAGE3 = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "flurka_forward", "flurka_forward_host", "flurka_workspace_bytes", "flurka_set_workspace",
-    "flurka_set_path", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
+    "flurka_set_path", "flurka_set_cta_limit", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
     "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
     "flurka_strerror", "flurka_version", "flurka_forward_static_scratch",
 ]
@@ -65,6 +65,8 @@ def load() -> ctypes.CDLL:
     lib.flurka_set_workspace.argtypes = [vp, sz]
     lib.flurka_set_path.restype = ci
     lib.flurka_set_path.argtypes = [ci]
+    lib.flurka_set_cta_limit.restype = ci
+    lib.flurka_set_cta_limit.argtypes = [ci]
     lib.flurka_last_path.restype = ci
     lib.flurka_last_launches.restype = ci
     lib.flurka_debug_copy.restype = ci
@@ -171,6 +173,10 @@ def flurka_set_workspace(buf) -> None:
 
 def flurka_set_path(path: int) -> int:
     return int(load().flurka_set_path(path))
+
+
+def flurka_set_cta_limit(max_ctas: int) -> int:
+    return int(load().flurka_set_cta_limit(max_ctas))
 
 
 def flurka_last_path() -> int:

@@ -65,6 +65,7 @@ struct State {
   void* stage = nullptr;
   size_t stage_bytes = 0;
   StageTimer timer;
+  TensorMaps maps;
 };
 
 State g;
@@ -197,29 +198,54 @@ int key_side_dispatch(const Problem& pr, const float* kpvp, const void* W, float
              : launch_simt_key_side<T, false>(pr, kpvp, W, weight, a32, aT16, st, launches);
 }
 
+// The three stages in order.  tc1 / tc3 choose the tensor-core kernel for stage 1 / stage 3
+// (bf16 only); stage 2 is the CUDA-core kernel on every path.
 template <typename T>
-int run_simt(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
-             const void* E, const void* F, const void* W, void* out, cudaStream_t st, int* launches) {
+int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
+                 const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc3,
+                 int* launches) {
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
   float* a32 = (float*)(ws + L.a32);
+  __half* aT16 = (__half*)(ws + L.aT16);
+  int* status = (int*)(ws + L.status);
+  const bool performer = pr.kernel == FLURKA_PERFORMER;
+  int cuda_err = 0;
   cudaError_t e = cudaMemsetAsync(kpvp, 0, (size_t)2 * pr.BH() * pr.k * pr.d * 4, st);
   if (e != cudaSuccess) return cuda_fail(e);
   g.timer.mark(0, st);
-  int rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
-  if (rc) return rc;
+  int rc;
+  if (tc1) {
+    rc = launch_k1(g.maps, K, V, E, F, kpvp, pr.BH(), pr.N, pr.d, pr.k, status, st, &cuda_err);
+    if (rc) { g.last_cuda_error = cuda_err; return rc; }
+    ++*launches;
+  } else {
+    rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
+    if (rc) return rc;
+  }
   g.timer.mark(1, st);
-  rc = key_side_dispatch<T>(pr, kpvp, W, weight, a32, nullptr, st, launches);
+  rc = key_side_dispatch<T>(pr, kpvp, W, weight, tc3 ? nullptr : a32, tc3 ? aT16 : nullptr, st, launches);
   if (rc) return rc;
   g.timer.mark(2, st);
-  rc = pr.kernel == FLURKA_PERFORMER
-           ? launch_simt_query_side<T, true>(pr, Q, W, weight, a32, out, st, launches)
-           : launch_simt_query_side<T, false>(pr, Q, W, weight, a32, out, st, launches);
-  if (rc) return rc;
+  if (tc3) {
+    rc = launch_k3(g.maps, performer, Q, W, aT16, weight, out, pr.BH(), pr.N, pr.d, pr.p(), status, st, &cuda_err);
+    if (rc) { g.last_cuda_error = cuda_err; return rc; }
+    ++*launches;
+  } else {
+    rc = performer ? launch_simt_query_side<T, true>(pr, Q, W, weight, a32, out, st, launches)
+                   : launch_simt_query_side<T, false>(pr, Q, W, weight, a32, out, st, launches);
+    if (rc) return rc;
+  }
   g.timer.mark(3, st);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return FLURKA_OK;
+}
+
+template <typename T>
+int run_simt(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
+             const void* E, const void* F, const void* W, void* out, cudaStream_t st, int* launches) {
+  return run_pipeline<T>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, launches);
 }
 
 int validate_pointers(const Problem& pr, const void* Q, const void* K, const void* V, const void* E,
@@ -251,7 +277,7 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
   if (rc) return rc;
   int path = g.path;
   const bool tensor_ok = tensor_path_ok(pr);
-  if (path == FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
+  if (path >= FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
   if (path == FLURKA_PATH_AUTO) path = tensor_ok ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
   rc = check_device();
   if (rc) return rc;
@@ -264,22 +290,12 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
   cudaError_t e = cudaMemsetAsync(ws + L.status, 0, 16, st);
   if (e != cudaSuccess) return cuda_fail(e);
 
-  if (path == FLURKA_PATH_TENSOR) {
-    TensorArgs ta;
-    ta.kernel = pr.kernel; ta.B = pr.B; ta.H = pr.H; ta.N = pr.N; ta.d = pr.d; ta.k = pr.k; ta.m = pr.m;
-    ta.Q = Q; ta.K = K; ta.V = V; ta.E = E; ta.F = F; ta.W = W; ta.out = out;
-    ta.kpvp = (float*)(ws + L.kpvp);
-    ta.weight = (float*)(ws + L.weight);
-    ta.a32 = (float*)(ws + L.a32);
-    ta.aT16 = (__half*)(ws + L.aT16);
-    ta.status = (int*)(ws + L.status);
-    int cuda_err = 0;
-    rc = run_tensor_path(ta, st, g.timer, &launches, &cuda_err);
-    if (rc == FLURKA_ERR_CUDA) g.last_cuda_error = cuda_err;
-  } else if (pr.fp32) {
+  if (pr.fp32) {
     rc = run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
   } else {
-    rc = run_simt<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
+    const bool tc1 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE1;
+    const bool tc3 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE3;
+    rc = run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, tc1, tc3, &launches);
   }
   if (rc) return rc;
   g.timer.have = g.timer.on;
@@ -363,7 +379,13 @@ int flurka_set_workspace(void* dev_ptr, size_t bytes) {
 
 int flurka_set_path(int path) {
   const int prev = g.path;
-  if (path == FLURKA_PATH_AUTO || path == FLURKA_PATH_SIMT || path == FLURKA_PATH_TENSOR) g.path = path;
+  if (path >= FLURKA_PATH_AUTO && path <= FLURKA_PATH_TENSOR_STAGE3) g.path = path;
+  return prev;
+}
+
+int flurka_set_cta_limit(int max_ctas) {
+  const int prev = cta_limit();
+  cta_limit() = max_ctas > 0 ? max_ctas : 0;
   return prev;
 }
 

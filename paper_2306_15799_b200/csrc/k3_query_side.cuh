@@ -1,0 +1,419 @@
+// Stage 3 on tensor cores: the query feature map, the associative product and the row division
+// (arxiv 2306.15799, Eq. (2); normalisation as in Appendix D), one pass over Q.
+//
+//   PERFORMER   S = Q W^T + 1 b^T      (tcgen05, bf16 x bf16 -> fp32 in TMEM; b_i rides along as
+//                                        three bf16 terms in one extra 16-wide contraction step)
+//               p = exp(S - rowmax S)   (two passes over TMEM by the thread that owns the row)
+//               O = (p a) / sum_i p_i   (p as fp16 back into TMEM, tcgen05 with A from TMEM,
+//                                        a^T resident in shared memory)
+//   RNN         p = (elu(q) + 1) z / max z  straight from the Q tile, then the same second product.
+//
+// The per-feature summaries a_i, b_i (or z_i) come from stage 2.  A persistent CTA walks a
+// contiguous range of 128-row tiles; warp 0 feeds TMA, warp 1 issues MMAs, warp 2 rebuilds the
+// bias operand when the head changes, and two groups of four warps alternate tiles (TMEM is
+// split in two 256-column halves: S/p in columns 0.., O in columns 128.. of each half).
+// The bf16 output tile is staged in the tile's own Q buffer and leaves through TMA.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "tc_common.cuh"
+
+namespace flurka {
+
+struct K3Params {
+  int N, d, p, BH;          // p = feature dimension (m, or d for RNN)
+  int tiles_per_head;       // N / 128
+  int total_tiles;
+  const float* weight;      // [BH][p]  b_i or z_i
+  int* status;
+};
+
+constexpr int kK3Threads = 384;
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// shared-memory plan (bytes, from a 1024-aligned base); see k3_smem_bytes()
+struct K3Smem {
+  uint32_t w, ones, bias, aT, q, scale, bars, total;
+  int q_stages;
+};
+
+__host__ __device__ inline K3Smem k3_smem_plan(int d, int p, bool performer) {
+  K3Smem s;
+  uint32_t off = 0;
+  s.w = off;    off += performer ? (uint32_t)p * d * 2 : 0;        // W: d/64 K-blocks of [p rows x 128 B]
+  s.ones = off; off += performer ? 4096 : 0;                       // [128 x 16] bf16, no swizzle
+  s.bias = off; off += performer ? 8192 : 0;                       // [256 x 16] bf16, no swizzle
+  s.aT = off;   off += (uint32_t)d * p * 2;                        // a^T: p/64 K-blocks of [d rows x 128 B]
+  s.aT = (s.aT + 1023u) & ~1023u;
+  off = s.aT + (uint32_t)d * p * 2;
+  off = (off + 1023u) & ~1023u;
+  s.q_stages = (d == 64) ? 3 : 2;
+  s.q = off;    off += (uint32_t)s.q_stages * 128 * d * 2;
+  s.scale = off; off += 1024;                                      // RNN: z_i / max z as floats
+  s.bars = off; off += 256;
+  s.total = off + 1024;                                            // alignment slack
+  return s;
+}
+
+template <bool kPerformer>
+__global__ void __launch_bounds__(kK3Threads, 1)
+k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmW,
+              const __grid_constant__ CUtensorMap tmAT, const __grid_constant__ CUtensorMap tmO,
+              const K3Params prm) {
+  using namespace tc;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const int d = prm.d, p = prm.p;
+  const K3Smem L = k3_smem_plan(d, p, kPerformer);
+  const int NS = L.q_stages;
+  const uint32_t q_stage_bytes = 128u * d * 2u;
+
+  // barriers
+  const uint32_t bars = base + L.bars;
+  const uint32_t bar_qfull = bars;            // [3]
+  const uint32_t bar_qempty = bars + 24;      // [3]
+  const uint32_t bar_sfull = bars + 48;       // [2]   S ready in TMEM (PERFORMER)
+  const uint32_t bar_pfull = bars + 64;       // [2]   p written to TMEM by the 128 row owners
+  const uint32_t bar_ofull = bars + 80;       // [2]   O ready in TMEM
+  const uint32_t bar_sfree = bars + 96;       // [2]   TMEM half read out, may be overwritten
+  const uint32_t bar_wfull = bars + 112;      //       W resident
+  const uint32_t bar_drained = bars + 120;    //       every MMA of the previous head is complete
+  const uint32_t bar_atfull = bars + 128;     //       a^T of the new head resident
+  const uint32_t bar_biasready = bars + 136;  //       bias operand / scale vector of the new head built
+  const uint32_t tmem_slot = bars + 192;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_shared;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // contiguous range of tiles for this CTA
+  const int t_begin = (int)(((long long)blockIdx.x * prm.total_tiles) / gridDim.x);
+  const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.total_tiles) / gridDim.x);
+  const int ntiles = t_end - t_begin;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < 3; ++i) {
+      mbar_init(bar_qfull + 8 * i, 1);
+      mbar_init(bar_qempty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_sfull + 8 * i, 1);
+      mbar_init(bar_pfull + 8 * i, 128);
+      mbar_init(bar_ofull + 8 * i, 1);
+      mbar_init(bar_sfree + 8 * i, 128);
+    }
+    mbar_init(bar_wfull, 1);
+    mbar_init(bar_drained, 1);
+    mbar_init(bar_atfull, 1);
+    mbar_init(bar_biasready, 32);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  if (kPerformer && warp == 2) {
+    // the all-ones A operand of the bias step: row r, column c (c < 16), no swizzle:
+    // offset = (r/8)*256 + (c/8)*128 + (r%8)*16 + (c%8)*2; columns 0..2 are 1, the rest 0
+    __nv_bfloat16* ones = reinterpret_cast<__nv_bfloat16*>(base_ptr + L.ones);
+    for (int e = lane; e < 128 * 16; e += 32) {
+      const int r = e >> 4, c = e & 15;
+      const int off = (r >> 3) * 128 + (c >> 3) * 64 + (r & 7) * 8 + (c & 7);
+      ones[off] = __float2bfloat16_rn(c < 3 ? 1.f : 0.f);
+    }
+    fence_proxy_async_smem();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  if (threadIdx.x == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_shared = v;
+  }
+  __syncthreads();
+  const uint32_t tmem = tmem_base_shared;
+
+  const int kq = d >> 6;      // 64-wide K-blocks of the Q / W tiles
+  const int kp = p >> 6;      // 64-wide K-blocks of a^T
+
+  if (ntiles > 0) {
+    if (warp == 0 && lane == 0) {
+      // ============================================================ TMA producer
+      prefetch_tmap(&tmQ);
+      prefetch_tmap(&tmAT);
+      prefetch_tmap(&tmO);
+      bool ok = true;
+      if (kPerformer) {
+        prefetch_tmap(&tmW);
+        mbar_arrive_expect_tx(bar_wfull, (uint32_t)p * d * 2);
+        for (int kb = 0; kb < kq; ++kb) tma_load_2d(base + L.w + kb * (p * 128), &tmW, bar_wfull, kb * 64, 0);
+      }
+      int head_prev = -1, events = 0;
+      int issued = 0;
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int tile = t_begin + i;
+        const int head = tile / prm.tiles_per_head;
+        const int row0 = (tile % prm.tiles_per_head) * 128;
+        if (head != head_prev) {
+          if (events > 0) ok = mbar_wait(bar_drained, (events - 1) & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(bar_atfull, (uint32_t)d * p * 2);
+          for (int kb = 0; kb < kp; ++kb) tma_load_3d(base + L.aT + kb * (d * 128), &tmAT, bar_atfull, kb * 64, 0, head);
+          head_prev = head;
+          ++events;
+        }
+        const int st = i % NS;
+        if (i >= NS) ok = mbar_wait(bar_qempty + 8 * st, ((i / NS) - 1) & 1, prm.status, &abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(bar_qfull + 8 * st, q_stage_bytes);
+        for (int kb = 0; kb < kq; ++kb)
+          tma_load_3d(base + L.q + st * q_stage_bytes + kb * 16384, &tmQ, bar_qfull + 8 * st, kb * 64, row0, head);
+        ++issued;
+      }
+      if (!ok) {
+        for (int i = max(0, issued - NS); i < issued; ++i)
+          (void)mbar_wait(bar_qfull + 8 * (i % NS), (i / NS) & 1, prm.status, &abort_flag);
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ============================================================ MMA issuer
+      const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, (uint32_t)p);   // S = Q W^T (+ bias step)
+      const uint32_t idesc2 = make_idesc(kFmtF16, 0, 0, 128, (uint32_t)d);    // O = p a
+      bool ok = true;
+      if (kPerformer) ok = mbar_wait(bar_wfull, 0, prm.status, &abort_flag);
+      int head_prev = -1, events = 0;
+      // second product of tile j (j = i-1 inside the loop, the last tile after it)
+      auto second_product = [&](int j) -> bool {
+        const int buf = j & 1;
+        if (!mbar_wait(bar_pfull + 8 * buf, (j >> 1) & 1, prm.status, &abort_flag)) return false;
+        tcgen05_fence_after();
+        const uint32_t tb = tmem + buf * 256;
+        const int ksteps = p >> 4;
+        for (int ks = 0; ks < ksteps; ++ks) {
+          const uint64_t bd = make_sdesc(base + L.aT + (ks >> 2) * (d * 128) + (ks & 3) * 32, 16, 1024, kSwizzle128);
+          mma_ts(tb + 128, tb + ks * 8, bd, idesc2, ks > 0 ? 1u : 0u);
+        }
+        mma_commit(bar_ofull + 8 * buf);
+        return true;
+      };
+      int pending = -1;     // tile whose second product has not been issued yet
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int head = (t_begin + i) / prm.tiles_per_head;
+        const int buf = i & 1, st = i % NS;
+        if (head != head_prev) {
+          if (events > 0) {
+            // drain: the old head's operands stay in use until its last second product completes
+            if (pending >= 0) { ok = second_product(pending); pending = -1; if (!ok) break; }
+            mma_commit(bar_drained);
+          }
+          ok = mbar_wait(bar_atfull, events & 1, prm.status, &abort_flag);
+          if (ok) ok = mbar_wait(bar_biasready, events & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          head_prev = head;
+          ++events;
+        }
+        if (kPerformer) {
+          // TMEM half `buf` must have been read out by the epilogue of tile i-2
+          if (i >= 2) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> 1) - 1) & 1, prm.status, &abort_flag);
+          if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          tcgen05_fence_after();
+          const uint32_t tb = tmem + buf * 256;
+          const uint32_t qb = base + L.q + st * q_stage_bytes;
+          const int ksteps = d >> 4;
+          for (int ks = 0; ks < ksteps; ++ks) {
+            const uint64_t ad = make_sdesc(qb + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128);
+            const uint64_t bd = make_sdesc(base + L.w + (ks >> 2) * (p * 128) + (ks & 3) * 32, 16, 1024, kSwizzle128);
+            mma_ss(tb, ad, bd, idesc1, ks > 0 ? 1u : 0u);
+          }
+          {
+            // bias step: ones[128 x 16] (columns 0..2 = 1) times bias[p x 16] (b split in three bf16)
+            const uint64_t ad = make_sdesc(base + L.ones, 128, 256, kSwizzleNone);
+            const uint64_t bd = make_sdesc(base + L.bias, 128, 256, kSwizzleNone);
+            mma_ss(tb, ad, bd, idesc1, 1u);
+          }
+          mma_commit(bar_sfull + 8 * buf);
+        }
+        // the second product of the previous tile goes after the first product of this one, so the
+        // row owners of this tile can start while the previous tile's output is still being formed
+        if (pending >= 0) { ok = second_product(pending); if (!ok) break; }
+        pending = i;
+      }
+      if (ok && pending >= 0) (void)second_product(pending);
+    } else if (warp == 2) {
+      // ============================================================ per-head operand builder
+      int head_prev = -1, events = 0;
+      bool ok = true;
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int head = (t_begin + i) / prm.tiles_per_head;
+        if (head == head_prev) continue;
+        if (events > 0) ok = mbar_wait(bar_drained, (events - 1) & 1, prm.status, &abort_flag);
+        if (!ok) break;
+        const float* wv = prm.weight + (size_t)head * p;
+        float mx = -INFINITY;
+        for (int f = lane; f < p; f += 32) mx = fmaxf(mx, wv[f]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (kPerformer) {
+          // bias[f][c], c < 16, no swizzle: offset = (f/8)*256 + (c/8)*128 + (f%8)*16 + (c%8)*2 bytes
+          __nv_bfloat16* bias = reinterpret_cast<__nv_bfloat16*>(base_ptr + L.bias);
+          for (int f = lane; f < 256; f += 32) {
+            float b = (f < p) ? wv[f] - mx : 0.f;
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(b);  b -= __bfloat162float(h0);
+            const __nv_bfloat16 h1 = __float2bfloat16_rn(b);  b -= __bfloat162float(h1);
+            const __nv_bfloat16 h2 = __float2bfloat16_rn(b);
+            __nv_bfloat16* row = bias + (f >> 3) * 128 + (f & 7) * 8;
+            row[0] = h0; row[1] = h1; row[2] = h2;
+#pragma unroll
+            for (int c = 3; c < 8; ++c) row[c] = __float2bfloat16_rn(0.f);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) row[64 + c] = __float2bfloat16_rn(0.f);
+          }
+          fence_proxy_async_smem();
+        } else {
+          float* sc = reinterpret_cast<float*>(base_ptr + L.scale);
+          const float inv = 1.f / mx;
+          for (int f = lane; f < p; f += 32) sc[f] = wv[f] * inv;
+        }
+        mbar_arrive(bar_biasready);
+        head_prev = head;
+        ++events;
+      }
+    } else if (warp >= 4) {
+      // ============================================================ row owners (two groups of 4 warps)
+      const int grp = (warp - 4) >> 2;                 // tiles with (i & 1) == grp
+      const int q4 = warp & 3;                         // TMEM lane quadrant
+      const int row = q4 * 32 + lane;                  // row of the tile this thread owns
+      const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+      const float kLog2e = 1.4426950408889634f;
+      int head_prev = -1, events = 0;
+      bool ok = true;
+      for (int i = grp; i < ntiles && ok; i += 2) {
+        const int tile = t_begin + i;
+        const int head = tile / prm.tiles_per_head;
+        const int row0 = (tile % prm.tiles_per_head) * 128;
+        const int buf = i & 1, st = i % NS;
+        const uint32_t tb = tmem + buf * 256 + lane_off;
+        const uint32_t qb = base + L.q + st * q_stage_bytes;
+        float denom = 0.f;
+        // count head changes the same way the other roles do (both groups see every tile index)
+        for (int j = (i >= 2 ? i - 1 : 0); j <= i; ++j) {
+          const int hj = (t_begin + j) / prm.tiles_per_head;
+          if (hj != head_prev) { head_prev = hj; ++events; }
+        }
+        if (kPerformer) {
+          ok = mbar_wait(bar_sfull + 8 * buf, (i >> 1) & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          tcgen05_fence_after();
+          // pass 1: row maximum
+          float mx = -INFINITY;
+          for (int c = 0; c < p; c += 32) {
+            uint32_t r[32];
+            tmem_ld32(tb + c, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+          }
+          const float shift = mx * kLog2e;
+          // pass 2: p = 2^(S log2e - shift), fp16 pairs back into columns [c/2, c/2+16)
+          for (int c = 0; c < p; c += 32) {
+            uint32_t r[32], h[16];
+            tmem_ld32(tb + c, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float e0 = ex2_approx(fmaf(__uint_as_float(r[2 * e]), kLog2e, -shift));
+              const float e1 = ex2_approx(fmaf(__uint_as_float(r[2 * e + 1]), kLog2e, -shift));
+              denom += e0 + e1;
+              const __half2 hh = __floats2half2_rn(e0, e1);
+              h[e] = *reinterpret_cast<const uint32_t*>(&hh);
+            }
+            tmem_st16(tb + (c >> 1), h);
+          }
+        } else {
+          // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
+          if (i >= 2) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> 1) - 1) & 1, prm.status, &abort_flag);
+          if (ok) ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
+          if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          const float* sc = reinterpret_cast<const float*>(base_ptr + L.scale);
+          for (int c = 0; c < d; c += 32) {
+            uint32_t h[16];
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+              const int col = c + ch * 8;
+              const uint32_t a = qb + (col >> 6) * 16384 + row * 128 + ((((col & 63) >> 3) ^ (row & 7)) << 4);
+              uint32_t v[4];
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                           : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(a));
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 qq = *reinterpret_cast<const __nv_bfloat162*>(&v[e]);
+                const float x0 = __bfloat162float(qq.x), x1 = __bfloat162float(qq.y);
+                const float f0 = (x0 > 0.f ? x0 + 1.f : __expf(x0)) * sc[col + 2 * e];
+                const float f1 = (x1 > 0.f ? x1 + 1.f : __expf(x1)) * sc[col + 2 * e + 1];
+                denom += f0 + f1;
+                const __half2 hh = __floats2half2_rn(f0, f1);
+                h[ch * 4 + e] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+            }
+            tmem_st16(tb + (c >> 1), h);
+          }
+        }
+        tmem_wait_st();
+        tcgen05_fence_before();
+        mbar_arrive(bar_pfull + 8 * buf);
+
+        // ---- epilogue of this tile: O / denom -> bf16 -> the tile's Q buffer -> TMA store
+        ok = mbar_wait(bar_ofull + 8 * buf, (i >> 1) & 1, prm.status, &abort_flag);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const float inv = 1.f / fmaxf(denom, 1.17549435e-38f);
+        for (int c = 0; c < d; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tb + 128 + c, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t v[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(r[ch * 8 + 2 * e]) * inv,
+                                                              __uint_as_float(r[ch * 8 + 2 * e + 1]) * inv);
+              v[e] = *reinterpret_cast<const uint32_t*>(&o2);
+            }
+            const int col = c + ch * 8;
+            const uint32_t a = qb + (col >> 6) * 16384 + row * 128 + ((((col & 63) >> 3) ^ (row & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3])
+                         : "memory");
+          }
+        }
+        tcgen05_fence_before();
+        mbar_arrive(bar_sfree + 8 * buf);               // this TMEM half may be overwritten now
+        fence_proxy_async_smem();
+        named_barrier_sync(1 + grp, 128);
+        if (q4 == 0 && lane == 0) {
+          for (int kb = 0; kb < kq; ++kb) tma_store_3d(&tmO, qb + kb * 16384, kb * 64, row0, head);
+          bulk_commit_group();
+          bulk_wait_group_read0();
+          mbar_arrive(bar_qempty + 8 * st);             // the Q buffer may be refilled
+        }
+      }
+      if (q4 == 0 && lane == 0) bulk_wait_group0();
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace flurka

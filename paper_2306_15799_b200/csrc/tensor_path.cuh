@@ -1,21 +1,15 @@
-// Tensor-core (tcgen05 / TMEM / TMA) path of the FLuRKA forward pass: interface to the host side.
+// Host side of the tensor-core (tcgen05 / TMEM / TMA) kernels: tensor-map encoding and launches.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
+#include <string.h>
+
+#include "k1_down_project.cuh"
+#include "k3_query_side.cuh"
 
 namespace flurka {
-
-struct TensorArgs {
-  int kernel, B, H, N, d, k, m;
-  const void *Q, *K, *V, *E, *F, *W;
-  void* out;
-  float* kpvp;     // [2][BH][k][d] fp32
-  float* weight;   // [BH][p]
-  float* a32;      // [BH][p][d]
-  __half* aT16;    // [BH][d][p]
-  int* status;     // 4 words
-};
 
 // Optional per-stage timing: events recorded on the launch stream around the three stages.
 struct StageTimer {
@@ -27,9 +21,172 @@ struct StageTimer {
   }
 };
 
-// false while the tensor-core kernels are not compiled into this library
-inline bool tensor_path_built() { return false; }
+inline bool tensor_path_built() { return true; }
 
-inline int run_tensor_path(const TensorArgs&, cudaStream_t, StageTimer&, int*, int*) { return -3; }
+// ---------------------------------------------------------------------------------------------
+// cuTensorMapEncodeTiled is fetched from the driver at run time, so the library links against
+// the CUDA runtime only and still loads on machines without a driver.
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess) {
+      (void)cudaGetLastError();
+      return nullptr;
+    }
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// A tensor map together with the arguments it was built from (re-encoded only when they change).
+struct CachedMap {
+  CUtensorMap map;
+  const void* ptr = nullptr;
+  unsigned long long key[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  bool valid = false;
+};
+
+// rank <= 3; dims/box in elements (innermost first); 128-byte swizzle; out-of-range reads give zero.
+inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int rank, const void* ptr,
+                       const unsigned long long* dims, const unsigned* box) {
+  unsigned long long key[8] = {(unsigned long long)dt, (unsigned long long)rank, dims[0], dims[1],
+                               rank > 2 ? dims[2] : 1ull, box[0], box[1], rank > 2 ? box[2] : 1u};
+  if (cm->valid && cm->ptr == ptr && memcmp(key, cm->key, sizeof(key)) == 0) return true;
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3] = {dims[0], dims[1], rank > 2 ? dims[2] : 1};
+  cuuint64_t gstride[2] = {dims[0] * (cuuint64_t)esize, dims[0] * dims[1] * (cuuint64_t)esize};
+  cuuint32_t bdim[3] = {box[0], box[1], rank > 2 ? box[2] : 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(&cm->map, dt, (cuuint32_t)rank, const_cast<void*>(ptr), gdim, gstride, bdim, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { cm->valid = false; return false; }
+  cm->ptr = ptr;
+  memcpy(cm->key, key, sizeof(key));
+  cm->valid = true;
+  return true;
+}
+
+struct TensorMaps {
+  CachedMap E, F, K, V, kpvp, Q, W, aT, O;
+};
+
+// 0 = use every SM; otherwise the persistent kernels are launched with at most this many CTAs
+inline int& cta_limit() {
+  static int limit = 0;
+  return limit;
+}
+
+inline int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  const int lim = cta_limit();
+  return (lim > 0 && lim < n) ? lim : n;
+}
+
+// Sequence splits of stage 1: fill whole waves of CTAs with 12..48 chunks of 64 positions each.
+inline int k1_choose_nsplit(int units, int chunks) {
+  const int sms = sm_count();
+  int best = 1;
+  for (int w = 1; w <= 8; ++w) {
+    int ns = (sms * w) / units;
+    if (ns < 1) ns = 1;
+    if (ns > chunks) ns = chunks;
+    best = ns;
+    if (chunks / ns <= 48) break;
+  }
+  return best;
+}
+
+// ---- stage 1: K' = E K, V' = F V into kpvp (already zeroed) ----------------------------------
+inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E, const void* F, float* kpvp,
+                     int BH, int N, int d, int k, int* status, cudaStream_t st, int* cuda_err) {
+  const unsigned long long dE[2] = {(unsigned long long)N, (unsigned long long)k};
+  const unsigned bE[2] = {64, 128};
+  const unsigned long long dX[3] = {(unsigned long long)d, (unsigned long long)N, (unsigned long long)BH};
+  const unsigned bX[3] = {64, 64, 1};
+  const unsigned long long dO[3] = {(unsigned long long)d, (unsigned long long)k, (unsigned long long)2 * BH};
+  const unsigned bO[3] = {32, 32, 1};
+  if (!encode_map(&tm.E, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, E, dE, bE) ||
+      !encode_map(&tm.F, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, F, dE, bE) ||
+      !encode_map(&tm.K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, K, dX, bX) ||
+      !encode_map(&tm.V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, V, dX, bX) ||
+      !encode_map(&tm.kpvp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 3, kpvp, dO, bO)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  K1Params p;
+  p.N = N; p.d = d; p.k = k; p.BH = BH;
+  p.col_groups = (BH * d + 255) / 256;
+  p.k_halves = (k + 255) / 256;
+  p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, N / 64);
+  p.status = status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k1_down_project, cudaFuncAttributeMaxDynamicSharedMemorySize, kK1SmemBytes);
+    if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+    attr_set = true;
+  }
+  const int grid = 2 * p.k_halves * p.col_groups * p.nsplit;
+  k1_down_project<<<grid, kK1Threads, kK1SmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
+
+// ---- stage 3: O from Q, W and the key-side summaries ------------------------------------------
+inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* W, const __half* aT16,
+                     const float* weight, void* out, int BH, int N, int d, int p, int* status, cudaStream_t st,
+                     int* cuda_err) {
+  const unsigned long long dQ[3] = {(unsigned long long)d, (unsigned long long)N, (unsigned long long)BH};
+  const unsigned bQ[3] = {64, 128, 1};
+  const unsigned long long dA[3] = {(unsigned long long)p, (unsigned long long)d, (unsigned long long)BH};
+  const unsigned bA[3] = {64, (unsigned)d, 1};
+  if (!encode_map(&tm.Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Q, dQ, bQ) ||
+      !encode_map(&tm.O, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, out, dQ, bQ) ||
+      !encode_map(&tm.aT, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, 3, aT16, dA, bA)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  if (performer) {
+    const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
+    const unsigned bW[2] = {64, (unsigned)p};
+    if (!encode_map(&tm.W, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW)) {
+      *cuda_err = (int)cudaErrorInvalidValue;
+      return -6;
+    }
+  }
+  K3Params prm;
+  prm.N = N; prm.d = d; prm.p = p; prm.BH = BH;
+  prm.tiles_per_head = N / 128;
+  prm.total_tiles = prm.tiles_per_head * BH;
+  prm.weight = weight;
+  prm.status = status;
+  const K3Smem L = k3_smem_plan(d, p, performer);
+  auto fn = performer ? k3_query_side<true> : k3_query_side<false>;
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  int grid = sm_count();
+  if (grid > prm.total_tiles) grid = prm.total_tiles;
+  // the RNN kernel ignores tmW; pass any valid map
+  fn<<<grid, kK3Threads, L.total, st>>>(tm.Q.map, performer ? tm.W.map : tm.Q.map, tm.aT.map, tm.O.map, prm);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
 
 }  // namespace flurka

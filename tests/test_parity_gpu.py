@@ -123,3 +123,64 @@ def test_repeated_calls_are_independent():
     o2b = pu.run_gpu(w2, i2).cpu().double().numpy()
     pu.assert_close(o2[0, 0], pu.oracle_head(i2, w2, 0, 0), "bf16", "second call")
     assert np.abs(o2 - o2b).max() <= 2e-2
+
+
+# ------------------------------------------------------------------------------- tensor-core path
+TENSOR_CASES = [
+    _wl("tc_perf_d64_k256_m256", PERFORMER, "bf16", 1, 3, 1024, 64, 256, 256, 101),
+    _wl("tc_perf_d64_k64_m64", PERFORMER, "bf16", 2, 2, 512, 64, 64, 64, 102),
+    _wl("tc_perf_d64_k128_m128", PERFORMER, "bf16", 1, 5, 768, 64, 128, 128, 103),
+    _wl("tc_perf_d128_k512_m256", PERFORMER, "bf16", 1, 2, 1024, 128, 512, 256, 104),
+    _wl("tc_perf_d128_k192_m192", PERFORMER, "bf16", 1, 3, 640, 128, 192, 192, 105),
+    _wl("tc_rnn_d64_k256", RNN, "bf16", 2, 3, 1024, 64, 256, 0, 106),
+    _wl("tc_rnn_d128_k64", RNN, "bf16", 1, 2, 512, 128, 64, 0, 107),
+]
+
+
+@pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
+def test_tensor_stage1_projections_match_oracle(w):
+    """K' = E K, V' = F V from the tcgen05 down-projection, element by element."""
+    inputs = synth.make_inputs(w)
+    pu.run_gpu(w, inputs, binding.PATH_TENSOR_STAGE1)
+    assert binding.flurka_last_path() == binding.PATH_TENSOR_STAGE1
+    Kp = binding.flurka_debug_copy(0, (w.B, w.H, w.k, w.d)).cpu().double().numpy()
+    Vp = binding.flurka_debug_copy(1, (w.B, w.H, w.k, w.d)).cpu().double().numpy()
+    torch.cuda.synchronize()
+    for b in range(w.B):
+        for h in range(w.H):
+            _, inter = pu.oracle_head(inputs, w, b, h, rows=[0], intermediates=True)
+            for got, ref, nm in ((Kp[b, h], inter["Kp"], "K'"), (Vp[b, h], inter["Vp"], "V'")):
+                err = np.abs(got - ref).max()
+                assert err < 3e-5 * max(1.0, np.abs(ref).max()), "%s %s head (%d,%d): %.3e" % (w.name, nm, b, h, err)
+
+
+@pytest.mark.parametrize("limit", [0, 3])
+@pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
+def test_tensor_stage3_matches_oracle(w, limit):
+    """tcgen05 query side (several tiles per CTA and head changes when the CTA count is limited)."""
+    prev = binding.flurka_set_cta_limit(limit)
+    try:
+        pu.check_all_heads(w, path=binding.PATH_TENSOR_STAGE3)
+    finally:
+        binding.flurka_set_cta_limit(prev)
+
+
+@pytest.mark.parametrize("limit", [0, 5])
+@pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
+def test_tensor_path_matches_oracle(w, limit):
+    prev = binding.flurka_set_cta_limit(limit)
+    try:
+        pu.check_all_heads(w, path=binding.PATH_TENSOR)
+        assert binding.flurka_last_path() == binding.PATH_TENSOR
+        assert binding.flurka_last_launches() == 3
+    finally:
+        binding.flurka_set_cta_limit(prev)
+
+
+def test_auto_picks_tensor_path_when_the_shape_allows():
+    w = TENSOR_CASES[0]
+    pu.check_all_heads(w)
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    odd = _wl("auto_simt", PERFORMER, "bf16", 1, 1, 200, 64, 64, 64, 108)      # N % 128 != 0
+    pu.check_all_heads(odd)
+    assert binding.flurka_last_path() == binding.PATH_SIMT
