@@ -57,7 +57,7 @@ class ClockSampler:
             self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
-                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -195,16 +195,23 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # the clock sampler runs from the warm-up to the end of the stage-timing pass; a steady load of
+    # untimed steps before the timed region gives nvidia-smi something to see (steps last < 1 ms)
+    sampler = ClockSampler(local)
+    sampler.start()
     with torch.cuda.stream(stream):
         for _ in range(max(args.warmup, 3)):
             step()
+        t_load = time.perf_counter()
+        while time.perf_counter() - t_load < 0.6:
+            for _ in range(20):
+                step()
+            stream.synchronize()
     barrier()
 
     # ---- timed region: K steps, CUDA events on the launch stream around each step
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    sampler = ClockSampler(local)
-    sampler.start()
     barrier()
     with torch.cuda.stream(stream):
         for i in range(args.steps):
@@ -214,7 +221,6 @@ def main():
             step()
             stops[i].record(stream)
     barrier()
-    clocks = sampler.stop()
     step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
     total_ms = sum(step_ms)
     launches = binding.flurka_last_launches() * args.steps
@@ -233,6 +239,7 @@ def main():
     binding.flurka_set_stage_timing(False)
     stage_ms = [x / args.steps for x in stage_ms]
     torch.cuda.synchronize()
+    clocks = sampler.stop()
 
     # ---- end to end: host buffers in, host buffer out, through the host entry point
     e2e_steps = max(1, min(args.steps, 5))

@@ -65,7 +65,8 @@ typedef enum {
   FLURKA_PATH_SIMT = 1,   /* fp32 CUDA-core kernels: any shape within the limits, both element types */
   FLURKA_PATH_TENSOR = 2, /* tcgen05 / TMEM / TMA kernels: bf16 only, shape rules below; else error  */
   FLURKA_PATH_TENSOR_STAGE1 = 3, /* for bisecting: tensor-core down-projection, the rest on CUDA cores */
-  FLURKA_PATH_TENSOR_STAGE3 = 4  /* for bisecting: tensor-core query side, the rest on CUDA cores      */
+  FLURKA_PATH_TENSOR_STAGE3 = 4, /* for bisecting: tensor-core query side, the rest on CUDA cores      */
+  FLURKA_PATH_TENSOR_STAGE23 = 5 /* for bisecting: tensor-core key and query side, CUDA-core stage 1   */
 } flurka_path_t;
 
 /*
@@ -121,7 +122,7 @@ int flurka_last_launches(void);
  * Copies an intermediate of the most recent flurka_forward to a DEVICE buffer, asynchronously on
  * `stream` (order it after the forward).  `which`: 0 = K' [B,H,k,d] fp32, 1 = V' [B,H,k,d] fp32
  * (Eq. (2)'s E K, F V), 2 = key-side summary a [B,H,p,d] fp32 (a_i = sum_j phi(k'_j)_i v'_j / z_i,
- * p = m or d; SIMT path only), 3 = per-feature weights [B,H,p] fp32 (PERFORMER: log z_i with the
+ * p = m or d; only on paths whose query side runs on CUDA cores), 3 = per-feature weights [B,H,p] fp32 (PERFORMER: log z_i with the
  * exponent maximum added back; RNN: z_i), 4 = status words (4 x int32).  `bytes` must equal the
  * intermediate's size.
  */

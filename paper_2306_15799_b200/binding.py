@@ -14,7 +14,7 @@ from .configs import PERFORMER, RNN
 
 IO_BF16 = 0x000
 IO_FP32 = 0x100
-PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_STAGE1, PATH_TENSOR_STAGE3 = 0, 1, 2, 3, 4
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_STAGE1, PATH_TENSOR_STAGE3, PATH_TENSOR_STAGE23 = 0, 1, 2, 3, 4, 5
 
 EXPORTS = [
     "flurka_forward", "flurka_forward_host", "flurka_workspace_bytes", "flurka_set_workspace",

@@ -199,11 +199,11 @@ int key_side_dispatch(const Problem& pr, const float* kpvp, const void* W, float
 }
 
 // The three stages in order.  tc1 / tc3 choose the tensor-core kernel for stage 1 / stage 3
-// (bf16 only); stage 2 is the CUDA-core kernel on every path.
+// (bf16 only); tc2 (which needs tc3) does the same for stage 2.
 template <typename T>
 int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
-                 const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc3,
-                 int* launches) {
+                 const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc2,
+                 bool tc3, int* launches) {
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
   float* a32 = (float*)(ws + L.a32);
@@ -224,8 +224,14 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
     if (rc) return rc;
   }
   g.timer.mark(1, st);
-  rc = key_side_dispatch<T>(pr, kpvp, W, weight, tc3 ? nullptr : a32, tc3 ? aT16 : nullptr, st, launches);
-  if (rc) return rc;
+  if (tc2) {
+    rc = launch_k2(g.maps, performer, kpvp, W, weight, aT16, pr.BH(), pr.d, pr.k, pr.p(), status, st, &cuda_err);
+    if (rc) { g.last_cuda_error = cuda_err; return rc; }
+    ++*launches;
+  } else {
+    rc = key_side_dispatch<T>(pr, kpvp, W, weight, tc3 ? nullptr : a32, tc3 ? aT16 : nullptr, st, launches);
+    if (rc) return rc;
+  }
   g.timer.mark(2, st);
   if (tc3) {
     rc = launch_k3(g.maps, performer, Q, W, aT16, weight, out, pr.BH(), pr.N, pr.d, pr.p(), status, st, &cuda_err);
@@ -245,7 +251,7 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
 template <typename T>
 int run_simt(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
              const void* E, const void* F, const void* W, void* out, cudaStream_t st, int* launches) {
-  return run_pipeline<T>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, launches);
+  return run_pipeline<T>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, false, launches);
 }
 
 int validate_pointers(const Problem& pr, const void* Q, const void* K, const void* V, const void* E,
@@ -294,8 +300,9 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
     rc = run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
   } else {
     const bool tc1 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE1;
-    const bool tc3 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE3;
-    rc = run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, tc1, tc3, &launches);
+    const bool tc2 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE23;
+    const bool tc3 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE3 || tc2;
+    rc = run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, tc1, tc2, tc3, &launches);
   }
   if (rc) return rc;
   g.timer.have = g.timer.on;
@@ -379,7 +386,7 @@ int flurka_set_workspace(void* dev_ptr, size_t bytes) {
 
 int flurka_set_path(int path) {
   const int prev = g.path;
-  if (path >= FLURKA_PATH_AUTO && path <= FLURKA_PATH_TENSOR_STAGE3) g.path = path;
+  if (path >= FLURKA_PATH_AUTO && path <= FLURKA_PATH_TENSOR_STAGE23) g.path = path;
   return prev;
 }
 

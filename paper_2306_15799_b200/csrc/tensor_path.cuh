@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include "k1_down_project.cuh"
+#include "k2_key_side.cuh"
 #include "k3_query_side.cuh"
 
 namespace flurka {
@@ -77,7 +78,7 @@ inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int ran
 }
 
 struct TensorMaps {
-  CachedMap E, F, K, V, kpvp, Q, W, aT, O;
+  CachedMap E, F, K, V, kpvp, Q, W, W2, aT, O;
 };
 
 // 0 = use every SM; otherwise the persistent kernels are launched with at most this many CTAs
@@ -144,6 +145,34 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
   const int grid = 2 * p.k_halves * p.col_groups * p.nsplit;
   k1_down_project<<<grid, kK1Threads, kK1SmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
   cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
+
+// ---- stage 2: per-feature summaries a (fp16, transposed) and weights b / z from K', V' --------
+inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const void* W, float* weight,
+                     __half* aT16, int BH, int d, int k, int p, int* status, cudaStream_t st, int* cuda_err) {
+  if (performer) {
+    const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
+    const unsigned bW[2] = {64, 128};
+    if (!encode_map(&tm.W2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW)) {
+      *cuda_err = (int)cudaErrorInvalidValue;
+      return -6;
+    }
+  }
+  K2Params prm;
+  prm.d = d; prm.k = k; prm.p = p; prm.BH = BH;
+  prm.ftiles = (p + 127) / 128;
+  prm.kpvp = kpvp;
+  prm.weight = weight;
+  prm.aT16 = aT16;
+  prm.status = status;
+  auto fn = performer ? k2_key_side<true> : k2_key_side<false>;
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK2SmemBytes);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  // the RNN kernel ignores tmW; pass any valid map
+  fn<<<BH * prm.ftiles, kK2Threads, kK2SmemBytes, st>>>(performer ? tm.W2.map : tm.kpvp.map, prm);
+  e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
 }

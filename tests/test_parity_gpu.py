@@ -165,6 +165,29 @@ def test_tensor_stage3_matches_oracle(w, limit):
         binding.flurka_set_cta_limit(prev)
 
 
+@pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
+def test_tensor_stage2_matches_oracle(w):
+    """tcgen05 key side (with the tcgen05 query side behind it) on CUDA-core projections; also the
+    per-feature log-weights against the oracle's z (differences, the global stabiliser drops out)."""
+    inputs = synth.make_inputs(w)
+    out = pu.run_gpu(w, inputs, binding.PATH_TENSOR_STAGE23).cpu().double().numpy()
+    p = w.m if w.variant == PERFORMER else w.d
+    bw = binding.flurka_debug_copy(3, (w.B, w.H, p)).cpu().double().numpy()
+    torch.cuda.synchronize()
+    for b in range(w.B):
+        for h in range(w.H):
+            ref, inter = pu.oracle_head(inputs, w, b, h, intermediates=True)
+            pu.assert_close(out[b, h], ref, w.io, "%s head (%d,%d)" % (w.name, b, h))
+            z = inter["z"]
+            big = z > 1e-30 * z.max()
+            if w.variant == PERFORMER:
+                lz = np.log(z[big])
+                got = bw[b, h][big]
+                assert np.abs((got - got[0]) - (lz - lz[0])).max() < 5e-3
+            else:
+                assert np.abs(bw[b, h] / z - 1.0).max() < 2e-3
+
+
 @pytest.mark.parametrize("limit", [0, 5])
 @pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
 def test_tensor_path_matches_oracle(w, limit):
