@@ -149,8 +149,13 @@ def main():
     ap.add_argument("--impl", default="flurka", choices=["flurka", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--heads", default="", help="B,H override: a smaller batch of the same workload (profiling)")
+    ap.add_argument("--no-load", action="store_true", help="skip the sustained-load phase before timing (profiling)")
     args = ap.parse_args()
     w = configs.get(args.config)
+    if args.heads:
+        b, h = (int(x) for x in args.heads.split(","))
+        w = configs.shrink(w, name="%s_B%d_H%d" % (w.name, b, h), B=b, H=h)
 
     if args.impl == "reference":
         run_reference(args, w)
@@ -203,7 +208,7 @@ def main():
         for _ in range(max(args.warmup, 3)):
             step()
         t_load = time.perf_counter()
-        while time.perf_counter() - t_load < 0.6:
+        while not args.no_load and time.perf_counter() - t_load < 0.6:
             for _ in range(20):
                 step()
             stream.synchronize()

@@ -21,6 +21,7 @@ struct K1Params {
   int col_groups;  // ceil(BH * d / 256)
   int k_halves;    // ceil(k / 256)
   int* status;
+  unsigned long long* trace;   // optional [gridDim.x][4] nanosecond stamps: start, set up, accumulated, done
 };
 
 constexpr int kK1Stages = 3;
@@ -44,6 +45,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   __shared__ uint32_t tmem_base_shared;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x] = global_timer_ns();
 
   // ---- which piece of the problem
   int idx = blockIdx.x;
@@ -85,6 +87,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   }
   __syncthreads();
   const uint32_t tmem = tmem_base_shared;
+  if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 1] = global_timer_ns();
 
   if (nchunks > 0) {
     if (warp == 0 && lane == 0) {
@@ -129,16 +132,13 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
         tcgen05_fence_after();
         const uint32_t a_base = smem_base + st * kK1StageBytes;
         const uint32_t b_base = a_base + 32768;
+        // A: K-major, 128-byte rows, 8-row groups 1024 B apart; 16 contraction elements = 32 B per step.
+        // B: MN-major, 64-column slabs 8192 B apart, 8-row (contraction) groups 1024 B apart;
+        //    16 contraction elements = 16 rows = 2048 B per step.
+        const uint64_t bd = make_sdesc(b_base, 8192, 1024, kSwizzle128);
         for (int m = 0; m < mt; ++m) {
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            // A: K-major, 128-byte rows, 8-row groups 1024 B apart; 16 contraction elements = 32 B
-            const uint64_t ad = make_sdesc(a_base + m * 16384 + ks * 32, 16, 1024, kSwizzle128);
-            // B: MN-major, 64-column slabs 8192 B apart, 8-row (contraction) groups 1024 B apart;
-            // 16 contraction elements = 16 rows = 2048 B
-            const uint64_t bd = make_sdesc(b_base + ks * 2048, 8192, 1024, kSwizzle128);
-            mma_ss(tmem + m * 256, ad, bd, idesc, (it > 0 || ks > 0) ? 1u : 0u);
-          }
+          const uint64_t ad = make_sdesc(a_base + m * 16384, 16, 1024, kSwizzle128);
+          mma_ss_x4(tmem + m * 256, ad, bd, 2, 128, idesc, it > 0 ? 1u : 0u);
         }
         mma_commit(bar_empty + 8 * st);
       }
@@ -147,6 +147,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
       // ------------------------------------------------ epilogue: TMEM -> smem -> TMA reduce-add
       const int q = warp & 3;                                // TMEM lane quadrant of this warp
       bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
+      if (p.trace && warp == 2 && lane == 0) p.trace[4 * blockIdx.x + 2] = global_timer_ns();
       if (ok) {
         tcgen05_fence_after();
         const uint32_t stage_buf = smem_base + (warp - 2) * 32768;   // 8 x 4 KB, pipeline is drained
@@ -156,7 +157,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
           for (int cc = 0; cc < ncc; ++cc) {
             uint32_t r[32];
             tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + m * 256 + cc * 32, r);
-            tmem_wait_ld();
+            tmem_wait_ld(r);
             const uint32_t row_addr = stage_buf + cc * 4096 + lane * 128;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
@@ -187,6 +188,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   }
   tcgen05_fence_before();
   __syncthreads();
+  if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 3] = global_timer_ns();
   if (warp == 1) tmem_dealloc(tmem, tmem_cols);
 }
 

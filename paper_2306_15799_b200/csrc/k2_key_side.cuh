@@ -6,13 +6,13 @@
 //               b_i  = log sum_j exp(L_ij),  a_i = sum_j softmax_j(L_i.) v'_j
 //   RNN         f_ij = elu(k'_ji) + 1,  z_i = sum_j f_ij,  a_i = sum_j f_ij v'_j / z_i
 //
-// One CTA owns 128 features of one head.  K' and V' arrive as fp32 (stage 1's workspace) and are
-// split on the fly into bf16 / fp16 terms so that the tensor-core products are fp32-accurate:
-// K' = hi + mid + lo (three bf16 terms, exact to 24 bits) against the exact bf16 W, and
-// -|k'|^2/2 as three bf16 terms in one extra 16-wide contraction step; V' = hi + lo in fp16.
-// L for all k keys sits in TMEM (k <= 512 columns); the thread that owns a row takes its maximum,
-// writes exp(L - max) back as fp16 pairs and keeps the sum of the rounded values, so the dominant
-// term cancels exactly in a_i.  The second product reads those weights straight from TMEM.
+// One CTA owns 128 features of one head and walks the keys in chunks of 128.  K' and V' arrive as
+// fp32 (stage 1's workspace) and are split on the fly into bf16 / fp16 terms so that the tensor-core
+// products are fp32-accurate: K' = hi + mid + lo (three bf16 terms, exact to 24 bits) against the
+// exact bf16 W, and -|k'|^2/2 as three bf16 terms in one extra 16-wide contraction step; V' = hi + lo
+// in fp16.  L for all k keys sits in TMEM (k <= 512 columns); the thread that owns a row takes its
+// maximum, writes exp(L - max) back as fp16 pairs and keeps the sum of the rounded values, so the
+// dominant term cancels exactly in a_i.  The second product reads those weights straight from TMEM.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -29,12 +29,21 @@ struct K2Params {
   float* weight;            // [BH][p]      b_i (PERFORMER) or z_i (RNN)
   __half* aT16;             // [BH][d][p]   a^T
   int* status;
+  long long* trace;         // optional [gridDim.x][8] cycle sums of thread 0 (see K2_STAMP)
 };
 
 constexpr int kK2Threads = 256;
-// shared memory: W tile (<= 32 KB) | ones 4 KB | -|k'|^2/2 tile 2 KB | three 16 KB operand tiles | barrier
-constexpr int kK2SmemBytes = 32768 + 4096 + 2048 + 3 * 16384 + 256 + 1024;
+constexpr int kK2Chunk = 128;  // keys per chunk (the last chunk may hold 64)
+// shared memory: W tile (<= 32 KB) | ones 4 KB | -|k'|^2/2 tile 4 KB | three 32 KB operand tiles | barriers
+constexpr int kK2SmemBytes = 32768 + 4096 + 4096 + 3 * 32768 + 256 + 1024;
 constexpr int kK2OCol = 256;   // TMEM column of the a accumulator
+
+// two floats -> {lo: bf16(a), hi: bf16(b)} with one rounding instruction
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(r) : "f"(a), "f"(b));
+  return r;
+}
 
 __device__ __forceinline__ float k2_ex2(float x) {
   float y;
@@ -52,21 +61,26 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   const uint32_t sm_w = base;
   const uint32_t sm_ones = base + 32768;
   const uint32_t sm_nrm = sm_ones + 4096;
-  const uint32_t sm_op = sm_nrm + 2048;          // 3 x 16 KB, 1024-aligned
-  const uint32_t bar_w = sm_op + 3 * 16384;
+  const uint32_t sm_op = sm_nrm + 4096;          // 3 x 32 KB, 1024-aligned
+  const uint32_t bar_w = sm_op + 3 * 32768;
   const uint32_t bar_mma = bar_w + 8;
   const uint32_t tmem_slot = bar_w + 16;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  long long tlast = clock64();
+  const bool tracing = prm.trace != nullptr && tid == 0;
+#define K2_STAMP(slot) \
+  if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
   const int d = prm.d, k = prm.k, p = prm.p;
   const int head = blockIdx.x / prm.ftiles;
   const int i0 = (blockIdx.x % prm.ftiles) * 128;            // first feature of this CTA
   const float* __restrict__ Kp = prm.kpvp + (size_t)head * k * d;
   const float* __restrict__ Vp = prm.kpvp + ((size_t)prm.BH + head) * (size_t)k * d;
   const int kq = d >> 6;                                      // 64-wide blocks of the head dimension
-  const int nchunks = k >> 6;                                 // 64 keys per chunk
+  const int nchunks = (k + kK2Chunk - 1) / kK2Chunk;
 
   if (tid == 0) {
     abort_flag = 0;
@@ -105,47 +119,79 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   const uint32_t tmem = tmem_base_shared;
   bool ok = true;
   uint32_t mma_phase = 0;
+  K2_STAMP(0)
 
-  // conversion geometry: 4 threads per key row, each a contiguous quarter of the d columns
-  const int crow = tid >> 2;                   // 0..63
-  const int cseg = (tid & 3) * (d >> 2);       // first column of this thread's segment
-  const int cper = d >> 2;                     // 16 or 32 columns
+  // conversion geometry: 2 threads per key row, each a contiguous half of the d columns,
+  // worked through in runs of 32 columns
+  const int crow = tid >> 1;                   // 0..127
+  const int cseg = (tid & 1) * (d >> 1);       // first column of this thread's segment
+  const int runs = d >> 6;                     // 32-column runs per chunk and thread (1 or 2)
+  const int total_runs = nchunks * runs;
+  // loads the next run of fp32 values (which may belong to the next chunk) while the current one is
+  // being converted: the rows come from L2 with a long latency
+  auto load_run = [&](const float* mat, int g, float4 (&buf)[8]) {
+    const int jc = g / runs, c32 = (g % runs) * 32;
+    const int rows = min(kK2Chunk, k - jc * kK2Chunk);
+    if (crow < rows) {
+      const float* src = mat + (size_t)(jc * kK2Chunk + crow) * d + cseg + c32;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) buf[q] = *reinterpret_cast<const float4*>(src + 4 * q);
+    }
+  };
+  // only the issuing warp polls the MMA barrier; everybody else sleeps in the block barrier
+  auto wait_mma = [&]() {
+    bool mine = true;
+    if (warp == 4) mine = mbar_wait(bar_mma, mma_phase, prm.status, &abort_flag);
+    ok = __syncthreads_and(mine) != 0;
+    mma_phase ^= 1;
+    tcgen05_fence_after();
+  };
 
   if (kPerformer) {
-    ok = __syncthreads_and(mbar_wait(bar_w, 0, prm.status, &abort_flag)) != 0;
-    const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, 64);
+    {
+      bool mine = true;
+      if (warp == 4) mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
+      ok = __syncthreads_and(mine) != 0;
+    }
+    float4 cur[8], nxt[8];
+    load_run(Kp, 0, cur);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
-      // ---- K' rows jc*64 .. +64: fp32 -> three bf16 tiles (K-major, 128-byte swizzle) and -|k'|^2/2
-      const float* src = Kp + (size_t)(jc * 64 + crow) * d + cseg;
+      const int rows = min(kK2Chunk, k - jc * kK2Chunk);        // 64 or 128 keys in this chunk
+      // ---- K' rows of the chunk: fp32 -> three bf16 tiles (K-major, 128-byte swizzle) and -|k'|^2/2
       float sq = 0.f;
-      for (int c8 = 0; c8 < cper; c8 += 8) {
-        const float4 v0 = *reinterpret_cast<const float4*>(src + c8);
-        const float4 v1 = *reinterpret_cast<const float4*>(src + c8 + 4);
-        const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        uint32_t w0[4], w1[4], w2[4];
+      for (int run = 0; run < runs; ++run) {
+        const int g = jc * runs + run;
+        if (g + 1 < total_runs) load_run(Kp, g + 1, nxt);
+        if (crow < rows) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float a = x[2 * e], b = x[2 * e + 1];
-          sq = fmaf(a, a, sq);
-          sq = fmaf(b, b, sq);
-          const __nv_bfloat16 a0 = __float2bfloat16_rn(a), b0 = __float2bfloat16_rn(b);
-          a -= __bfloat162float(a0); b -= __bfloat162float(b0);
-          const __nv_bfloat16 a1 = __float2bfloat16_rn(a), b1 = __float2bfloat16_rn(b);
-          a -= __bfloat162float(a1); b -= __bfloat162float(b1);
-          const __nv_bfloat16 a2 = __float2bfloat16_rn(a), b2 = __float2bfloat16_rn(b);
-          w0[e] = (uint32_t)__bfloat16_as_ushort(a0) | ((uint32_t)__bfloat16_as_ushort(b0) << 16);
-          w1[e] = (uint32_t)__bfloat16_as_ushort(a1) | ((uint32_t)__bfloat16_as_ushort(b1) << 16);
-          w2[e] = (uint32_t)__bfloat16_as_ushort(a2) | ((uint32_t)__bfloat16_as_ushort(b2) << 16);
+          for (int c8i = 0; c8i < 4; ++c8i) {
+            const float4 v0 = cur[2 * c8i], v1 = cur[2 * c8i + 1];
+            const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+            uint32_t w0[4], w1[4], w2[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // packed conversions: one instruction rounds two values; a bf16 is the top half of an fp32
+              float a = x[2 * e], b = x[2 * e + 1];
+              sq = fmaf(a, a, sq);
+              sq = fmaf(b, b, sq);
+              w0[e] = pack_bf16x2(a, b);
+              a -= __uint_as_float(w0[e] << 16); b -= __uint_as_float(w0[e] & 0xffff0000u);
+              w1[e] = pack_bf16x2(a, b);
+              a -= __uint_as_float(w1[e] << 16); b -= __uint_as_float(w1[e] & 0xffff0000u);
+              w2[e] = pack_bf16x2(a, b);
+            }
+            const int col = cseg + run * 32 + 8 * c8i;
+            const uint32_t off = (uint32_t)(col >> 6) * 16384 + crow * 128 + ((((col & 63) >> 3) ^ (crow & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + off), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 32768 + off), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 65536 + off), "r"(w2[0]), "r"(w2[1]), "r"(w2[2]), "r"(w2[3]) : "memory");
+          }
         }
-        const int col = cseg + c8;
-        const uint32_t off = (uint32_t)(col >> 6) * 8192 + crow * 128 + ((((col & 63) >> 3) ^ (crow & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + off), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 16384 + off), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 32768 + off), "r"(w2[0]), "r"(w2[1]), "r"(w2[2]), "r"(w2[3]) : "memory");
+#pragma unroll
+        for (int q = 0; q < 8; ++q) cur[q] = nxt[q];
       }
       sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-      sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-      if ((tid & 3) == 0) {
+      if ((tid & 1) == 0 && crow < rows) {
         // B operand of the bias step: row j, columns 0..2 = three bf16 terms of -|k'_j|^2/2
         float b = -0.5f * sq;
         const __nv_bfloat16 h0 = __float2bfloat16_rn(b);  b -= __bfloat162float(h0);
@@ -160,50 +206,49 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       }
       fence_proxy_async_smem();
       __syncthreads();
+      K2_STAMP(1)
       if (tid == 128) {
         tcgen05_fence_after();
-        const int ksteps = d >> 4;
-        bool first = true;
-        for (int s = 0; s < 3; ++s) {
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const uint64_t ad = make_sdesc(sm_w + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128);
-            const uint64_t bd = make_sdesc(sm_op + s * 16384 + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024, kSwizzle128);
-            mma_ss(tmem + jc * 64, ad, bd, idesc1, first ? 0u : 1u);
-            first = false;
+        const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, (uint32_t)rows);
+        const uint32_t dcol = tmem + jc * kK2Chunk;
+        for (int s3 = 0; s3 < 3; ++s3) {
+          for (int kb = 0; kb < kq; ++kb) {
+            const uint64_t ad = make_sdesc(sm_w + kb * 16384, 16, 1024, kSwizzle128);
+            const uint64_t bd = make_sdesc(sm_op + s3 * 32768 + kb * 16384, 16, 1024, kSwizzle128);
+            mma_ss_x4(dcol, ad, bd, 2, 2, idesc1, (s3 > 0 || kb > 0) ? 1u : 0u);
           }
         }
         const uint64_t ad = make_sdesc(sm_ones, 128, 256, kSwizzleNone);
         const uint64_t bd = make_sdesc(sm_nrm, 128, 256, kSwizzleNone);
-        mma_ss(tmem + jc * 64, ad, bd, idesc1, 1u);
+        mma_ss(dcol, ad, bd, idesc1, 1u);
         mma_commit(bar_mma);
       }
       // the operand tiles are rewritten for the next chunk: wait until the MMAs have read them
-      ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, prm.status, &abort_flag)) != 0;
-      mma_phase ^= 1;
-      tcgen05_fence_after();
+      wait_mma();
+      K2_STAMP(2)
     }
   }
 
   // ---- feature weights: one thread per feature row (warps 0..3)
   float zsum = 0.f;
-  const int feat = i0 + warp * 32 + lane;                   // valid for warps 0..3
-  if (warp < 4 && ok) {
-    const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16);
-    if (kPerformer) {
+  const int feat = i0 + (warp & 3) * 32 + lane;             // valid for warps 0..3
+  if (kPerformer) {
+    if (warp < 4 && ok) {
+      const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16);
       const float kLog2e = 1.4426950408889634f;
       float mx = -INFINITY;
       for (int c = 0; c < k; c += 32) {
         uint32_t r[32];
         tmem_ld32(tb + c, r);
-        tmem_wait_ld();
+        tmem_wait_ld(r);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+        for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
       }
       const float shift = mx * kLog2e;
       for (int c = 0; c < k; c += 32) {
         uint32_t r[32], h[16];
         tmem_ld32(tb + c, r);
-        tmem_wait_ld();
+        tmem_wait_ld(r);
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const float e0 = k2_ex2(fmaf(__uint_as_float(r[2 * e]), kLog2e, -shift));
@@ -216,73 +261,103 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
         tmem_st16(tb + (c >> 1), h);
       }
       if (feat < p) prm.weight[(size_t)head * p + feat] = mx + __logf(zsum);
-    } else {
-      // RNN: f_ij = elu(k'_ji) + 1 for this thread's feature i, all keys j (coalesced over i)
-      for (int c = 0; c < k; c += 32) {
-        uint32_t h[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          float x0 = 0.f, x1 = 0.f;
-          if (feat < p) {
-            x0 = Kp[(size_t)(c + 2 * e) * d + feat];
-            x1 = Kp[(size_t)(c + 2 * e + 1) * d + feat];
-          }
-          const float f0 = x0 > 0.f ? x0 + 1.f : __expf(x0);
-          const float f1 = x1 > 0.f ? x1 + 1.f : __expf(x1);
-          const __half2 hh = __floats2half2_rn(f0, f1);
-          const float2 back = __half22float2(hh);
-          zsum += back.x + back.y;
-          h[e] = *reinterpret_cast<const uint32_t*>(&hh);
-        }
-        tmem_st16(tb + (c >> 1), h);
-      }
-      if (feat < p) prm.weight[(size_t)head * p + feat] = zsum;
+      tmem_wait_st();
+      tcgen05_fence_before();
     }
-    tmem_wait_st();
-    tcgen05_fence_before();
+  } else {
+    // RNN: f_ij = elu(k'_ji) + 1.  All threads stage 64 rows of K' in shared memory (coalesced), then
+    // the thread that owns feature i walks down column i (row stride d + 1 words: no bank conflicts).
+    float* stage = reinterpret_cast<float*>(base_ptr + (sm_op - base));
+    const uint32_t tb = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    for (int jc = 0; jc < (k >> 6); ++jc) {
+      __syncthreads();
+      for (int idx = tid * 4; idx < 64 * d; idx += kK2Threads * 4) {
+        const int r = idx / d, c = idx % d;
+        const float4 v = *reinterpret_cast<const float4*>(Kp + (size_t)(jc * 64 + r) * d + c);
+        float* dst = stage + r * (d + 1) + c;
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+      }
+      __syncthreads();
+      if (warp < 4) {
+        const int col = feat < p ? feat : 0;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t h[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float x0 = stage[(half * 32 + 2 * e) * (d + 1) + col];
+            const float x1 = stage[(half * 32 + 2 * e + 1) * (d + 1) + col];
+            const float f0 = x0 > 0.f ? x0 + 1.f : __expf(x0);
+            const float f1 = x1 > 0.f ? x1 + 1.f : __expf(x1);
+            const __half2 hh = __floats2half2_rn(f0, f1);
+            const float2 back = __half22float2(hh);
+            zsum += back.x + back.y;
+            h[e] = *reinterpret_cast<const uint32_t*>(&hh);
+          }
+          tmem_st16(tb + jc * 32 + half * 16, h);
+        }
+      }
+    }
+    if (warp < 4) {
+      if (feat < p) prm.weight[(size_t)head * p + feat] = zsum;
+      tmem_wait_st();
+      tcgen05_fence_before();
+    }
   }
   __syncthreads();
+  K2_STAMP(3)
 
-  // ---- a = weights x V', streamed in chunks of 64 keys; V' = hi + lo in fp16, MN-major slabs
+  // ---- a = weights x V', streamed in chunks of up to 128 keys; V' = hi + lo in fp16, MN-major slabs
   {
     const uint32_t idesc2 = make_idesc(kFmtF16, 0, /*B MN-major*/ 1, 128, (uint32_t)d);
+    float4 cur[8], nxt[8];
+    load_run(Vp, 0, cur);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
-      const float* src = Vp + (size_t)(jc * 64 + crow) * d + cseg;
-      for (int c8 = 0; c8 < cper; c8 += 8) {
-        const float4 v0 = *reinterpret_cast<const float4*>(src + c8);
-        const float4 v1 = *reinterpret_cast<const float4*>(src + c8 + 4);
-        const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        uint32_t w0[4], w1[4];
+      const int rows = min(kK2Chunk, k - jc * kK2Chunk);
+      for (int run = 0; run < runs; ++run) {
+        const int g = jc * runs + run;
+        if (g + 1 < total_runs) load_run(Vp, g + 1, nxt);
+        if (crow < rows) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const __half2 hi = __floats2half2_rn(x[2 * e], x[2 * e + 1]);
-          const float2 hb = __half22float2(hi);
-          const __half2 lo = __floats2half2_rn(x[2 * e] - hb.x, x[2 * e + 1] - hb.y);
-          w0[e] = *reinterpret_cast<const uint32_t*>(&hi);
-          w1[e] = *reinterpret_cast<const uint32_t*>(&lo);
+          for (int c8i = 0; c8i < 4; ++c8i) {
+            const float4 v0 = cur[2 * c8i], v1 = cur[2 * c8i + 1];
+            const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+            uint32_t w0[4], w1[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __half2 hi = __floats2half2_rn(x[2 * e], x[2 * e + 1]);
+              const float2 hb = __half22float2(hi);
+              const __half2 lo = __floats2half2_rn(x[2 * e] - hb.x, x[2 * e + 1] - hb.y);
+              w0[e] = *reinterpret_cast<const uint32_t*>(&hi);
+              w1[e] = *reinterpret_cast<const uint32_t*>(&lo);
+            }
+            const int col = cseg + run * 32 + 8 * c8i;
+            const uint32_t off = (uint32_t)(col >> 6) * 16384 + crow * 128 + ((((col & 63) >> 3) ^ (crow & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + off), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 32768 + off), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
+          }
         }
-        const int col = cseg + c8;
-        const uint32_t off = (uint32_t)(col >> 6) * 8192 + crow * 128 + ((((col & 63) >> 3) ^ (crow & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + off), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 16384 + off), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
+#pragma unroll
+        for (int q = 0; q < 8; ++q) cur[q] = nxt[q];
       }
       fence_proxy_async_smem();
       __syncthreads();
+      K2_STAMP(4)
       if (tid == 128) {
         tcgen05_fence_after();
-        for (int s = 0; s < 2; ++s) {
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            // B: 64-column slabs 8192 B apart, 8-key groups 1024 B apart, 16 keys = 2048 B per step
-            const uint64_t bd = make_sdesc(sm_op + s * 16384 + ks * 2048, 8192, 1024, kSwizzle128);
-            mma_ts(tmem + kK2OCol, tmem + jc * 32 + ks * 8, bd, idesc2, (jc > 0 || s > 0 || ks > 0) ? 1u : 0u);
+        // B: 64-column slabs 16384 B apart, 8-key groups 1024 B apart, 16 keys = 2048 B per step;
+        // A: the fp16 weights of these keys, 8 TMEM columns per step
+        for (int s2 = 0; s2 < 2; ++s2) {
+          for (int q4 = 0; q4 < (rows >> 6); ++q4) {
+            const uint64_t bd = make_sdesc(sm_op + s2 * 32768 + q4 * 8192, 16384, 1024, kSwizzle128);
+            mma_ts_x4(tmem + kK2OCol, tmem + jc * (kK2Chunk >> 1) + q4 * 32, bd, 128, idesc2,
+                      (jc > 0 || s2 > 0 || q4 > 0) ? 1u : 0u);
           }
         }
         mma_commit(bar_mma);
       }
-      ok = __syncthreads_and(mbar_wait(bar_mma, mma_phase, prm.status, &abort_flag)) != 0;
-      mma_phase ^= 1;
-      tcgen05_fence_after();
+      wait_mma();
+      K2_STAMP(5)
     }
   }
 
@@ -296,7 +371,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     for (int c = 0; c < d; c += 32) {
       uint32_t r[32];
       tmem_ld32(tb + c, r);
-      tmem_wait_ld();
+      tmem_wait_ld(r);
       if (feat < p) {
 #pragma unroll
         for (int e = 0; e < 32; ++e) dst[(size_t)(c + e) * p] = __float2half_rn(__uint_as_float(r[e]) * inv);
@@ -305,6 +380,11 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   }
   tcgen05_fence_before();
   __syncthreads();
+  K2_STAMP(6)
+#undef K2_STAMP
+  if (tracing) {
+    for (int sidx = 0; sidx < 8; ++sidx) prm.trace[(size_t)blockIdx.x * 8 + sidx] = tacc[sidx];
+  }
   if (warp == 4) tmem_dealloc(tmem, 512);
 }
 

@@ -9,10 +9,10 @@
 //   RNN         p = (elu(q) + 1) z / max z  straight from the Q tile, then the same second product.
 //
 // The per-feature summaries a_i, b_i (or z_i) come from stage 2.  A persistent CTA walks a
-// contiguous range of 128-row tiles; warp 0 feeds TMA, warp 1 issues MMAs, warp 2 rebuilds the
-// bias operand when the head changes, and two groups of four warps alternate tiles (TMEM is
-// split in two 256-column halves: S/p in columns 0.., O in columns 128.. of each half).
-// The bf16 output tile is staged in the tile's own Q buffer and leaves through TMA.
+// contiguous range of 128-row tiles; warp 0 feeds TMA, warps 1 and 3 issue the first and the second
+// products, warp 2 rebuilds the bias operand when the head changes, and two groups of four warps
+// alternate tiles (TMEM is split in two 256-column halves: S/p in columns 0.., O in columns 128..
+// of each half).  Every thread of a group owns one output row and writes it with 32-byte stores.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -27,10 +27,13 @@ struct K3Params {
   int tiles_per_head;       // N / 128
   int total_tiles;
   const float* weight;      // [BH][p]  b_i or z_i
+  __nv_bfloat16* out;       // [BH][N][d]
   int* status;
+  long long* trace;         // optional [gridDim.x][3][8] cycle sums: two row-owner groups, then the issuers
 };
 
 constexpr int kK3Threads = 384;
+constexpr int kK3MaxQStages = 4;
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -38,7 +41,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
-// shared-memory plan (bytes, from a 1024-aligned base); see k3_smem_bytes()
+// shared-memory plan (byte offsets from a 1024-aligned base)
 struct K3Smem {
   uint32_t w, ones, bias, aT, q, scale, bars, total;
   int q_stages;
@@ -50,11 +53,10 @@ __host__ __device__ inline K3Smem k3_smem_plan(int d, int p, bool performer) {
   s.w = off;    off += performer ? (uint32_t)p * d * 2 : 0;        // W: d/64 K-blocks of [p rows x 128 B]
   s.ones = off; off += performer ? 4096 : 0;                       // [128 x 16] bf16, no swizzle
   s.bias = off; off += performer ? 8192 : 0;                       // [256 x 16] bf16, no swizzle
-  s.aT = off;   off += (uint32_t)d * p * 2;                        // a^T: p/64 K-blocks of [d rows x 128 B]
-  s.aT = (s.aT + 1023u) & ~1023u;
-  off = s.aT + (uint32_t)d * p * 2;
   off = (off + 1023u) & ~1023u;
-  s.q_stages = (d == 64) ? 3 : 2;
+  s.aT = off;   off += (uint32_t)d * p * 2;                        // a^T: p/64 K-blocks of [d rows x 128 B]
+  off = (off + 1023u) & ~1023u;
+  s.q_stages = (d == 64) ? 4 : 2;
   s.q = off;    off += (uint32_t)s.q_stages * 128 * d * 2;
   s.scale = off; off += 1024;                                      // RNN: z_i / max z as floats
   s.bars = off; off += 256;
@@ -65,8 +67,7 @@ __host__ __device__ inline K3Smem k3_smem_plan(int d, int p, bool performer) {
 template <bool kPerformer>
 __global__ void __launch_bounds__(kK3Threads, 1)
 k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmW,
-              const __grid_constant__ CUtensorMap tmAT, const __grid_constant__ CUtensorMap tmO,
-              const K3Params prm) {
+              const __grid_constant__ CUtensorMap tmAT, const K3Params prm) {
   using namespace tc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -78,16 +79,16 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 
   // barriers
   const uint32_t bars = base + L.bars;
-  const uint32_t bar_qfull = bars;            // [3]
-  const uint32_t bar_qempty = bars + 24;      // [3]
-  const uint32_t bar_sfull = bars + 48;       // [2]   S ready in TMEM (PERFORMER)
-  const uint32_t bar_pfull = bars + 64;       // [2]   p written to TMEM by the 128 row owners
-  const uint32_t bar_ofull = bars + 80;       // [2]   O ready in TMEM
-  const uint32_t bar_sfree = bars + 96;       // [2]   TMEM half read out, may be overwritten
-  const uint32_t bar_wfull = bars + 112;      //       W resident
-  const uint32_t bar_drained = bars + 120;    //       every MMA of the previous head is complete
-  const uint32_t bar_atfull = bars + 128;     //       a^T of the new head resident
-  const uint32_t bar_biasready = bars + 136;  //       bias operand / scale vector of the new head built
+  const uint32_t bar_qfull = bars;            // [4]   Q tile landed
+  const uint32_t bar_qempty = bars + 32;      // [4]   Q tile consumed (MMA commit, or 128 readers for RNN)
+  const uint32_t bar_sfull = bars + 64;       // [2]   S ready in TMEM (PERFORMER)
+  const uint32_t bar_pfull = bars + 80;       // [2]   p written to TMEM by the 128 row owners
+  const uint32_t bar_ofull = bars + 96;       // [2]   O ready in TMEM
+  const uint32_t bar_sfree = bars + 112;      // [2]   TMEM half read out, may be overwritten
+  const uint32_t bar_wfull = bars + 128;      //       W resident
+  const uint32_t bar_drained = bars + 136;    //       every MMA of the previous head is complete
+  const uint32_t bar_atfull = bars + 144;     //       a^T of the new head resident
+  const uint32_t bar_biasready = bars + 152;  //       bias operand / scale vector of the new head built
   const uint32_t tmem_slot = bars + 192;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
@@ -101,9 +102,9 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < kK3MaxQStages; ++i) {
       mbar_init(bar_qfull + 8 * i, 1);
-      mbar_init(bar_qempty + 8 * i, 1);
+      mbar_init(bar_qempty + 8 * i, kPerformer ? 1 : 128);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_sfull + 8 * i, 1);
@@ -151,7 +152,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       // ============================================================ TMA producer
       prefetch_tmap(&tmQ);
       prefetch_tmap(&tmAT);
-      prefetch_tmap(&tmO);
       bool ok = true;
       if (kPerformer) {
         prefetch_tmap(&tmW);
@@ -185,55 +185,37 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           (void)mbar_wait(bar_qfull + 8 * (i % NS), (i / NS) & 1, prm.status, &abort_flag);
       }
     } else if (warp == 1 && lane == 0) {
-      // ============================================================ MMA issuer
-      const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, (uint32_t)p);   // S = Q W^T (+ bias step)
-      const uint32_t idesc2 = make_idesc(kFmtF16, 0, 0, 128, (uint32_t)d);    // O = p a
-      bool ok = true;
-      if (kPerformer) ok = mbar_wait(bar_wfull, 0, prm.status, &abort_flag);
-      int head_prev = -1, events = 0;
-      // second product of tile j (j = i-1 inside the loop, the last tile after it)
-      auto second_product = [&](int j) -> bool {
-        const int buf = j & 1;
-        if (!mbar_wait(bar_pfull + 8 * buf, (j >> 1) & 1, prm.status, &abort_flag)) return false;
-        tcgen05_fence_after();
-        const uint32_t tb = tmem + buf * 256;
-        const int ksteps = p >> 4;
-        for (int ks = 0; ks < ksteps; ++ks) {
-          const uint64_t bd = make_sdesc(base + L.aT + (ks >> 2) * (d * 128) + (ks & 3) * 32, 16, 1024, kSwizzle128);
-          mma_ts(tb + 128, tb + ks * 8, bd, idesc2, ks > 0 ? 1u : 0u);
-        }
-        mma_commit(bar_ofull + 8 * buf);
-        return true;
-      };
-      int pending = -1;     // tile whose second product has not been issued yet
-      for (int i = 0; i < ntiles && ok; ++i) {
-        const int head = (t_begin + i) / prm.tiles_per_head;
-        const int buf = i & 1, st = i % NS;
-        if (head != head_prev) {
-          if (events > 0) {
-            // drain: the old head's operands stay in use until its last second product completes
-            if (pending >= 0) { ok = second_product(pending); pending = -1; if (!ok) break; }
-            mma_commit(bar_drained);
+      // ============================================================ issuer of the first products
+      // S_i = Q_i W^T + 1 b^T (PERFORMER only).  A new head's bias operand is ready once
+      // bar_biasready flips, which also means every MMA of the old head has completed.
+      if (kPerformer) {
+        const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, (uint32_t)p);
+        bool ok = mbar_wait(bar_wfull, 0, prm.status, &abort_flag);
+        int head_prev = -1, events = 0;
+        const bool mtracing = prm.trace != nullptr;
+        long long macc[2] = {0, 0};
+        long long mlast = mtracing ? clock64() : 0;
+        for (int i = 0; i < ntiles && ok; ++i) {
+          const int head = (t_begin + i) / prm.tiles_per_head;
+          const int buf = i & 1, st = i % NS;
+          if (head != head_prev) {
+            ok = mbar_wait(bar_biasready, events & 1, prm.status, &abort_flag);
+            if (!ok) break;
+            head_prev = head;
+            ++events;
           }
-          ok = mbar_wait(bar_atfull, events & 1, prm.status, &abort_flag);
-          if (ok) ok = mbar_wait(bar_biasready, events & 1, prm.status, &abort_flag);
-          if (!ok) break;
-          head_prev = head;
-          ++events;
-        }
-        if (kPerformer) {
-          // TMEM half `buf` must have been read out by the epilogue of tile i-2
+          // TMEM half `buf` must have been read out by the row owners of tile i-2
           if (i >= 2) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> 1) - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
           if (!ok) break;
           tcgen05_fence_after();
+          if (mtracing) { const long long now = clock64(); macc[0] += now - mlast; mlast = now; }
           const uint32_t tb = tmem + buf * 256;
           const uint32_t qb = base + L.q + st * q_stage_bytes;
-          const int ksteps = d >> 4;
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const uint64_t ad = make_sdesc(qb + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024, kSwizzle128);
-            const uint64_t bd = make_sdesc(base + L.w + (ks >> 2) * (p * 128) + (ks & 3) * 32, 16, 1024, kSwizzle128);
-            mma_ss(tb, ad, bd, idesc1, ks > 0 ? 1u : 0u);
+          for (int kb = 0; kb < kq; ++kb) {
+            const uint64_t ad = make_sdesc(qb + kb * 16384, 16, 1024, kSwizzle128);
+            const uint64_t bd = make_sdesc(base + L.w + kb * (p * 128), 16, 1024, kSwizzle128);
+            mma_ss_x4(tb, ad, bd, 2, 2, idesc1, kb > 0 ? 1u : 0u);
           }
           {
             // bias step: ones[128 x 16] (columns 0..2 = 1) times bias[p x 16] (b split in three bf16)
@@ -242,13 +224,54 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             mma_ss(tb, ad, bd, idesc1, 1u);
           }
           mma_commit(bar_sfull + 8 * buf);
+          mma_commit(bar_qempty + 8 * st);         // the Q tile is free once these MMAs have read it
+          if (mtracing) { const long long now = clock64(); macc[1] += now - mlast; mlast = now; }
         }
-        // the second product of the previous tile goes after the first product of this one, so the
-        // row owners of this tile can start while the previous tile's output is still being formed
-        if (pending >= 0) { ok = second_product(pending); if (!ok) break; }
-        pending = i;
+        if (mtracing) {
+          prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 0] = macc[0];
+          prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 1] = macc[1];
+        }
       }
-      if (ok && pending >= 0) (void)second_product(pending);
+    } else if (warp == 3 && lane == 0) {
+      // ============================================================ issuer of the second products
+      // O_j = p_j a once the 128 row owners of tile j have written p_j.  Before the first tile of a
+      // new head it waits for that head's a^T; after the last tile of a head it commits to
+      // bar_drained, which therefore flips when every MMA that used the old operands is complete
+      // (a tile's second product completes after its first product).
+      const uint32_t idesc2 = make_idesc(kFmtF16, 0, 0, 128, (uint32_t)d);
+      bool ok = true;
+      int head_prev = -1, events = 0;
+      const bool mtracing = prm.trace != nullptr;
+      long long macc[2] = {0, 0};
+      long long mlast = mtracing ? clock64() : 0;
+      for (int j = 0; j < ntiles && ok; ++j) {
+        const int head = (t_begin + j) / prm.tiles_per_head;
+        const int buf = j & 1;
+        if (head != head_prev) {
+          ok = mbar_wait(bar_atfull, events & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          head_prev = head;
+          ++events;
+        }
+        ok = mbar_wait(bar_pfull + 8 * buf, (j >> 1) & 1, prm.status, &abort_flag);
+        if (!ok) break;
+        tcgen05_fence_after();
+        if (mtracing) { const long long now = clock64(); macc[0] += now - mlast; mlast = now; }
+        const uint32_t tb = tmem + buf * 256;
+        // four 16-wide steps per call: one 64-feature block of p (TMEM) against one block of a^T
+        for (int kb = 0; kb < kp; ++kb) {
+          const uint64_t bd = make_sdesc(base + L.aT + kb * (d * 128), 16, 1024, kSwizzle128);
+          mma_ts_x4(tb + 128, tb + kb * 32, bd, 2, idesc2, kb > 0 ? 1u : 0u);
+        }
+        mma_commit(bar_ofull + 8 * buf);
+        const bool last_of_head = (j + 1 < ntiles) && ((t_begin + j + 1) / prm.tiles_per_head != head);
+        if (last_of_head) mma_commit(bar_drained);
+        if (mtracing) { const long long now = clock64(); macc[1] += now - mlast; mlast = now; }
+      }
+      if (mtracing) {
+        prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 2] = macc[0];
+        prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 3] = macc[1];
+      }
     } else if (warp == 2) {
       // ============================================================ per-head operand builder
       int head_prev = -1, events = 0;
@@ -297,13 +320,19 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const float kLog2e = 1.4426950408889634f;
       int head_prev = -1, events = 0;
       bool ok = true;
+      // optional cycle accounting of one thread per group: 0 wait for S (or Q), 1 pass 1,
+      // 2 pass 2 + hand-over, 3 wait for O, 4 normalise + store
+      const bool tracing = prm.trace != nullptr && q4 == 0 && lane == 0;
+      long long tacc[6] = {0, 0, 0, 0, 0, 0};
+      long long tlast = tracing ? clock64() : 0;
+#define K3_STAMP(slot) \
+  if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
       for (int i = grp; i < ntiles && ok; i += 2) {
         const int tile = t_begin + i;
         const int head = tile / prm.tiles_per_head;
         const int row0 = (tile % prm.tiles_per_head) * 128;
         const int buf = i & 1, st = i % NS;
         const uint32_t tb = tmem + buf * 256 + lane_off;
-        const uint32_t qb = base + L.q + st * q_stage_bytes;
         float denom = 0.f;
         // count head changes the same way the other roles do (both groups see every tile index)
         for (int j = (i >= 2 ? i - 1 : 0); j <= i; ++j) {
@@ -314,30 +343,50 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           ok = mbar_wait(bar_sfull + 8 * buf, (i >> 1) & 1, prm.status, &abort_flag);
           if (!ok) break;
           tcgen05_fence_after();
+          K3_STAMP(0)
+          // Two passes over the row with double-buffered TMEM loads: while one 32-column chunk is
+          // being worked on, the next one is already in flight.
           // pass 1: row maximum
           float mx = -INFINITY;
-          for (int c = 0; c < p; c += 32) {
-            uint32_t r[32];
-            tmem_ld32(tb + c, r);
-            tmem_wait_ld();
+          uint32_t ra[32], rb[32];
+          tmem_ld32(tb, ra);
+          for (int c = 0; c < p; c += 64) {
+            tmem_wait_ld(ra);
+            tmem_ld32(tb + c + 32, rb);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+            for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            tmem_wait_ld(rb);
+            tmem_ld32(tb + ((c + 64 < p) ? c + 64 : 0), ra);      // last round: first chunk of pass 2
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
           }
           const float shift = mx * kLog2e;
+          K3_STAMP(1)
           // pass 2: p = 2^(S log2e - shift), fp16 pairs back into columns [c/2, c/2+16)
-          for (int c = 0; c < p; c += 32) {
-            uint32_t r[32], h[16];
-            tmem_ld32(tb + c, r);
-            tmem_wait_ld();
+          for (int c = 0; c < p; c += 64) {
+            uint32_t h[16];
+            tmem_wait_ld(ra);
+            tmem_ld32(tb + c + 32, rb);
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const float e0 = ex2_approx(fmaf(__uint_as_float(r[2 * e]), kLog2e, -shift));
-              const float e1 = ex2_approx(fmaf(__uint_as_float(r[2 * e + 1]), kLog2e, -shift));
+              const float e0 = ex2_approx(fmaf(__uint_as_float(ra[2 * e]), kLog2e, -shift));
+              const float e1 = ex2_approx(fmaf(__uint_as_float(ra[2 * e + 1]), kLog2e, -shift));
               denom += e0 + e1;
               const __half2 hh = __floats2half2_rn(e0, e1);
               h[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
             tmem_st16(tb + (c >> 1), h);
+            tmem_wait_ld(rb);
+            if (c + 64 < p) tmem_ld32(tb + c + 64, ra);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float e0 = ex2_approx(fmaf(__uint_as_float(rb[2 * e]), kLog2e, -shift));
+              const float e1 = ex2_approx(fmaf(__uint_as_float(rb[2 * e + 1]), kLog2e, -shift));
+              denom += e0 + e1;
+              const __half2 hh = __floats2half2_rn(e0, e1);
+              h[e] = *reinterpret_cast<const uint32_t*>(&hh);
+            }
+            tmem_st16(tb + ((c + 32) >> 1), h);
           }
         } else {
           // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
@@ -345,6 +394,8 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           if (ok) ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
           if (!ok) break;
+          K3_STAMP(0)
+          const uint32_t qb = base + L.q + st * q_stage_bytes;
           const float* sc = reinterpret_cast<const float*>(base_ptr + L.scale);
           for (int c = 0; c < d; c += 32) {
             uint32_t h[16];
@@ -368,47 +419,52 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             }
             tmem_st16(tb + (c >> 1), h);
           }
+          mbar_arrive(bar_qempty + 8 * st);             // this thread is done with the Q tile
         }
         tmem_wait_st();
         tcgen05_fence_before();
         mbar_arrive(bar_pfull + 8 * buf);
+        K3_STAMP(2)
 
-        // ---- epilogue of this tile: O / denom -> bf16 -> the tile's Q buffer -> TMA store
+        // ---- O / denom -> bf16 -> this thread's output row, 32 bytes per store
         ok = mbar_wait(bar_ofull + 8 * buf, (i >> 1) & 1, prm.status, &abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
+        K3_STAMP(3)
         const float inv = 1.f / fmaxf(denom, 1.17549435e-38f);
-        for (int c = 0; c < d; c += 32) {
-          uint32_t r[32];
-          tmem_ld32(tb + 128 + c, r);
-          tmem_wait_ld();
+        __nv_bfloat16* orow = prm.out + ((size_t)head * prm.N + row0 + row) * d;
+        for (int c = 0; c < d; c += 64) {
+          uint32_t ra[32], rb[32];
+          tmem_ld32(tb + 128 + c, ra);
+          tmem_ld32(tb + 128 + c + 32, rb);
+          tmem_wait_ld(ra);
+          tmem_wait_ld(rb);
+          if (c + 64 >= d) {
+            // everything this tile needs from TMEM is in registers: hand the half back before storing
+            tcgen05_fence_before();
+            mbar_arrive(bar_sfree + 8 * buf);
+          }
 #pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t v[4];
+          for (int g8 = 0; g8 < 4; ++g8) {
+            const uint32_t* src = g8 < 2 ? ra : rb;
+            uint32_t v[8];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(r[ch * 8 + 2 * e]) * inv,
-                                                              __uint_as_float(r[ch * 8 + 2 * e + 1]) * inv);
+            for (int e = 0; e < 8; ++e) {
+              const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(src[(g8 & 1) * 16 + 2 * e]) * inv,
+                                                              __uint_as_float(src[(g8 & 1) * 16 + 2 * e + 1]) * inv);
               v[e] = *reinterpret_cast<const uint32_t*>(&o2);
             }
-            const int col = c + ch * 8;
-            const uint32_t a = qb + (col >> 6) * 16384 + row * 128 + ((((col & 63) >> 3) ^ (row & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3])
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(orow + c + g8 * 16),
+                         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
                          : "memory");
           }
         }
-        tcgen05_fence_before();
-        mbar_arrive(bar_sfree + 8 * buf);               // this TMEM half may be overwritten now
-        fence_proxy_async_smem();
-        named_barrier_sync(1 + grp, 128);
-        if (q4 == 0 && lane == 0) {
-          for (int kb = 0; kb < kq; ++kb) tma_store_3d(&tmO, qb + kb * 16384, kb * 64, row0, head);
-          bulk_commit_group();
-          bulk_wait_group_read0();
-          mbar_arrive(bar_qempty + 8 * st);             // the Q buffer may be refilled
-        }
+        K3_STAMP(4)
       }
-      if (q4 == 0 && lane == 0) bulk_wait_group0();
+#undef K3_STAMP
+      if (tracing) {
+        for (int sidx = 0; sidx < 6; ++sidx) prm.trace[((size_t)blockIdx.x * 3 + grp) * 8 + sidx] = tacc[sidx];
+      }
     }
   }
   tcgen05_fence_before();

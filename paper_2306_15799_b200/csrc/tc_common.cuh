@@ -151,7 +151,23 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Waits for this thread's TMEM loads.  The loaded registers are tied to the wait as in/out operands:
+// a TMEM load only defines its registers once the wait has returned, so no use may move above it.
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+        "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+        "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+        "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :
+      : "memory");
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------ MMA
@@ -173,6 +189,47 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Four consecutive 16-wide contraction steps in one go.  Queuing an MMA costs the issuing thread
+// far more than the instruction count suggests (measured: ~170 cycles per MMA when every step
+// builds its own descriptors, ~70 when four steps share one block like this), so the four steps
+// share one predicate and their descriptors are formed by adding constants: `a_step` / `b_step`
+// are the per-step advances of the descriptors' start-address fields (bytes >> 4: 2 for a K-major
+// 128-byte-swizzled operand, 128 for an MN-major one).  The first step accumulates only if
+// `accumulate` is non-zero, the other three always do.
+__device__ __forceinline__ void mma_ss_x4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t a_step,
+                                          uint32_t b_step, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 a1, a2, a3, b1, b2, b3, sa, sb;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.eq.b32 q, 0, 0;\n\t"
+      "cvt.u64.u32 sa, %3;\n\t"
+      "cvt.u64.u32 sb, %4;\n\t"
+      "add.u64 a1, %1, sa;\n\t add.u64 a2, a1, sa;\n\t add.u64 a3, a2, sa;\n\t"
+      "add.u64 b1, %2, sb;\n\t add.u64 b2, b1, sb;\n\t add.u64 b3, b2, sb;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %5, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %5, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %5, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %5, q;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(a_step), "r"(b_step), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The same with A in TMEM: four steps are 8 columns of packed 16-bit values apart.
+__device__ __forceinline__ void mma_ts_x4(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t b_step,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t.reg .b64 b1, b2, b3, sb;\n\t.reg .b32 t1, t2, t3;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "setp.eq.b32 q, 0, 0;\n\t"
+      "cvt.u64.u32 sb, %3;\n\t"
+      "add.u64 b1, %2, sb;\n\t add.u64 b2, b1, sb;\n\t add.u64 b3, b2, sb;\n\t"
+      "add.u32 t1, %1, 8;\n\t add.u32 t2, %1, 16;\n\t add.u32 t3, %1, 24;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [t1], b1, %4, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [t2], b2, %4, q;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [t3], b3, %4, q;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(b_step), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // Arrives on the mbarrier once every MMA issued so far by this thread has completed.

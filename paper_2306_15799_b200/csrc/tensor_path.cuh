@@ -78,7 +78,7 @@ inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int ran
 }
 
 struct TensorMaps {
-  CachedMap E, F, K, V, kpvp, Q, W, W2, aT, O;
+  CachedMap E, F, K, V, kpvp, Q, W, W2, aT;
 };
 
 // 0 = use every SM; otherwise the persistent kernels are launched with at most this many CTAs
@@ -99,18 +99,14 @@ inline int sm_count() {
   return (lim > 0 && lim < n) ? lim : n;
 }
 
-// Sequence splits of stage 1: fill whole waves of CTAs with 12..48 chunks of 64 positions each.
+// Sequence splits of stage 1: as few as fill the machine once.  Every split adds a full copy of
+// the output to the fp32 reduction (measured: the reduce-add traffic of all CTAs drains at about
+// 2.5 TB/s after the last MMA, so more, shorter CTAs lose more in that tail than they gain).
 inline int k1_choose_nsplit(int units, int chunks) {
-  const int sms = sm_count();
-  int best = 1;
-  for (int w = 1; w <= 8; ++w) {
-    int ns = (sms * w) / units;
-    if (ns < 1) ns = 1;
-    if (ns > chunks) ns = chunks;
-    best = ns;
-    if (chunks / ns <= 48) break;
-  }
-  return best;
+  int ns = sm_count() / units;
+  if (ns < 1) ns = 1;
+  if (ns > chunks) ns = chunks;
+  return ns;
 }
 
 // ---- stage 1: K' = E K, V' = F V into kpvp (already zeroed) ----------------------------------
@@ -136,6 +132,7 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
   p.k_halves = (k + 255) / 256;
   p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, N / 64);
   p.status = status;
+  p.trace = nullptr;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(k1_down_project, cudaFuncAttributeMaxDynamicSharedMemorySize, kK1SmemBytes);
@@ -167,6 +164,7 @@ inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const vo
   prm.weight = weight;
   prm.aT16 = aT16;
   prm.status = status;
+  prm.trace = nullptr;
   auto fn = performer ? k2_key_side<true> : k2_key_side<false>;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK2SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
@@ -186,7 +184,6 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
   const unsigned long long dA[3] = {(unsigned long long)p, (unsigned long long)d, (unsigned long long)BH};
   const unsigned bA[3] = {64, (unsigned)d, 1};
   if (!encode_map(&tm.Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Q, dQ, bQ) ||
-      !encode_map(&tm.O, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, out, dQ, bQ) ||
       !encode_map(&tm.aT, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, 3, aT16, dA, bA)) {
     *cuda_err = (int)cudaErrorInvalidValue;
     return -6;
@@ -204,7 +201,9 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
   prm.tiles_per_head = N / 128;
   prm.total_tiles = prm.tiles_per_head * BH;
   prm.weight = weight;
+  prm.out = reinterpret_cast<__nv_bfloat16*>(out);
   prm.status = status;
+  prm.trace = nullptr;
   const K3Smem L = k3_smem_plan(d, p, performer);
   auto fn = performer ? k3_query_side<true> : k3_query_side<false>;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
@@ -212,7 +211,7 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
   int grid = sm_count();
   if (grid > prm.total_tiles) grid = prm.total_tiles;
   // the RNN kernel ignores tmW; pass any valid map
-  fn<<<grid, kK3Threads, L.total, st>>>(tm.Q.map, performer ? tm.W.map : tm.Q.map, tm.aT.map, tm.O.map, prm);
+  fn<<<grid, kK3Threads, L.total, st>>>(tm.Q.map, performer ? tm.W.map : tm.Q.map, tm.aT.map, prm);
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
