@@ -1,0 +1,81 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot produce a whole full-size output in reasonable time, so each workload is checked on
+sampled heads and query rows (the oracle still forms the complete K' and V' of a sampled head), plus
+the convexity invariant of Appendix D's normalised weights over the whole GPU output: every output
+column lies between the smallest and largest entry of that column of V' = F V.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2306_15799_b200 import binding, build, configs, synth
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    binding.load()
+
+
+def _check_full(w, heads, n_rows, seed=0):
+    inputs = synth.make_inputs(w)
+    dev = pu.to_device(inputs)
+    out = binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant)
+    torch.cuda.synchronize()
+    assert binding.flurka_last_status() == 0
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    assert binding.flurka_last_launches() == 3
+    # convexity over the whole output, against the library's own fp32 V'
+    Vp = binding.flurka_debug_copy(1, (w.B, w.H, w.k, w.d))
+    torch.cuda.synchronize()
+    lo = Vp.min(dim=2, keepdim=True).values
+    hi = Vp.max(dim=2, keepdim=True).values
+    o32 = out.float()
+    slack = 2.0 ** -7 * torch.maximum(lo.abs(), hi.abs()) + 1e-3          # bf16 rounding of the output
+    assert bool(torch.isfinite(o32).all())
+    assert bool((o32 >= lo - slack).all()) and bool((o32 <= hi + slack).all())
+    rng = np.random.default_rng(seed)
+    worst = (0.0, 0.0)
+    for (b, h) in heads:
+        rows = np.sort(rng.choice(w.N, size=n_rows, replace=False))
+        rows[0], rows[-1] = 0, w.N - 1                                    # first and last row of the head
+        ref = pu.oracle_head(inputs, w, b, h, rows=rows)
+        got = out[b, h].cpu()[torch.from_numpy(rows)].double().numpy()
+        rel, mx = pu.assert_close(got, ref, w.io, "%s head (%d,%d)" % (w.name, b, h))
+        worst = (max(worst[0], rel), max(worst[1], mx))
+    print("%s: worst rel-Fro %.3e, worst max-abs %.3e over %d heads x %d rows" % (w.name, worst[0], worst[1], len(heads), n_rows))
+
+
+def test_c2_full_size():
+    _check_full(configs.C2, heads=[(0, 0), (3, 7), (7, 11)], n_rows=512)
+
+
+def test_c3_full_size():
+    _check_full(configs.C3, heads=[(0, 0), (2, 9), (3, 15)], n_rows=512)
+
+
+def test_c4_full_size():
+    _check_full(configs.C4, heads=[(0, 5)], n_rows=384)
+
+
+@pytest.mark.parametrize("k,m", configs.C5_GRID, ids=lambda v: str(v))
+def test_c5_sweep_points(k, m):
+    """Every (k, m) of the projection-size sweep, at the sweep's N and d with a smaller batch."""
+    w = configs.shrink(configs.c5(k, m), B=1, H=3)
+    inputs = synth.make_inputs(w)
+    out = pu.run_gpu(w, inputs).cpu().double().numpy()
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    rng = np.random.default_rng(k * 1000 + m)
+    for h in range(w.H):
+        rows = np.sort(rng.choice(w.N, size=256, replace=False))
+        ref = pu.oracle_head(inputs, w, 0, h, rows=rows)
+        pu.assert_close(out[0, h][rows], ref, w.io, "%s head %d" % (w.name, h))
+
+
+def test_c5_one_point_full_batch():
+    _check_full(configs.c5(512, 256), heads=[(0, 0), (7, 11)], n_rows=256)
