@@ -345,7 +345,7 @@ def main():
             tt = oracle_sample(wr, host, heads)
             line["cpu_baseline"] = {"value": heads * w.N / tt, "unit": UNIT, "cores": oracle.threads(),
                                     "kind": "oracle",
-                                    "sample": "%d of %d heads of %s, all %d rows each, %.1f s" % (heads, w.B * w.H, w.name, w.N, tt)}
+                                    "sample": "%d head passes over the %d heads of %s, all %d rows each, %.1f s" % (heads, w.B * w.H, w.name, w.N, tt)}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
