@@ -121,21 +121,24 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   uint32_t mma_phase = 0;
   K2_STAMP(0)
 
-  // conversion geometry: 2 threads per key row, each a contiguous half of the d columns,
-  // worked through in runs of 32 columns
-  const int crow = tid >> 1;                   // 0..127
-  const int cseg = (tid & 1) * (d >> 1);       // first column of this thread's segment
-  const int runs = d >> 6;                     // 32-column runs per chunk and thread (1 or 2)
-  const int total_runs = nchunks * runs;
-  // loads the next run of fp32 values (which may belong to the next chunk) while the current one is
-  // being converted: the rows come from L2 with a long latency
-  auto load_run = [&](const float* mat, int g, float4 (&buf)[8]) {
-    const int jc = g / runs, c32 = (g % runs) * 32;
+  // conversion geometry: a warp instruction reads whole rows (d/4 lanes x float4 per row), so the fp32
+  // rows arrive in full 128-byte lines; each lane converts four consecutive columns of its rows
+  const int lpr = d >> 2;                        // lanes per row: 16 or 32
+  const int rpi = 32 / lpr;                      // rows per warp instruction: 2 or 1
+  const int ccol = (lane % lpr) * 4;             // this lane's first column
+  const int crow0 = warp * rpi + lane / lpr;     // this lane's row in iteration 0; iteration t adds 8*rpi
+  const int citers = kK2Chunk / (8 * rpi);       // 8 or 16 iterations cover the 128 rows of a chunk
+  const uint32_t coff = (uint32_t)(ccol >> 6) * 16384 + (uint32_t)((ccol & 7) >> 2) * 8;
+  const int cchunk = (ccol & 63) >> 3;           // 16-byte chunk of the 128-byte row before the swizzle
+  float4 ld[16];
+  // issues the loads of a whole chunk; they are in flight while the previous chunk's MMAs run
+  auto load_chunk = [&](const float* mat, int jc) {
     const int rows = min(kK2Chunk, k - jc * kK2Chunk);
-    if (crow < rows) {
-      const float* src = mat + (size_t)(jc * kK2Chunk + crow) * d + cseg + c32;
 #pragma unroll
-      for (int q = 0; q < 8; ++q) buf[q] = *reinterpret_cast<const float4*>(src + 4 * q);
+    for (int t = 0; t < 16; ++t) {
+      const int r = crow0 + t * 8 * rpi;
+      if (t < citers && r < rows)
+        ld[t] = *reinterpret_cast<const float4*>(mat + (size_t)(jc * kK2Chunk + r) * d + ccol);
     }
   };
   // only the issuing warp polls the MMA barrier; everybody else sleeps in the block barrier
@@ -153,57 +156,54 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       if (warp == 4) mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
       ok = __syncthreads_and(mine) != 0;
     }
-    float4 cur[8], nxt[8];
-    load_run(Kp, 0, cur);
+    load_chunk(Kp, 0);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
       const int rows = min(kK2Chunk, k - jc * kK2Chunk);        // 64 or 128 keys in this chunk
       // ---- K' rows of the chunk: fp32 -> three bf16 tiles (K-major, 128-byte swizzle) and -|k'|^2/2
-      float sq = 0.f;
-      for (int run = 0; run < runs; ++run) {
-        const int g = jc * runs + run;
-        if (g + 1 < total_runs) load_run(Kp, g + 1, nxt);
-        if (crow < rows) {
 #pragma unroll
-          for (int c8i = 0; c8i < 4; ++c8i) {
-            const float4 v0 = cur[2 * c8i], v1 = cur[2 * c8i + 1];
-            const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-            uint32_t w0[4], w1[4], w2[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              // packed conversions: one instruction rounds two values; a bf16 is the top half of an fp32
-              float a = x[2 * e], b = x[2 * e + 1];
-              sq = fmaf(a, a, sq);
-              sq = fmaf(b, b, sq);
-              w0[e] = pack_bf16x2(a, b);
-              a -= __uint_as_float(w0[e] << 16); b -= __uint_as_float(w0[e] & 0xffff0000u);
-              w1[e] = pack_bf16x2(a, b);
-              a -= __uint_as_float(w1[e] << 16); b -= __uint_as_float(w1[e] & 0xffff0000u);
-              w2[e] = pack_bf16x2(a, b);
-            }
-            const int col = cseg + run * 32 + 8 * c8i;
-            const uint32_t off = (uint32_t)(col >> 6) * 16384 + crow * 128 + ((((col & 63) >> 3) ^ (crow & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + off), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 32768 + off), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 65536 + off), "r"(w2[0]), "r"(w2[1]), "r"(w2[2]), "r"(w2[3]) : "memory");
+      for (int t = 0; t < 16; ++t) {
+        if (t < citers) {                                        // uniform over the warp
+          const int r = crow0 + t * 8 * rpi;
+          float sq = 0.f;
+          if (r < rows) {
+            // packed conversions: one instruction rounds two values; a bf16 is the top half of an fp32
+            float a = ld[t].x, b = ld[t].y, c = ld[t].z, e = ld[t].w;
+            sq = fmaf(a, a, fmaf(b, b, fmaf(c, c, e * e)));
+            const uint32_t h0 = pack_bf16x2(a, b), h1 = pack_bf16x2(c, e);
+            a -= __uint_as_float(h0 << 16); b -= __uint_as_float(h0 & 0xffff0000u);
+            c -= __uint_as_float(h1 << 16); e -= __uint_as_float(h1 & 0xffff0000u);
+            const uint32_t m0 = pack_bf16x2(a, b), m1 = pack_bf16x2(c, e);
+            a -= __uint_as_float(m0 << 16); b -= __uint_as_float(m0 & 0xffff0000u);
+            c -= __uint_as_float(m1 << 16); e -= __uint_as_float(m1 & 0xffff0000u);
+            const uint32_t l0 = pack_bf16x2(a, b), l1 = pack_bf16x2(c, e);
+            const uint32_t off = sm_op + coff + r * 128 + ((cchunk ^ (r & 7)) << 4);
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off), "r"(h0), "r"(h1) : "memory");
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 32768), "r"(m0), "r"(m1) : "memory");
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 65536), "r"(l0), "r"(l1) : "memory");
+          }
+          // |k'_r|^2 over the lanes that share the row
+          if (lpr == 32) sq += __shfl_xor_sync(0xffffffffu, sq, 16);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 8);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+          if ((lane % lpr) == 0 && r < rows) {
+            // B operand of the bias step: row r, columns 0..2 = three bf16 terms of -|k'_r|^2/2
+            float bb = -0.5f * sq;
+            const __nv_bfloat16 g0 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g0);
+            const __nv_bfloat16 g1 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g1);
+            const __nv_bfloat16 g2 = __float2bfloat16_rn(bb);
+            const uint32_t na = sm_nrm + (r >> 3) * 256 + (r & 7) * 16;
+            const uint32_t z = 0;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na),
+                         "r"((uint32_t)__bfloat16_as_ushort(g0) | ((uint32_t)__bfloat16_as_ushort(g1) << 16)),
+                         "r"((uint32_t)__bfloat16_as_ushort(g2)), "r"(z), "r"(z) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
           }
         }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) cur[q] = nxt[q];
       }
-      sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-      if ((tid & 1) == 0 && crow < rows) {
-        // B operand of the bias step: row j, columns 0..2 = three bf16 terms of -|k'_j|^2/2
-        float b = -0.5f * sq;
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(b);  b -= __bfloat162float(h0);
-        const __nv_bfloat16 h1 = __float2bfloat16_rn(b);  b -= __bfloat162float(h1);
-        const __nv_bfloat16 h2 = __float2bfloat16_rn(b);
-        const uint32_t a = sm_nrm + (crow >> 3) * 256 + (crow & 7) * 16;
-        const uint32_t z = 0;
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a),
-                     "r"((uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16)),
-                     "r"((uint32_t)__bfloat16_as_ushort(h2)), "r"(z), "r"(z) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
-      }
+      if (jc + 1 < nchunks) load_chunk(Kp, jc + 1);
+      else load_chunk(Vp, 0);                                    // first chunk of the second product
       fence_proxy_async_smem();
       __syncthreads();
       K2_STAMP(1)
@@ -265,6 +265,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       tcgen05_fence_before();
     }
   } else {
+    load_chunk(Vp, 0);
     // RNN: f_ij = elu(k'_ji) + 1.  All threads stage 64 rows of K' in shared memory (coalesced), then
     // the thread that owns feature i walks down column i (row stride d + 1 words: no bank conflicts).
     float* stage = reinterpret_cast<float*>(base_ptr + (sm_op - base));
@@ -310,36 +311,24 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   // ---- a = weights x V', streamed in chunks of up to 128 keys; V' = hi + lo in fp16, MN-major slabs
   {
     const uint32_t idesc2 = make_idesc(kFmtF16, 0, /*B MN-major*/ 1, 128, (uint32_t)d);
-    float4 cur[8], nxt[8];
-    load_run(Vp, 0, cur);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
       const int rows = min(kK2Chunk, k - jc * kK2Chunk);
-      for (int run = 0; run < runs; ++run) {
-        const int g = jc * runs + run;
-        if (g + 1 < total_runs) load_run(Vp, g + 1, nxt);
-        if (crow < rows) {
 #pragma unroll
-          for (int c8i = 0; c8i < 4; ++c8i) {
-            const float4 v0 = cur[2 * c8i], v1 = cur[2 * c8i + 1];
-            const float x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-            uint32_t w0[4], w1[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const __half2 hi = __floats2half2_rn(x[2 * e], x[2 * e + 1]);
-              const float2 hb = __half22float2(hi);
-              const __half2 lo = __floats2half2_rn(x[2 * e] - hb.x, x[2 * e + 1] - hb.y);
-              w0[e] = *reinterpret_cast<const uint32_t*>(&hi);
-              w1[e] = *reinterpret_cast<const uint32_t*>(&lo);
-            }
-            const int col = cseg + run * 32 + 8 * c8i;
-            const uint32_t off = (uint32_t)(col >> 6) * 16384 + crow * 128 + ((((col & 63) >> 3) ^ (crow & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + off), "r"(w0[0]), "r"(w0[1]), "r"(w0[2]), "r"(w0[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sm_op + 32768 + off), "r"(w1[0]), "r"(w1[1]), "r"(w1[2]), "r"(w1[3]) : "memory");
-          }
+      for (int t = 0; t < 16; ++t) {
+        const int r = crow0 + t * 8 * rpi;
+        if (t < citers && r < rows) {
+          const __half2 hi0 = __floats2half2_rn(ld[t].x, ld[t].y), hi1 = __floats2half2_rn(ld[t].z, ld[t].w);
+          const float2 b0 = __half22float2(hi0), b1 = __half22float2(hi1);
+          const __half2 lo0 = __floats2half2_rn(ld[t].x - b0.x, ld[t].y - b0.y);
+          const __half2 lo1 = __floats2half2_rn(ld[t].z - b1.x, ld[t].w - b1.y);
+          const uint32_t off = sm_op + coff + r * 128 + ((cchunk ^ (r & 7)) << 4);
+          asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off), "r"(*reinterpret_cast<const uint32_t*>(&hi0)),
+                       "r"(*reinterpret_cast<const uint32_t*>(&hi1)) : "memory");
+          asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 32768), "r"(*reinterpret_cast<const uint32_t*>(&lo0)),
+                       "r"(*reinterpret_cast<const uint32_t*>(&lo1)) : "memory");
         }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) cur[q] = nxt[q];
       }
+      if (jc + 1 < nchunks) load_chunk(Vp, jc + 1);
       fence_proxy_async_smem();
       __syncthreads();
       K2_STAMP(4)
