@@ -160,46 +160,55 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     for (int jc = 0; jc < nchunks && ok; ++jc) {
       const int rows = min(kK2Chunk, k - jc * kK2Chunk);        // 64 or 128 keys in this chunk
       // ---- K' rows of the chunk: fp32 -> three bf16 tiles (K-major, 128-byte swizzle) and -|k'|^2/2
+      // three passes with independent work per row, so the conversions, the shuffles and the
+      // stores of different rows overlap instead of forming one long dependent chain
+      float sq[16];
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
-        if (t < citers) {                                        // uniform over the warp
-          const int r = crow0 + t * 8 * rpi;
-          float sq = 0.f;
-          if (r < rows) {
-            // packed conversions: one instruction rounds two values; a bf16 is the top half of an fp32
-            float a = ld[t].x, b = ld[t].y, c = ld[t].z, e = ld[t].w;
-            sq = fmaf(a, a, fmaf(b, b, fmaf(c, c, e * e)));
-            const uint32_t h0 = pack_bf16x2(a, b), h1 = pack_bf16x2(c, e);
-            a -= __uint_as_float(h0 << 16); b -= __uint_as_float(h0 & 0xffff0000u);
-            c -= __uint_as_float(h1 << 16); e -= __uint_as_float(h1 & 0xffff0000u);
-            const uint32_t m0 = pack_bf16x2(a, b), m1 = pack_bf16x2(c, e);
-            a -= __uint_as_float(m0 << 16); b -= __uint_as_float(m0 & 0xffff0000u);
-            c -= __uint_as_float(m1 << 16); e -= __uint_as_float(m1 & 0xffff0000u);
-            const uint32_t l0 = pack_bf16x2(a, b), l1 = pack_bf16x2(c, e);
-            const uint32_t off = sm_op + coff + r * 128 + ((cchunk ^ (r & 7)) << 4);
-            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off), "r"(h0), "r"(h1) : "memory");
-            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 32768), "r"(m0), "r"(m1) : "memory");
-            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 65536), "r"(l0), "r"(l1) : "memory");
-          }
-          // |k'_r|^2 over the lanes that share the row
-          if (lpr == 32) sq += __shfl_xor_sync(0xffffffffu, sq, 16);
-          sq += __shfl_xor_sync(0xffffffffu, sq, 8);
-          sq += __shfl_xor_sync(0xffffffffu, sq, 4);
-          sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-          sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-          if ((lane % lpr) == 0 && r < rows) {
-            // B operand of the bias step: row r, columns 0..2 = three bf16 terms of -|k'_r|^2/2
-            float bb = -0.5f * sq;
-            const __nv_bfloat16 g0 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g0);
-            const __nv_bfloat16 g1 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g1);
-            const __nv_bfloat16 g2 = __float2bfloat16_rn(bb);
-            const uint32_t na = sm_nrm + (r >> 3) * 256 + (r & 7) * 16;
-            const uint32_t z = 0;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na),
-                         "r"((uint32_t)__bfloat16_as_ushort(g0) | ((uint32_t)__bfloat16_as_ushort(g1) << 16)),
-                         "r"((uint32_t)__bfloat16_as_ushort(g2)), "r"(z), "r"(z) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
-          }
+        const int r = crow0 + t * 8 * rpi;
+        sq[t] = 0.f;
+        if (t < citers && r < rows) {
+          // packed conversions: one instruction rounds two values; a bf16 is the top half of an fp32
+          float a = ld[t].x, b = ld[t].y, c = ld[t].z, e = ld[t].w;
+          sq[t] = fmaf(a, a, fmaf(b, b, fmaf(c, c, e * e)));
+          const uint32_t h0 = pack_bf16x2(a, b), h1 = pack_bf16x2(c, e);
+          a -= __uint_as_float(h0 << 16); b -= __uint_as_float(h0 & 0xffff0000u);
+          c -= __uint_as_float(h1 << 16); e -= __uint_as_float(h1 & 0xffff0000u);
+          const uint32_t m0 = pack_bf16x2(a, b), m1 = pack_bf16x2(c, e);
+          a -= __uint_as_float(m0 << 16); b -= __uint_as_float(m0 & 0xffff0000u);
+          c -= __uint_as_float(m1 << 16); e -= __uint_as_float(m1 & 0xffff0000u);
+          const uint32_t l0 = pack_bf16x2(a, b), l1 = pack_bf16x2(c, e);
+          const uint32_t off = sm_op + coff + r * 128 + ((cchunk ^ (r & 7)) << 4);
+          asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off), "r"(h0), "r"(h1) : "memory");
+          asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 32768), "r"(m0), "r"(m1) : "memory");
+          asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 65536), "r"(l0), "r"(l1) : "memory");
+        }
+      }
+      // |k'_r|^2 over the lanes that share a row: sixteen independent butterfly reductions
+      if (lpr == 32) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) sq[t] += __shfl_xor_sync(0xffffffffu, sq[t], 16);
+      }
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) sq[t] += __shfl_xor_sync(0xffffffffu, sq[t], o);
+      }
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const int r = crow0 + t * 8 * rpi;
+        if (t < citers && (lane % lpr) == 0 && r < rows) {
+          // B operand of the bias step: row r, columns 0..2 = three bf16 terms of -|k'_r|^2/2
+          float bb = -0.5f * sq[t];
+          const __nv_bfloat16 g0 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g0);
+          const __nv_bfloat16 g1 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g1);
+          const __nv_bfloat16 g2 = __float2bfloat16_rn(bb);
+          const uint32_t na = sm_nrm + (r >> 3) * 256 + (r & 7) * 16;
+          const uint32_t z = 0;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na),
+                       "r"((uint32_t)__bfloat16_as_ushort(g0) | ((uint32_t)__bfloat16_as_ushort(g1) << 16)),
+                       "r"((uint32_t)__bfloat16_as_ushort(g2)), "r"(z), "r"(z) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
         }
       }
       if (jc + 1 < nchunks) load_chunk(Kp, jc + 1);
