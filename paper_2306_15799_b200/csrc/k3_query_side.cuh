@@ -333,7 +333,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         const int row0 = (tile % prm.tiles_per_head) * 128;
         const int buf = i & 1, st = i % NS;
         const uint32_t tb = tmem + buf * 256 + lane_off;
-        float denom = 0.f;
+        float denom = 0.f, denom1 = 0.f;
         // count head changes the same way the other roles do (both groups see every tile index)
         for (int j = (i >= 2 ? i - 1 : 0); j <= i; ++j) {
           const int hj = (t_begin + j) / prm.tiles_per_head;
@@ -347,19 +347,30 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           // Two passes over the row with double-buffered TMEM loads: while one 32-column chunk is
           // being worked on, the next one is already in flight.
           // pass 1: row maximum
-          float mx = -INFINITY;
+          float mx = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
           uint32_t ra[32], rb[32];
           tmem_ld32(tb, ra);
           for (int c = 0; c < p; c += 64) {
             tmem_wait_ld(ra);
             tmem_ld32(tb + c + 32, rb);
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            for (int e = 0; e < 32; e += 8) {      // four independent chains
+              mx = fmax3(mx, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+              mx1 = fmax3(mx1, __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
+              mx2 = fmax3(mx2, __uint_as_float(ra[e + 4]), __uint_as_float(ra[e + 5]));
+              mx3 = fmax3(mx3, __uint_as_float(ra[e + 6]), __uint_as_float(ra[e + 7]));
+            }
             tmem_wait_ld(rb);
             tmem_ld32(tb + ((c + 64 < p) ? c + 64 : 0), ra);      // last round: first chunk of pass 2
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+            for (int e = 0; e < 32; e += 8) {
+              mx = fmax3(mx, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+              mx1 = fmax3(mx1, __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
+              mx2 = fmax3(mx2, __uint_as_float(rb[e + 4]), __uint_as_float(rb[e + 5]));
+              mx3 = fmax3(mx3, __uint_as_float(rb[e + 6]), __uint_as_float(rb[e + 7]));
+            }
           }
+          mx = fmaxf(fmax3(mx, mx1, mx2), mx3);
           const float shift = mx * kLog2e;
           K3_STAMP(1)
           // pass 2: p = 2^(S log2e - shift), fp16 pairs back into columns [c/2, c/2+16)
@@ -369,9 +380,12 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             tmem_ld32(tb + c + 32, rb);
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const float e0 = ex2_approx(fmaf(__uint_as_float(ra[2 * e]), kLog2e, -shift));
-              const float e1 = ex2_approx(fmaf(__uint_as_float(ra[2 * e + 1]), kLog2e, -shift));
-              denom += e0 + e1;
+              const float x0 = fmaf(__uint_as_float(ra[2 * e]), kLog2e, -shift);
+              const float x1 = fmaf(__uint_as_float(ra[2 * e + 1]), kLog2e, -shift);
+              const float e0 = ex2_approx(x0);
+              const float e1 = ex2_approx(x1);
+              denom += e0;
+              denom1 += e1;
               const __half2 hh = __floats2half2_rn(e0, e1);
               h[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
@@ -380,9 +394,12 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             if (c + 64 < p) tmem_ld32(tb + c + 64, ra);
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const float e0 = ex2_approx(fmaf(__uint_as_float(rb[2 * e]), kLog2e, -shift));
-              const float e1 = ex2_approx(fmaf(__uint_as_float(rb[2 * e + 1]), kLog2e, -shift));
-              denom += e0 + e1;
+              const float x0 = fmaf(__uint_as_float(rb[2 * e]), kLog2e, -shift);
+              const float x1 = fmaf(__uint_as_float(rb[2 * e + 1]), kLog2e, -shift);
+              const float e0 = ex2_approx(x0);
+              const float e1 = ex2_approx(x1);
+              denom += e0;
+              denom1 += e1;
               const __half2 hh = __floats2half2_rn(e0, e1);
               h[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
@@ -431,7 +448,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (!ok) break;
         tcgen05_fence_after();
         K3_STAMP(3)
-        const float inv = 1.f / fmaxf(denom, 1.17549435e-38f);
+        const float inv = 1.f / fmaxf(denom + denom1, 1.17549435e-38f);
         __nv_bfloat16* orow = prm.out + ((size_t)head * prm.N + row0 + row) * d;
         for (int c = 0; c < d; c += 64) {
           uint32_t ra[32], rb[32];
