@@ -211,10 +211,7 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   int* status = (int*)(ws + L.status);
   const bool performer = pr.kernel == FLURKA_PERFORMER;
   int cuda_err = 0;
-  // the accumulating stage-1 kernels need zeroed K', V'; a single cluster per tile writes them outright
-  cudaError_t e = cudaSuccess;
-  if (!tc1 || k1_plan(pr.BH(), pr.N, pr.d, pr.k).needs_zero())
-    e = cudaMemsetAsync(kpvp, 0, (size_t)2 * pr.BH() * pr.k * pr.d * 4, st);
+  cudaError_t e = cudaMemsetAsync(kpvp, 0, (size_t)2 * pr.BH() * pr.k * pr.d * 4, st);
   if (e != cudaSuccess) return cuda_fail(e);
   g.timer.mark(0, st);
   int rc;

@@ -6,15 +6,9 @@
 // 64-wide sequence chunks.  Per chunk TMA brings a [rows x 64] slab of E (K-major, the sequence is
 // contiguous) and, per 64 columns, a [64 x 64] slab of K or V (MN-major: the head dimension is
 // contiguous, the contracted sequence index is the slow one), both 128-byte swizzled.  A single
-// thread issues tcgen05.mma (M=128, N=ncols, K=16, four steps per call) into fp32 TMEM accumulators.
-//
-// The CTAs that split one output tile along the sequence form a thread-block cluster.  When the
-// range is done every CTA drops its accumulators into its own shared memory, the cluster
-// synchronises, and each CTA sums a share of the 32x32 sub-tiles over all members through
-// distributed shared memory and writes them out with TMA: a plain store when one cluster covers the
-// whole sequence (no zero-fill, no atomics), an fp32 reduce-add when several clusters share a tile.
-// (Letting every CTA reduce-add its full tile into L2 costs a ~15 us tail: the adds of all CTAs
-// arrive at once and drain at about 2.5 TB/s.)
+// thread issues tcgen05.mma (M=128, N=ncols, K=16) into fp32 TMEM accumulators; when the range is
+// done four warps move the accumulators to shared memory and add them to the fp32 workspace with
+// TMA reduce-add, so partial sums from different CTAs meet in L2.
 #pragma once
 
 #include "tc_common.cuh"
@@ -23,9 +17,7 @@ namespace flurka {
 
 struct K1Params {
   int N, d, k, BH;
-  int nsplit;      // CTAs along the sequence = cluster * nclusters
-  int cluster;     // CTAs per cluster (1..8)
-  int nclusters;   // clusters per output tile; > 1 means the output is accumulated (zeroed before)
+  int nsplit;      // CTAs along the sequence
   int col_groups;  // ceil(BH * d / 256)
   int k_halves;    // ceil(k / 256)
   int* status;
@@ -36,27 +28,6 @@ constexpr int kK1Stages = 3;
 constexpr int kK1StageBytes = 65536;                  // 32 KB of E rows + 32 KB of K/V slabs
 constexpr int kK1SmemBytes = kK1Stages * kK1StageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 constexpr int kK1Threads = 192;
-
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t cluster_cta_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// address of the same shared-memory location in another CTA of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
-  uint32_t a;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank));
-  return a;
-}
-__device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
-  return v;
-}
 
 __global__ void __launch_bounds__(kK1Threads, 1)
 k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmF,
@@ -76,13 +47,12 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x] = global_timer_ns();
 
-  // ---- which piece of the problem (the sequence split is the fastest index: a cluster is made of
-  //      consecutive CTAs, which therefore share t, kh and cg)
+  // ---- which piece of the problem
   int idx = blockIdx.x;
-  const int s = idx % p.nsplit;      idx /= p.nsplit;
   const int cg = idx % p.col_groups; idx /= p.col_groups;
   const int kh = idx % p.k_halves;   idx /= p.k_halves;
   const int t = idx & 1;
+  const int s = idx >> 1;
   const int rows = min(256, p.k - kh * 256);
   const int mt = (rows + 127) >> 7;                         // MMA M-tiles (1 or 2)
   const int total_cols = p.BH * p.d;
@@ -93,8 +63,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const int c_end = (int)(((long long)(s + 1) * chunks_total) / p.nsplit);
   const int nchunks = c_end - c_begin;
   const uint32_t tmem_cols = mt == 2 ? 512u : 256u;
-  const uint32_t cs = (uint32_t)p.cluster;
-  const uint32_t rank = cs > 1 ? cluster_cta_rank() : 0u;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -121,152 +89,103 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const uint32_t tmem = tmem_base_shared;
   if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 1] = global_timer_ns();
 
-  if (warp == 0 && lane == 0) {
-    // ------------------------------------------------ TMA producer
-    const CUtensorMap* tmP = t ? &tmF : &tmE;
-    const CUtensorMap* tmX = t ? &tmV : &tmK;
-    prefetch_tmap(tmP);
-    prefetch_tmap(tmX);
-    prefetch_tmap(&tmOut);
-    const uint32_t tx_bytes = (uint32_t)(mt * 16384 + nb * 8192);
-    const int dblocks = p.d >> 6;                         // 64-column slabs per head
-    int issued = 0;
-    bool ok = true;
-    for (int it = 0; it < nchunks && ok; ++it) {
-      const int st = it % kK1Stages;
-      if (it >= kK1Stages) ok = mbar_wait(bar_empty + 8 * st, ((it / kK1Stages) - 1) & 1, p.status, &abort_flag);
-      if (!ok) break;
-      const uint32_t a_dst = smem_base + st * kK1StageBytes;
-      const uint32_t b_dst = a_dst + 32768;
-      const int n0 = (c_begin + it) << 6;
-      mbar_arrive_expect_tx(bar_full + 8 * st, tx_bytes);
-      for (int m = 0; m < mt; ++m) tma_load_2d(a_dst + m * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + m * 128);
-      for (int b = 0; b < nb; ++b) {
-        const int slab = cg * 4 + b;                       // global 64-column slab index
-        const int head = slab / dblocks, dc = slab % dblocks;
-        tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, dc * 64, n0, head);
-      }
-      ++issued;
-    }
-    if (!ok) {
-      // loads already in flight still land in this CTA's shared memory: wait for them (bounded)
-      for (int it = max(0, issued - kK1Stages); it < issued; ++it)
-        (void)mbar_wait(bar_full + 8 * (it % kK1Stages), (it / kK1Stages) & 1, p.status, &abort_flag);
-    }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------ MMA issuer
-    const uint32_t idesc = make_idesc(kFmtBF16, /*A K-major*/ 0, /*B MN-major*/ 1, 128, (uint32_t)ncols);
-    bool ok = true;
-    for (int it = 0; it < nchunks; ++it) {
-      const int st = it % kK1Stages;
-      ok = mbar_wait(bar_full + 8 * st, (it / kK1Stages) & 1, p.status, &abort_flag);
-      if (!ok) break;
-      tcgen05_fence_after();
-      const uint32_t a_base = smem_base + st * kK1StageBytes;
-      const uint32_t b_base = a_base + 32768;
-      // A: K-major, 128-byte rows, 8-row groups 1024 B apart; 16 contraction elements = 32 B per step.
-      // B: MN-major, 64-column slabs 8192 B apart, 8-row (contraction) groups 1024 B apart;
-      //    16 contraction elements = 16 rows = 2048 B per step.
-      const uint64_t bd = make_sdesc(b_base, 8192, 1024, kSwizzle128);
-      for (int m = 0; m < mt; ++m) {
-        const uint64_t ad = make_sdesc(a_base + m * 16384, 16, 1024, kSwizzle128);
-        mma_ss_x4(tmem + m * 256, ad, bd, 2, 128, idesc, it > 0 ? 1u : 0u);
-      }
-      mma_commit(bar_empty + 8 * st);
-    }
-    if (ok) mma_commit(bar_accum);
-  }
-
-  // ------------------------------------------------ epilogue (all threads take part in the syncs)
-  // Shared memory is free now (this CTA's pipeline is drained before bar_accum flips):
-  //   [0, 128 KB)      this CTA's partial tile, 32 sub-tiles of [32 rows][32 fp32], slot = q*8 + cc,
-  //                    128-byte swizzled rows (same layout in every CTA of the cluster)
-  //   [128, 192 KB)    output staging, 4 x 4 KB per epilogue warp
-  const int q = warp & 3;                                  // TMEM lane quadrant of an epilogue warp
-  const int ncc = ncols >> 5;                              // 32-column sub-tiles per row quadrant
-  bool eok = true;
-  if (warp >= 2) {
-    eok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
-    if (p.trace && warp == 2 && lane == 0) p.trace[4 * blockIdx.x + 2] = global_timer_ns();
-    tcgen05_fence_after();
-  }
-  for (int m = 0; m < mt; ++m) {
-    if (warp >= 2 && eok) {
-      for (int cc = 0; cc < ncc; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + m * 256 + cc * 32, r);
-        tmem_wait_ld(r);
-        const uint32_t row_addr = smem_base + (q * 8 + cc) * 4096 + lane * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint32_t a = row_addr + ((c ^ (lane & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(r[4 * c]), "r"(r[4 * c + 1]),
-                       "r"(r[4 * c + 2]), "r"(r[4 * c + 3])
-                       : "memory");
+  if (nchunks > 0) {
+    if (warp == 0 && lane == 0) {
+      // ------------------------------------------------ TMA producer
+      const CUtensorMap* tmP = t ? &tmF : &tmE;
+      const CUtensorMap* tmX = t ? &tmV : &tmK;
+      prefetch_tmap(tmP);
+      prefetch_tmap(tmX);
+      const uint32_t tx_bytes = (uint32_t)(mt * 16384 + nb * 8192);
+      const int dblocks = p.d >> 6;                         // 64-column slabs per head
+      int issued = 0;
+      bool ok = true;
+      for (int it = 0; it < nchunks && ok; ++it) {
+        const int st = it % kK1Stages;
+        if (it >= kK1Stages) ok = mbar_wait(bar_empty + 8 * st, ((it / kK1Stages) - 1) & 1, p.status, &abort_flag);
+        if (!ok) break;
+        const uint32_t a_dst = smem_base + st * kK1StageBytes;
+        const uint32_t b_dst = a_dst + 32768;
+        const int n0 = (c_begin + it) << 6;
+        mbar_arrive_expect_tx(bar_full + 8 * st, tx_bytes);
+        for (int m = 0; m < mt; ++m) tma_load_2d(a_dst + m * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + m * 128);
+        for (int b = 0; b < nb; ++b) {
+          const int slab = cg * 4 + b;                       // global 64-column slab index
+          const int head = slab / dblocks, dc = slab % dblocks;
+          tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, dc * 64, n0, head);
         }
+        ++issued;
       }
-    }
-    if (cs > 1) cluster_sync_all(); else __syncthreads();
-    if (warp >= 2 && eok) {
-      // sub-tiles j = rank, rank + cs, ... belong to this CTA; its four warps take them in turn
-      const int nitems = 4 * ncc;
-      int mine = 0;
-      for (int j = (int)rank; j < nitems; j += (int)cs, ++mine) {
-        if ((mine & 3) != warp - 2) continue;
-        const int qj = j / ncc, ccj = j % ncc;
-        const uint32_t local = smem_base + (qj * 8 + ccj) * 4096 + lane * 128;
-        float4 acc[8];
+      if (!ok) {
+        // loads already in flight still land in this CTA's shared memory: wait for them (bounded)
+        for (int it = max(0, issued - kK1Stages); it < issued; ++it)
+          (void)mbar_wait(bar_full + 8 * (it % kK1Stages), (it / kK1Stages) & 1, p.status, &abort_flag);
+      }
+    } else if (warp == 1 && lane == 0) {
+      // ------------------------------------------------ MMA issuer
+      const uint32_t idesc = make_idesc(kFmtBF16, /*A K-major*/ 0, /*B MN-major*/ 1, 128, (uint32_t)ncols);
+      bool ok = true;
+      for (int it = 0; it < nchunks; ++it) {
+        const int st = it % kK1Stages;
+        ok = mbar_wait(bar_full + 8 * st, (it / kK1Stages) & 1, p.status, &abort_flag);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_base = smem_base + st * kK1StageBytes;
+        const uint32_t b_base = a_base + 32768;
+        // A: K-major, 128-byte rows, 8-row groups 1024 B apart; 16 contraction elements = 32 B per step.
+        // B: MN-major, 64-column slabs 8192 B apart, 8-row (contraction) groups 1024 B apart;
+        //    16 contraction elements = 16 rows = 2048 B per step.
+        const uint64_t bd = make_sdesc(b_base, 8192, 1024, kSwizzle128);
+        for (int m = 0; m < mt; ++m) {
+          const uint64_t ad = make_sdesc(a_base + m * 16384, 16, 1024, kSwizzle128);
+          mma_ss_x4(tmem + m * 256, ad, bd, 2, 128, idesc, it > 0 ? 1u : 0u);
+        }
+        mma_commit(bar_empty + 8 * st);
+      }
+      if (ok) mma_commit(bar_accum);
+    } else if (warp >= 2) {
+      // ------------------------------------------------ epilogue: TMEM -> smem -> TMA reduce-add
+      const int q = warp & 3;                                // TMEM lane quadrant of this warp
+      bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
+      if (p.trace && warp == 2 && lane == 0) p.trace[4 * blockIdx.x + 2] = global_timer_ns();
+      if (ok) {
+        tcgen05_fence_after();
+        const uint32_t stage_buf = smem_base + (warp - 2) * 32768;   // 8 x 4 KB, pipeline is drained
+        for (int m = 0; m < mt; ++m) {
+          const int row0 = kh * 256 + m * 128 + q * 32;
+          const int ncc = ncols >> 5;
+          for (int cc = 0; cc < ncc; ++cc) {
+            uint32_t r[32];
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + m * 256 + cc * 32, r);
+            tmem_wait_ld(r);
+            const uint32_t row_addr = stage_buf + cc * 4096 + lane * 128;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (uint32_t peer = 0; peer < cs; ++peer) {
-          const uint32_t remote = cs > 1 ? map_to_cta(local, peer) : local;
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint32_t a = remote + ((c ^ (lane & 7)) << 4);
-            float4 v;
-            if (cs > 1) {
-              v = ld_cluster_v4(a);
-            } else {
-              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                           : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+            for (int c = 0; c < 8; ++c) {
+              const uint32_t a = row_addr + ((c ^ (lane & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(r[4 * c]), "r"(r[4 * c + 1]),
+                           "r"(r[4 * c + 2]), "r"(r[4 * c + 3])
+                           : "memory");
             }
-            acc[c].x += v.x; acc[c].y += v.y; acc[c].z += v.z; acc[c].w += v.w;
           }
-        }
-        const int slot = (mine >> 2) & 3;
-        if (slot == 0 && mine >= 16) {                     // staging buffers come round again
-          if (lane == 0) bulk_wait_group_read0();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (row0 < p.k) {
+              for (int cc = 0; cc < ncc; ++cc) {
+                const int col = cg * 256 + cc * 32;
+                const int head = col / p.d, c0 = col % p.d;
+                tma_reduce_add_3d(&tmOut, stage_buf + cc * 4096, c0, row0, t * p.BH + head);
+              }
+            }
+            bulk_commit_group();
+            bulk_wait_group_read0();
+          }
           __syncwarp();
         }
-        const uint32_t ob = smem_base + 131072 + (warp - 2) * 16384 + slot * 4096;
-        const uint32_t orow = ob + lane * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint32_t a = orow + ((c ^ (lane & 7)) << 4);
-          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(acc[c].x), "f"(acc[c].y),
-                       "f"(acc[c].z), "f"(acc[c].w)
-                       : "memory");
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          const int row0 = kh * 256 + m * 128 + qj * 32;
-          if (row0 < p.k) {
-            const int col = cg * 256 + ccj * 32;
-            const int head = col / p.d, c0 = col % p.d;
-            if (p.nclusters > 1) tma_reduce_add_3d(&tmOut, ob, c0, row0, t * p.BH + head);
-            else tma_store_3d(&tmOut, ob, c0, row0, t * p.BH + head);
-          }
-          bulk_commit_group();
-        }
+        if (lane == 0) bulk_wait_group0();
       }
-      if (lane == 0) bulk_wait_group_read0();
-      __syncwarp();
     }
-    // nobody may overwrite its partial tile (next M-tile) or leave while a neighbour still reads it
-    if (cs > 1) cluster_sync_all(); else __syncthreads();
   }
-  if (warp >= 2 && lane == 0) bulk_wait_group0();
   tcgen05_fence_before();
   __syncthreads();
   if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 3] = global_timer_ns();

@@ -99,34 +99,14 @@ inline int sm_count() {
   return (lim > 0 && lim < n) ? lim : n;
 }
 
-// Sequence splits of stage 1: as few as fill the machine once (every extra split is another partial
-// tile to reduce), grouped in clusters of up to 8 CTAs that reduce among themselves.
-struct K1Plan {
-  int col_groups, k_halves, nsplit, cluster, nclusters;
-  bool needs_zero() const { return nclusters > 1; }   // several clusters accumulate into the output
-};
-
-inline K1Plan k1_plan(int BH, int N, int d, int k) {
-  K1Plan pl;
-  pl.col_groups = (BH * d + 255) / 256;
-  pl.k_halves = (k + 255) / 256;
-  const int units = 2 * pl.col_groups * pl.k_halves;
-  const int chunks = N / 64;
+// Sequence splits of stage 1: as few as fill the machine once.  Every split adds a full copy of
+// the output to the fp32 reduction (measured: the reduce-add traffic of all CTAs drains at about
+// 2.5 TB/s after the last MMA, so more, shorter CTAs lose more in that tail than they gain).
+inline int k1_choose_nsplit(int units, int chunks) {
   int ns = sm_count() / units;
   if (ns < 1) ns = 1;
   if (ns > chunks) ns = chunks;
-  if (ns <= 8) {
-    pl.cluster = ns;
-    pl.nclusters = 1;
-  } else {
-    pl.cluster = 1;
-    for (int cs = 8; cs >= 2; --cs) {
-      if ((ns / cs) * cs * 20 >= ns * 19) { pl.cluster = cs; break; }   // lose at most 5 % of the CTAs
-    }
-    pl.nclusters = ns / pl.cluster;
-  }
-  pl.nsplit = pl.cluster * pl.nclusters;
-  return pl;
+  return ns;
 }
 
 // ---- stage 1: K' = E K, V' = F V into kpvp (already zeroed) ----------------------------------
@@ -146,14 +126,11 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
     *cuda_err = (int)cudaErrorInvalidValue;
     return -6;
   }
-  const K1Plan pl = k1_plan(BH, N, d, k);
   K1Params p;
   p.N = N; p.d = d; p.k = k; p.BH = BH;
-  p.col_groups = pl.col_groups;
-  p.k_halves = pl.k_halves;
-  p.nsplit = pl.nsplit;
-  p.cluster = pl.cluster;
-  p.nclusters = pl.nclusters;
+  p.col_groups = (BH * d + 255) / 256;
+  p.k_halves = (k + 255) / 256;
+  p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, N / 64);
   p.status = status;
   p.trace = nullptr;
   static bool attr_set = false;
@@ -162,20 +139,8 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
     if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
     attr_set = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * p.k_halves * p.col_groups * p.nsplit), 1, 1);
-  cfg.blockDim = dim3(kK1Threads, 1, 1);
-  cfg.dynamicSmemBytes = kK1SmemBytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)p.cluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, k1_down_project, tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
-  if (le != cudaSuccess) { *cuda_err = (int)le; (void)cudaGetLastError(); return -6; }
+  const int grid = 2 * p.k_halves * p.col_groups * p.nsplit;
+  k1_down_project<<<grid, kK1Threads, kK1SmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
