@@ -31,19 +31,27 @@ struct Problem {
 //   aT16    fp16 [BH][d][p]        the same, transposed, as the tensor-core B operand
 //   status  int32[4]
 struct Layout {
-  size_t kpvp, weight, a32, aT16, status, total;
+  size_t kpvp, weight, a32, aT16, status, status_bytes, part, total;
 };
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-Layout make_layout(const Problem& pr) {
+// `with_split_scratch`: reserve room for the partial results of a key-split tensor-core stage 2
+// (the SIMT path never needs it)
+Layout make_layout(const Problem& pr, bool with_split_scratch = true) {
   Layout L;
   size_t off = 0;
   L.kpvp = off;   off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
   L.weight = off; off = align256(off + (size_t)pr.BH() * pr.p() * 4);
   L.a32 = off;    off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 4);
   L.aT16 = off;   off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 2);
-  L.status = off; off = align256(off + 16);
+  // four status words, then one arrival counter per (head, 128-feature tile) of stage 2
+  L.status_bytes = 16 + (with_split_scratch ? (size_t)pr.BH() * ((pr.p() + 127) / 128) * 4 : 0);
+  L.status = off; off = align256(off + L.status_bytes);
+  const size_t part_floats = (with_split_scratch && !pr.fp32)
+                                 ? k2_part_floats(pr.kernel == FLURKA_PERFORMER, pr.BH(), pr.d, pr.k, pr.p())
+                                 : 0;
+  L.part = off;   off = align256(off + part_floats * 4);
   L.total = off;
   return L;
 }
@@ -225,7 +233,9 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   }
   g.timer.mark(1, st);
   if (tc2) {
-    rc = launch_k2(g.maps, performer, kpvp, W, weight, aT16, pr.BH(), pr.d, pr.k, pr.p(), status, st, &cuda_err);
+    float* part = L.total > L.part ? (float*)(ws + L.part) : nullptr;
+    rc = launch_k2(g.maps, performer, kpvp, W, weight, aT16, part, status + 4, pr.BH(), pr.d, pr.k, pr.p(), status, st,
+                   &cuda_err);
     if (rc) { g.last_cuda_error = cuda_err; return rc; }
     ++*launches;
   } else {
@@ -293,7 +303,7 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
-  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, 16, st);
+  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, L.status_bytes, st);
   if (e != cudaSuccess) return cuda_fail(e);
 
   if (pr.fp32) {
@@ -519,7 +529,7 @@ extern "C" int flurka_forward_static_scratch(const void* Q, const void* K, const
   if (rc) return rc;
   rc = validate_pointers(pr, Q, K, V, E, F, W, out);
   if (rc) return rc;
-  const Layout L = make_layout(pr);
+  const Layout L = make_layout(pr, /*with_split_scratch=*/false);
   if (L.total > (size_t)FLURKA_STATIC_SCRATCH_BYTES) return FLURKA_ERR_TOO_LARGE;
   rc = check_device();
   if (rc) return rc;

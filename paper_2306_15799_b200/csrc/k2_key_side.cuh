@@ -13,6 +13,11 @@
 // in fp16.  L for all k keys sits in TMEM (k <= 512 columns); the thread that owns a row takes its
 // maximum, writes exp(L - max) back as fp16 pairs and keeps the sum of the rounded values, so the
 // dominant term cancels exactly in a_i.  The second product reads those weights straight from TMEM.
+//
+// With few heads the keys are split over `nsplit` CTAs per (head, feature tile): each keeps its own
+// maximum, sum and unnormalised accumulator, writes them to a scratch area, and the CTA that arrives
+// last at the tile's counter merges them (log-sum-exp over the partial maxima) and writes a_i, b_i.
+// Nobody waits for anybody: the last arrival finds every partial result already in memory.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -30,6 +35,9 @@ struct K2Params {
   __half* aT16;             // [BH][d][p]   a^T
   int* status;
   long long* trace;         // optional [gridDim.x][8] cycle sums of thread 0 (see K2_STAMP)
+  int nsplit;               // CTAs per (head, feature tile) along the keys (1..4; PERFORMER only)
+  float* part;              // nsplit > 1: [BH * ftiles][nsplit][d + 2][128]  max, sum, accumulator columns
+  int* counters;            // nsplit > 1: [BH * ftiles], zero on entry, zero again on exit
 };
 
 constexpr int kK2Threads = 256;
@@ -75,12 +83,18 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
 #define K2_STAMP(slot) \
   if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
   const int d = prm.d, k = prm.k, p = prm.p;
-  const int head = blockIdx.x / prm.ftiles;
-  const int i0 = (blockIdx.x % prm.ftiles) * 128;            // first feature of this CTA
+  const int nsplit = prm.nsplit;
+  const int sp = blockIdx.x % nsplit;                         // which part of the keys
+  const int unit = blockIdx.x / nsplit;                       // (head, feature tile)
+  const int head = unit / prm.ftiles;
+  const int i0 = (unit % prm.ftiles) * 128;                   // first feature of this CTA
   const float* __restrict__ Kp = prm.kpvp + (size_t)head * k * d;
   const float* __restrict__ Vp = prm.kpvp + ((size_t)prm.BH + head) * (size_t)k * d;
   const int kq = d >> 6;                                      // 64-wide blocks of the head dimension
-  const int nchunks = (k + kK2Chunk - 1) / kK2Chunk;
+  const int nchunks_all = (k + kK2Chunk - 1) / kK2Chunk;
+  const int jc_begin = (sp * nchunks_all) / nsplit;           // this CTA's chunks [jc_begin, jc_begin + nchunks)
+  const int nchunks = ((sp + 1) * nchunks_all) / nsplit - jc_begin;
+  const int klocal = min(k, (jc_begin + nchunks) * kK2Chunk) - jc_begin * kK2Chunk;   // keys of this CTA
 
   if (tid == 0) {
     abort_flag = 0;
@@ -156,9 +170,9 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       if (warp == 4) mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
       ok = __syncthreads_and(mine) != 0;
     }
-    load_chunk(Kp, 0);
+    load_chunk(Kp, jc_begin);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
-      const int rows = min(kK2Chunk, k - jc * kK2Chunk);        // 64 or 128 keys in this chunk
+      const int rows = min(kK2Chunk, k - (jc_begin + jc) * kK2Chunk);   // 64 or 128 keys in this chunk
       // ---- K' rows of the chunk: fp32 -> three bf16 tiles (K-major, 128-byte swizzle) and -|k'|^2/2
       // three passes with independent work per row, so the conversions, the shuffles and the
       // stores of different rows overlap instead of forming one long dependent chain
@@ -211,8 +225,8 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
         }
       }
-      if (jc + 1 < nchunks) load_chunk(Kp, jc + 1);
-      else load_chunk(Vp, 0);                                    // first chunk of the second product
+      if (jc + 1 < nchunks) load_chunk(Kp, jc_begin + jc + 1);
+      else load_chunk(Vp, jc_begin);                             // first chunk of the second product
       fence_proxy_async_smem();
       __syncthreads();
       K2_STAMP(1)
@@ -239,22 +253,23 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   }
 
   // ---- feature weights: one thread per feature row (warps 0..3)
-  float zsum = 0.f;
+  float zsum = 0.f, row_max = 0.f;
   const int feat = i0 + (warp & 3) * 32 + lane;             // valid for warps 0..3
   if (kPerformer) {
     if (warp < 4 && ok) {
       const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16);
       const float kLog2e = 1.4426950408889634f;
       float mx = -INFINITY;
-      for (int c = 0; c < k; c += 32) {
+      for (int c = 0; c < klocal; c += 32) {
         uint32_t r[32];
         tmem_ld32(tb + c, r);
         tmem_wait_ld(r);
 #pragma unroll
         for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
       }
+      row_max = mx;
       const float shift = mx * kLog2e;
-      for (int c = 0; c < k; c += 32) {
+      for (int c = 0; c < klocal; c += 32) {
         uint32_t r[32], h[16];
         tmem_ld32(tb + c, r);
         tmem_wait_ld(r);
@@ -269,7 +284,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
         }
         tmem_st16(tb + (c >> 1), h);
       }
-      if (feat < p) prm.weight[(size_t)head * p + feat] = mx + __logf(zsum);
+      if (nsplit == 1 && feat < p) prm.weight[(size_t)head * p + feat] = mx + __logf(zsum);
       tmem_wait_st();
       tcgen05_fence_before();
     }
@@ -321,7 +336,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   {
     const uint32_t idesc2 = make_idesc(kFmtF16, 0, /*B MN-major*/ 1, 128, (uint32_t)d);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
-      const int rows = min(kK2Chunk, k - jc * kK2Chunk);
+      const int rows = min(kK2Chunk, k - (jc_begin + jc) * kK2Chunk);
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
         const int r = crow0 + t * 8 * rpi;
@@ -337,7 +352,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
                        "r"(*reinterpret_cast<const uint32_t*>(&lo1)) : "memory");
         }
       }
-      if (jc + 1 < nchunks) load_chunk(Vp, jc + 1);
+      if (jc + 1 < nchunks) load_chunk(Vp, jc_begin + jc + 1);
       fence_proxy_async_smem();
       __syncthreads();
       K2_STAMP(4)
@@ -360,20 +375,88 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   }
 
   // ---- a_i = accumulator / z_i, stored transposed ([d][p], fp16) for stage 3
-  if (warp < 4 && ok) {
-    // whole warps are either inside or outside the p features (p is a multiple of 64); the TMEM
-    // loads are warp-wide either way, only the stores are predicated
-    const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16) + kK2OCol;
-    const float inv = 1.f / zsum;
-    __half* dst = prm.aT16 + (size_t)head * d * p + feat;
-    for (int c = 0; c < d; c += 32) {
-      uint32_t r[32];
-      tmem_ld32(tb + c, r);
-      tmem_wait_ld(r);
-      if (feat < p) {
+  if (nsplit == 1) {
+    if (warp < 4 && ok) {
+      // whole warps are either inside or outside the p features (p is a multiple of 64); the TMEM
+      // loads are warp-wide either way, only the stores are predicated
+      const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16) + kK2OCol;
+      const float inv = 1.f / zsum;
+      __half* dst = prm.aT16 + (size_t)head * d * p + feat;
+      for (int c = 0; c < d; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(tb + c, r);
+        tmem_wait_ld(r);
+        if (feat < p) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) dst[(size_t)(c + e) * p] = __float2half_rn(__uint_as_float(r[e]) * inv);
+          for (int e = 0; e < 32; ++e) dst[(size_t)(c + e) * p] = __float2half_rn(__uint_as_float(r[e]) * inv);
+        }
       }
+    }
+  } else {
+    // partial results of this part of the keys: row 0 = maxima, row 1 = sums, rows 2.. = accumulator
+    // columns, each row 128 features wide (consecutive lanes write consecutive words)
+    const size_t part_stride = (size_t)(d + 2) * 128;
+    float* mine = prm.part + ((size_t)unit * nsplit + sp) * part_stride;
+    if (warp < 4 && ok) {
+      const int fl = warp * 32 + lane;
+      const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16) + kK2OCol;
+      mine[fl] = row_max;
+      mine[128 + fl] = zsum;
+      for (int c = 0; c < d; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(tb + c, r);
+        tmem_wait_ld(r);
+#pragma unroll
+        for (int e = 0; e < 32; ++e) mine[(size_t)(2 + c + e) * 128 + fl] = __uint_as_float(r[e]);
+      }
+    }
+    __threadfence();
+    __syncthreads();
+    __shared__ int last_arrival;
+    if (tid == 0) last_arrival = (atomicAdd(prm.counters + unit, 1) == nsplit - 1) ? 1 : 0;
+    __syncthreads();
+    if (last_arrival && ok) {
+      __threadfence();
+      // merge: feature fl, half of the d columns per thread; the partial results bypass L1
+      const float* all = prm.part + (size_t)unit * nsplit * part_stride;
+      const int fl = tid & 127, half = tid >> 7;
+      const int f = i0 + fl;
+      float m_all = -INFINITY;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (q < nsplit) m_all = fmaxf(m_all, __ldcg(all + q * part_stride + fl));
+      float scale[4] = {0.f, 0.f, 0.f, 0.f};
+      float z_all = 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q < nsplit) {
+          scale[q] = __expf(__ldcg(all + q * part_stride + fl) - m_all);
+          z_all = fmaf(scale[q], __ldcg(all + q * part_stride + 128 + fl), z_all);
+        }
+      }
+      if (half == 0 && f < p) prm.weight[(size_t)head * p + f] = m_all + __logf(z_all);
+      const float inv = 1.f / z_all;
+      __half* dst = prm.aT16 + (size_t)head * d * p + f;
+      // sixteen columns at a time so that up to 64 loads are in flight per thread
+      for (int c0 = half * (d >> 1); c0 < (half + 1) * (d >> 1); c0 += 16) {
+        float v[4][16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (q < nsplit) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[q][e] = __ldcg(all + q * part_stride + (size_t)(2 + c0 + e) * 128 + fl);
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          float acc = 0.f;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (q < nsplit) acc = fmaf(scale[q], v[q][e], acc);
+          if (f < p) dst[(size_t)(c0 + e) * p] = __float2half_rn(acc * inv);
+        }
+      }
+      if (tid == 0) prm.counters[unit] = 0;
     }
   }
   tcgen05_fence_before();

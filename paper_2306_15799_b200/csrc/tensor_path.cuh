@@ -146,9 +146,39 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
   return 0;
 }
 
+// Key splits of stage 2: with few (head, feature tile) pairs the keys are divided over up to four
+// CTAs per pair, as long as all of them fit on the machine at once.
+inline int k2_nsplit(bool performer, int BH, int k, int p) {
+  if (!performer) return 1;
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+  }
+  const int units = BH * ((p + 127) / 128);
+  const int chunks = (k + kK2Chunk - 1) / kK2Chunk;
+  int ns = sms / units;
+  if (ns > chunks) ns = chunks;
+  if (ns > 4) ns = 4;
+  return ns < 1 ? 1 : ns;
+}
+
+// scratch floats for the partial results of a split stage 2, sized for the largest split the
+// problem could get on any device (so the workspace size does not depend on the device)
+inline size_t k2_part_floats(bool performer, int BH, int d, int k, int p) {
+  if (!performer) return 0;
+  int chunks = (k + kK2Chunk - 1) / kK2Chunk;
+  if (chunks > 4) chunks = 4;
+  if (chunks < 2) return 0;
+  return (size_t)BH * ((p + 127) / 128) * chunks * (size_t)(d + 2) * 128;
+}
+
 // ---- stage 2: per-feature summaries a (fp16, transposed) and weights b / z from K', V' --------
 inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const void* W, float* weight,
-                     __half* aT16, int BH, int d, int k, int p, int* status, cudaStream_t st, int* cuda_err) {
+                     __half* aT16, float* part, int* counters, int BH, int d, int k, int p, int* status,
+                     cudaStream_t st, int* cuda_err) {
   if (performer) {
     const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
     const unsigned bW[2] = {64, 128};
@@ -165,11 +195,14 @@ inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const vo
   prm.aT16 = aT16;
   prm.status = status;
   prm.trace = nullptr;
+  prm.nsplit = (part && counters) ? k2_nsplit(performer, BH, k, p) : 1;
+  prm.part = part;
+  prm.counters = counters;
   auto fn = performer ? k2_key_side<true> : k2_key_side<false>;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK2SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   // the RNN kernel ignores tmW; pass any valid map
-  fn<<<BH * prm.ftiles, kK2Threads, kK2SmemBytes, st>>>(performer ? tm.W2.map : tm.kpvp.map, prm);
+  fn<<<BH * prm.ftiles * prm.nsplit, kK2Threads, kK2SmemBytes, st>>>(performer ? tm.W2.map : tm.kpvp.map, prm);
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
