@@ -7,7 +7,10 @@
 //   RNN         f_ij = elu(k'_ji) + 1,  z_i = sum_j f_ij,  a_i = sum_j f_ij v'_j / z_i
 //
 // One CTA owns 128 features of one head and walks the keys in chunks of 128.  K' and V' arrive as
-// fp32 (stage 1's workspace) and are split on the fly into bf16 / fp16 terms so that the tensor-core
+// fp32 (stage 1's workspace): a bulk copy brings the rows of a chunk, which are contiguous, into a
+// staging buffer while the previous chunk's MMAs run, and short rolled loops (each part of this
+// kernel runs only a few times per CTA, so its time is largely instruction fetch and compact code
+// matters) split them into bf16 / fp16 terms so that the tensor-core
 // products are fp32-accurate: K' = hi + mid + lo (three bf16 terms, exact to 24 bits) against the
 // exact bf16 W, and -|k'|^2/2 as three bf16 terms in one extra 16-wide contraction step; V' = hi + lo
 // in fp16.  L for all k keys sits in TMEM (k <= 512 columns); the thread that owns a row takes its
@@ -42,8 +45,9 @@ struct K2Params {
 
 constexpr int kK2Threads = 256;
 constexpr int kK2Chunk = 128;  // keys per chunk (the last chunk may hold 64)
-// shared memory: W tile (<= 32 KB) | ones 4 KB | -|k'|^2/2 tile 4 KB | three 32 KB operand tiles | barriers
-constexpr int kK2SmemBytes = 32768 + 4096 + 4096 + 3 * 32768 + 256 + 1024;
+// shared memory: W tile (<= 32 KB) | ones 4 KB | -|k'|^2/2 tile 4 KB | three 32 KB operand tiles |
+// 64 KB fp32 staging (128 rows x d <= 128) | barriers
+constexpr int kK2SmemBytes = 32768 + 4096 + 4096 + 3 * 32768 + 65536 + 256 + 1024;
 constexpr int kK2OCol = 256;   // TMEM column of the a accumulator
 
 // two floats -> {lo: bf16(a), hi: bf16(b)} with one rounding instruction
@@ -70,9 +74,11 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   const uint32_t sm_ones = base + 32768;
   const uint32_t sm_nrm = sm_ones + 4096;
   const uint32_t sm_op = sm_nrm + 4096;          // 3 x 32 KB, 1024-aligned
-  const uint32_t bar_w = sm_op + 3 * 32768;
+  const uint32_t sm_stage = sm_op + 3 * 32768;   // fp32 rows of the current chunk
+  const uint32_t bar_w = sm_stage + 65536;
   const uint32_t bar_mma = bar_w + 8;
-  const uint32_t tmem_slot = bar_w + 16;
+  const uint32_t bar_stage = bar_w + 16;
+  const uint32_t tmem_slot = bar_w + 32;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
 
@@ -100,6 +106,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     abort_flag = 0;
     mbar_init(bar_w, 1);
     mbar_init(bar_mma, 1);
+    mbar_init(bar_stage, 1);
     fence_mbar_init();
   }
   if (warp == 4) {
@@ -144,16 +151,25 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   const int citers = kK2Chunk / (8 * rpi);       // 8 or 16 iterations cover the 128 rows of a chunk
   const uint32_t coff = (uint32_t)(ccol >> 6) * 16384 + (uint32_t)((ccol & 7) >> 2) * 8;
   const int cchunk = (ccol & 63) >> 3;           // 16-byte chunk of the 128-byte row before the swizzle
-  float4 ld[16];
-  // issues the loads of a whole chunk; they are in flight while the previous chunk's MMAs run
-  auto load_chunk = [&](const float* mat, int jc) {
-    const int rows = min(kK2Chunk, k - jc * kK2Chunk);
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      const int r = crow0 + t * 8 * rpi;
-      if (t < citers && r < rows)
-        ld[t] = *reinterpret_cast<const float4*>(mat + (size_t)(jc * kK2Chunk + r) * d + ccol);
-    }
+  // thread 0 starts the copy of a chunk's fp32 rows (contiguous in the workspace) into the staging buffer
+  uint32_t stage_phase = 0;
+  auto stage_chunk = [&](const float* mat, int jg) {
+    const int rows = min(kK2Chunk, k - jg * kK2Chunk);
+    const uint32_t bytes = (uint32_t)rows * d * 4;
+    mbar_arrive_expect_tx(bar_stage, bytes);
+    bulk_load(sm_stage, mat + (size_t)jg * kK2Chunk * d, bytes, bar_stage);
+  };
+  auto wait_stage = [&]() {
+    bool mine = true;
+    if (warp == 4) mine = mbar_wait(bar_stage, stage_phase, prm.status, &abort_flag);
+    ok = __syncthreads_and(mine) != 0;
+    stage_phase ^= 1;
+  };
+  auto stage_ld = [&](int r) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(sm_stage + (uint32_t)(r * d + ccol) * 4u));
+    return v;
   };
   // only the issuing warp polls the MMA barrier; everybody else sleeps in the block barrier
   auto wait_mma = [&]() {
@@ -170,21 +186,20 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       if (warp == 4) mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
       ok = __syncthreads_and(mine) != 0;
     }
-    load_chunk(Kp, jc_begin);
+    if (tid == 0) stage_chunk(Kp, jc_begin);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
       const int rows = min(kK2Chunk, k - (jc_begin + jc) * kK2Chunk);   // 64 or 128 keys in this chunk
+      wait_stage();
+      if (!ok) break;
       // ---- K' rows of the chunk: fp32 -> three bf16 tiles (K-major, 128-byte swizzle) and -|k'|^2/2
-      // three passes with independent work per row, so the conversions, the shuffles and the
-      // stores of different rows overlap instead of forming one long dependent chain
-      float sq[16];
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
+#pragma unroll 2
+      for (int t = 0; t < citers; ++t) {
         const int r = crow0 + t * 8 * rpi;
-        sq[t] = 0.f;
-        if (t < citers && r < rows) {
+        if (r < rows) {                                        // uniform over the warp (rows is even)
+          const float4 x = stage_ld(r);
           // packed conversions: one instruction rounds two values; a bf16 is the top half of an fp32
-          float a = ld[t].x, b = ld[t].y, c = ld[t].z, e = ld[t].w;
-          sq[t] = fmaf(a, a, fmaf(b, b, fmaf(c, c, e * e)));
+          float a = x.x, b = x.y, c = x.z, e = x.w;
+          float sq = fmaf(a, a, fmaf(b, b, fmaf(c, c, e * e)));
           const uint32_t h0 = pack_bf16x2(a, b), h1 = pack_bf16x2(c, e);
           a -= __uint_as_float(h0 << 16); b -= __uint_as_float(h0 & 0xffff0000u);
           c -= __uint_as_float(h1 << 16); e -= __uint_as_float(h1 & 0xffff0000u);
@@ -196,39 +211,30 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
           asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off), "r"(h0), "r"(h1) : "memory");
           asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 32768), "r"(m0), "r"(m1) : "memory");
           asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off + 65536), "r"(l0), "r"(l1) : "memory");
+          // |k'_r|^2 over the lanes that share the row
+          if (lpr == 32) sq += __shfl_xor_sync(0xffffffffu, sq, 16);
+#pragma unroll
+          for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          if ((lane % lpr) == 0) {
+            // B operand of the bias step: row r, columns 0..2 = three bf16 terms of -|k'_r|^2/2
+            float bb = -0.5f * sq;
+            const __nv_bfloat16 g0 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g0);
+            const __nv_bfloat16 g1 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g1);
+            const __nv_bfloat16 g2 = __float2bfloat16_rn(bb);
+            const uint32_t na = sm_nrm + (r >> 3) * 256 + (r & 7) * 16;
+            const uint32_t z = 0;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na),
+                         "r"((uint32_t)__bfloat16_as_ushort(g0) | ((uint32_t)__bfloat16_as_ushort(g1) << 16)),
+                         "r"((uint32_t)__bfloat16_as_ushort(g2)), "r"(z), "r"(z) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
+          }
         }
       }
-      // |k'_r|^2 over the lanes that share a row: sixteen independent butterfly reductions
-      if (lpr == 32) {
-#pragma unroll
-        for (int t = 0; t < 16; ++t) sq[t] += __shfl_xor_sync(0xffffffffu, sq[t], 16);
-      }
-#pragma unroll
-      for (int o = 8; o > 0; o >>= 1) {
-#pragma unroll
-        for (int t = 0; t < 16; ++t) sq[t] += __shfl_xor_sync(0xffffffffu, sq[t], o);
-      }
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
-        const int r = crow0 + t * 8 * rpi;
-        if (t < citers && (lane % lpr) == 0 && r < rows) {
-          // B operand of the bias step: row r, columns 0..2 = three bf16 terms of -|k'_r|^2/2
-          float bb = -0.5f * sq[t];
-          const __nv_bfloat16 g0 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g0);
-          const __nv_bfloat16 g1 = __float2bfloat16_rn(bb);  bb -= __bfloat162float(g1);
-          const __nv_bfloat16 g2 = __float2bfloat16_rn(bb);
-          const uint32_t na = sm_nrm + (r >> 3) * 256 + (r & 7) * 16;
-          const uint32_t z = 0;
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na),
-                       "r"((uint32_t)__bfloat16_as_ushort(g0) | ((uint32_t)__bfloat16_as_ushort(g1) << 16)),
-                       "r"((uint32_t)__bfloat16_as_ushort(g2)), "r"(z), "r"(z) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(na + 128), "r"(z), "r"(z), "r"(z), "r"(z) : "memory");
-        }
-      }
-      if (jc + 1 < nchunks) load_chunk(Kp, jc_begin + jc + 1);
-      else load_chunk(Vp, jc_begin);                             // first chunk of the second product
       fence_proxy_async_smem();
       __syncthreads();
+      // the staging buffer has been read out: start the next copy (the next K' chunk, or the first
+      // V' chunk of the second product) under this chunk's MMAs
+      if (tid == 0) stage_chunk(jc + 1 < nchunks ? Kp : Vp, jc + 1 < nchunks ? jc_begin + jc + 1 : jc_begin);
       K2_STAMP(1)
       if (tid == 128) {
         tcgen05_fence_after();
@@ -289,7 +295,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       tcgen05_fence_before();
     }
   } else {
-    load_chunk(Vp, 0);
+    if (tid == 0) stage_chunk(Vp, jc_begin);
     // RNN: f_ij = elu(k'_ji) + 1.  All threads stage 64 rows of K' in shared memory (coalesced), then
     // the thread that owns feature i walks down column i (row stride d + 1 words: no bank conflicts).
     float* stage = reinterpret_cast<float*>(base_ptr + (sm_op - base));
@@ -337,14 +343,17 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     const uint32_t idesc2 = make_idesc(kFmtF16, 0, /*B MN-major*/ 1, 128, (uint32_t)d);
     for (int jc = 0; jc < nchunks && ok; ++jc) {
       const int rows = min(kK2Chunk, k - (jc_begin + jc) * kK2Chunk);
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
+      wait_stage();
+      if (!ok) break;
+#pragma unroll 2
+      for (int t = 0; t < citers; ++t) {
         const int r = crow0 + t * 8 * rpi;
-        if (t < citers && r < rows) {
-          const __half2 hi0 = __floats2half2_rn(ld[t].x, ld[t].y), hi1 = __floats2half2_rn(ld[t].z, ld[t].w);
+        if (r < rows) {
+          const float4 x = stage_ld(r);
+          const __half2 hi0 = __floats2half2_rn(x.x, x.y), hi1 = __floats2half2_rn(x.z, x.w);
           const float2 b0 = __half22float2(hi0), b1 = __half22float2(hi1);
-          const __half2 lo0 = __floats2half2_rn(ld[t].x - b0.x, ld[t].y - b0.y);
-          const __half2 lo1 = __floats2half2_rn(ld[t].z - b1.x, ld[t].w - b1.y);
+          const __half2 lo0 = __floats2half2_rn(x.x - b0.x, x.y - b0.y);
+          const __half2 lo1 = __floats2half2_rn(x.z - b1.x, x.w - b1.y);
           const uint32_t off = sm_op + coff + r * 128 + ((cchunk ^ (r & 7)) << 4);
           asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(off), "r"(*reinterpret_cast<const uint32_t*>(&hi0)),
                        "r"(*reinterpret_cast<const uint32_t*>(&hi1)) : "memory");
@@ -352,9 +361,9 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
                        "r"(*reinterpret_cast<const uint32_t*>(&lo1)) : "memory");
         }
       }
-      if (jc + 1 < nchunks) load_chunk(Vp, jc_begin + jc + 1);
       fence_proxy_async_smem();
       __syncthreads();
+      if (tid == 0 && jc + 1 < nchunks) stage_chunk(Vp, jc_begin + jc + 1);
       K2_STAMP(4)
       if (tid == 128) {
         tcgen05_fence_after();
