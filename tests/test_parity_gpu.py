@@ -134,6 +134,10 @@ TENSOR_CASES = [
     _wl("tc_perf_d128_k192_m192", PERFORMER, "bf16", 1, 3, 640, 128, 192, 192, 105),
     _wl("tc_rnn_d64_k256", RNN, "bf16", 2, 3, 1024, 64, 256, 0, 106),
     _wl("tc_rnn_d128_k64", RNN, "bf16", 1, 2, 512, 128, 64, 0, 107),
+    # one 128-row tile per head, and key counts whose last 128-key chunk holds 64 keys
+    _wl("tc_perf_d64_k320_m256_n128", PERFORMER, "bf16", 1, 2, 128, 64, 320, 256, 109),
+    _wl("tc_perf_d128_k448_m128", PERFORMER, "bf16", 2, 1, 256, 128, 448, 128, 110),
+    _wl("tc_rnn_d128_k512_n128", RNN, "bf16", 1, 1, 128, 128, 512, 0, 111),
 ]
 
 
@@ -207,3 +211,18 @@ def test_auto_picks_tensor_path_when_the_shape_allows():
     odd = _wl("auto_simt", PERFORMER, "bf16", 1, 1, 200, 64, 64, 64, 108)      # N % 128 != 0
     pu.check_all_heads(odd)
     assert binding.flurka_last_path() == binding.PATH_SIMT
+
+
+@pytest.mark.parametrize("scale", [2.0, 0.05])
+def test_tensor_path_with_large_and_small_logits(scale):
+    """Q and K scaled away from the benchmark recipe: logits of several tens (sharply peaked
+    weights, every stabiliser at work) and logits near zero (almost uniform weights)."""
+    w = _wl("tc_perf_scaled", PERFORMER, "bf16", 1, 2, 512, 64, 128, 256, 112)
+    inputs = synth.make_inputs(w)
+    for name in ("Q", "K"):
+        inputs[name] = (inputs[name].double() * scale).to(inputs[name].dtype)
+    out = pu.run_gpu(w, inputs, binding.PATH_TENSOR).cpu().double().numpy()
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    assert np.isfinite(out).all()
+    for h in range(w.H):
+        pu.assert_close(out[0, h], pu.oracle_head(inputs, w, 0, h), "bf16", "scaled x%g head %d" % (scale, h))
