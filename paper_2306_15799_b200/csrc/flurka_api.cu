@@ -26,10 +26,12 @@ struct Problem {
 
 // Workspace layout (all offsets 256-byte aligned):
 //   kpvp    fp32 [2][BH][k][d]     K' then V'
+//   status  int32[4], then one arrival counter per (head, 128-feature tile) of stage 2
+//           (kpvp and status are adjacent: one memset per forward clears both)
 //   weight  fp32 [BH][p]           b_i (PERFORMER) or z_i (RNN)
 //   a32     fp32 [BH][p][d]        key-side summary, feature-major
 //   aT16    fp16 [BH][d][p]        the same, transposed, as the tensor-core B operand
-//   status  int32[4]
+//   part    fp32 partial results of a key-split stage 2 (tensor-core path only)
 struct Layout {
   size_t kpvp, weight, a32, aT16, status, status_bytes, part, total;
 };
@@ -42,12 +44,11 @@ Layout make_layout(const Problem& pr, bool with_split_scratch = true) {
   Layout L;
   size_t off = 0;
   L.kpvp = off;   off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
+  L.status_bytes = 16 + (with_split_scratch ? (size_t)pr.BH() * ((pr.p() + 127) / 128) * 4 : 0);
+  L.status = off; off = align256(off + L.status_bytes);
   L.weight = off; off = align256(off + (size_t)pr.BH() * pr.p() * 4);
   L.a32 = off;    off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 4);
   L.aT16 = off;   off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 2);
-  // four status words, then one arrival counter per (head, 128-feature tile) of stage 2
-  L.status_bytes = 16 + (with_split_scratch ? (size_t)pr.BH() * ((pr.p() + 127) / 128) * 4 : 0);
-  L.status = off; off = align256(off + L.status_bytes);
   const size_t part_floats = (with_split_scratch && !pr.fp32)
                                  ? k2_part_floats(pr.kernel == FLURKA_PERFORMER, pr.BH(), pr.d, pr.k, pr.p())
                                  : 0;
@@ -219,7 +220,8 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   int* status = (int*)(ws + L.status);
   const bool performer = pr.kernel == FLURKA_PERFORMER;
   int cuda_err = 0;
-  cudaError_t e = cudaMemsetAsync(kpvp, 0, (size_t)2 * pr.BH() * pr.k * pr.d * 4, st);
+  // one memset: the K', V' accumulators (the kernels add into them), the status words and the counters
+  cudaError_t e = cudaMemsetAsync(ws + L.kpvp, 0, L.status + L.status_bytes - L.kpvp, st);
   if (e != cudaSuccess) return cuda_fail(e);
   g.timer.mark(0, st);
   int rc;
@@ -303,9 +305,6 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
-  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, L.status_bytes, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-
   if (pr.fp32) {
     rc = run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
   } else {
@@ -537,10 +536,8 @@ extern "C" int flurka_forward_static_scratch(const void* Q, const void* K, const
   rc = static_scratch_address(&ws);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  // The array still holds the previous call's contents: the status words are cleared here and
-  // run_simt zeroes the K', V' accumulators before the kernels add into them.
-  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, 16, st);
-  if (e != cudaSuccess) return cuda_fail(e);
+  // The array still holds the previous call's contents: run_simt zeroes the K', V' accumulators
+  // and the status words before the kernels add into them.
   int launches = 0;
   if (pr.fp32) return run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
   return run_simt<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);

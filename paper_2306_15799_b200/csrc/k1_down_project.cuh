@@ -147,6 +147,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
       // ------------------------------------------------ epilogue: TMEM -> smem -> TMA reduce-add
       const int q = warp & 3;                                // TMEM lane quadrant of this warp
       bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
+      if (warp == 2 && lane == 0) grid_launch_dependents();   // only the epilogue is left
       if (p.trace && warp == 2 && lane == 0) p.trace[4 * blockIdx.x + 2] = global_timer_ns();
       if (ok) {
         tcgen05_fence_after();

@@ -141,6 +141,8 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   bool ok = true;
   uint32_t mma_phase = 0;
   K2_STAMP(0)
+  // everything above (and the W tile on its way) is independent of stage 1
+  grid_dependency_wait();
 
   // conversion geometry: a warp instruction reads whole rows (d/4 lanes x float4 per row), so the fp32
   // rows arrive in full 128-byte lines; each lane converts four consecutive columns of its rows
@@ -383,6 +385,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     }
   }
 
+  if (tid == 0) grid_launch_dependents();   // only the write-out (and the merge) is left
   // ---- a_i = accumulator / z_i, stored transposed ([d][p], fp16) for stage 3
   if (nsplit == 1) {
     if (warp < 4 && ok) {

@@ -147,17 +147,22 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const int kq = d >> 6;      // 64-wide K-blocks of the Q / W tiles
   const int kp = p >> 6;      // 64-wide K-blocks of a^T
 
+  if (ntiles > 0 && warp == 0 && lane == 0) {
+    // W is an input, not a result of stage 2: its load starts before the dependency wait
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmAT);
+    if (kPerformer) {
+      prefetch_tmap(&tmW);
+      mbar_arrive_expect_tx(bar_wfull, (uint32_t)p * d * 2);
+      for (int kb = 0; kb < kq; ++kb) tma_load_2d(base + L.w + kb * (p * 128), &tmW, bar_wfull, kb * 64, 0);
+    }
+  }
+  grid_dependency_wait();
+
   if (ntiles > 0) {
     if (warp == 0 && lane == 0) {
       // ============================================================ TMA producer
-      prefetch_tmap(&tmQ);
-      prefetch_tmap(&tmAT);
       bool ok = true;
-      if (kPerformer) {
-        prefetch_tmap(&tmW);
-        mbar_arrive_expect_tx(bar_wfull, (uint32_t)p * d * 2);
-        for (int kb = 0; kb < kq; ++kb) tma_load_2d(base + L.w + kb * (p * 128), &tmW, bar_wfull, kb * 64, 0);
-      }
       int head_prev = -1, events = 0;
       int issued = 0;
       for (int i = 0; i < ntiles && ok; ++i) {

@@ -21,6 +21,19 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
+// ------------------------------------------------------------------------------ dependent launch
+// A kernel launched with programmatic stream serialisation may start while its predecessor in the
+// stream is still running; it must not touch the predecessor's results before this wait (which
+// returns once the predecessor has completed and its writes are visible).  Without the launch
+// attribute the wait returns at once.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream be scheduled once every CTA of this grid has said so or has
+// exited.  Called late in a CTA's life: when the last CTA calls it, every CTA of this grid already
+// holds its SM, so the successor's CTAs can never keep one of ours from starting.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

@@ -146,6 +146,25 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
   return 0;
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the previous
+// kernel in the stream is finishing (its CTAs call griddepcontrol.launch_dependents late in their
+// life) and waits in griddepcontrol.wait before it touches that kernel's results.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after_predecessor(void (*fn)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
+                                            Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3((unsigned)block, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, fn, KArgs(args)...);
+}
+
 // Key splits of stage 2: with few (head, feature tile) pairs the keys are divided over up to four
 // CTAs per pair, as long as all of them fit on the machine at once.
 inline int k2_nsplit(bool performer, int BH, int k, int p) {
@@ -202,7 +221,9 @@ inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const vo
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK2SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   // the RNN kernel ignores tmW; pass any valid map
-  fn<<<BH * prm.ftiles * prm.nsplit, kK2Threads, kK2SmemBytes, st>>>(performer ? tm.W2.map : tm.kpvp.map, prm);
+  e = launch_after_predecessor(fn, BH * prm.ftiles * prm.nsplit, kK2Threads, kK2SmemBytes, st,
+                               performer ? tm.W2.map : tm.kpvp.map, prm);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
@@ -244,7 +265,9 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
   int grid = sm_count();
   if (grid > prm.total_tiles) grid = prm.total_tiles;
   // the RNN kernel ignores tmW; pass any valid map
-  fn<<<grid, kK3Threads, L.total, st>>>(tm.Q.map, performer ? tm.W.map : tm.Q.map, tm.aT.map, prm);
+  e = launch_after_predecessor(fn, grid, kK3Threads, L.total, st, tm.Q.map, performer ? tm.W.map : tm.Q.map,
+                               tm.aT.map, prm);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
