@@ -11,8 +11,12 @@
 // The per-feature summaries a_i, b_i (or z_i) come from stage 2.  A persistent CTA walks a
 // contiguous range of 128-row tiles; warp 0 feeds TMA, warps 1 and 3 issue the first and the second
 // products, warp 2 rebuilds the bias operand when the head changes, and two groups of four warps
-// alternate tiles (TMEM is split in two 256-column halves: S/p in columns 0.., O in columns 128..
-// of each half).  Every thread of a group owns one output row and writes it with 32-byte stores.
+// alternate tiles.  TMEM holds S/p and O of the tiles in flight: two 256-column buffers (S/p in
+// columns 0.., O in columns 128..) in general; four 128-column buffers (S/p in columns 0.., O in
+// columns 64.., which S has vacated by then) when d = 64 and p <= 128.  With four buffers each group
+// has two tiles in flight and reads tile i-2 out after it has handed tile i to the second product,
+// so it never waits for a product it has just asked for.  Every thread of a group owns one output
+// row and writes it with 32-byte stores.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -81,15 +85,15 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const uint32_t bars = base + L.bars;
   const uint32_t bar_qfull = bars;            // [4]   Q tile landed
   const uint32_t bar_qempty = bars + 32;      // [4]   Q tile consumed (MMA commit, or 128 readers for RNN)
-  const uint32_t bar_sfull = bars + 64;       // [2]   S ready in TMEM (PERFORMER)
-  const uint32_t bar_pfull = bars + 80;       // [2]   p written to TMEM by the 128 row owners
-  const uint32_t bar_ofull = bars + 96;       // [2]   O ready in TMEM
-  const uint32_t bar_sfree = bars + 112;      // [2]   TMEM half read out, may be overwritten
-  const uint32_t bar_wfull = bars + 128;      //       W resident
-  const uint32_t bar_drained = bars + 136;    //       every MMA of the previous head is complete
-  const uint32_t bar_atfull = bars + 144;     //       a^T of the new head resident
-  const uint32_t bar_biasready = bars + 152;  //       bias operand / scale vector of the new head built
-  const uint32_t tmem_slot = bars + 192;
+  const uint32_t bar_sfull = bars + 64;       // [4]   S ready in TMEM (PERFORMER)
+  const uint32_t bar_pfull = bars + 96;       // [4]   p written to TMEM by the 128 row owners
+  const uint32_t bar_ofull = bars + 128;      // [4]   O ready in TMEM
+  const uint32_t bar_sfree = bars + 160;      // [4]   TMEM buffer read out, may be overwritten
+  const uint32_t bar_wfull = bars + 192;      //       W resident
+  const uint32_t bar_drained = bars + 200;    //       every MMA of the previous head is complete
+  const uint32_t bar_atfull = bars + 208;     //       a^T of the new head resident
+  const uint32_t bar_biasready = bars + 216;  //       bias operand / scale vector of the new head built
+  const uint32_t tmem_slot = bars + 232;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
 
@@ -106,7 +110,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       mbar_init(bar_qfull + 8 * i, 1);
       mbar_init(bar_qempty + 8 * i, kPerformer ? 1 : 128);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {
       mbar_init(bar_sfull + 8 * i, 1);
       mbar_init(bar_pfull + 8 * i, 128);
       mbar_init(bar_ofull + 8 * i, 1);
@@ -146,6 +150,11 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 
   const int kq = d >> 6;      // 64-wide K-blocks of the Q / W tiles
   const int kp = p >> 6;      // 64-wide K-blocks of a^T
+  // TMEM buffers: tile i uses buffer i % NB, its barriers flip once per NB tiles
+  const int NB = (d == 64 && p <= 128) ? 4 : 2;
+  const int nb_shift = NB == 4 ? 2 : 1;
+  const uint32_t buf_cols = 512u / NB;
+  const uint32_t o_col = NB == 4 ? 64u : 128u;
 
   if (ntiles > 0 && warp == 0 && lane == 0) {
     // W is an input, not a result of stage 2: its load starts before the dependency wait
@@ -202,7 +211,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         long long mlast = mtracing ? clock64() : 0;
         for (int i = 0; i < ntiles && ok; ++i) {
           const int head = (t_begin + i) / prm.tiles_per_head;
-          const int buf = i & 1, st = i % NS;
+          const int buf = i & (NB - 1), st = i % NS;
           if (head != head_prev) {
             ok = mbar_wait(bar_biasready, events & 1, prm.status, &abort_flag);
             if (!ok) break;
@@ -210,12 +219,12 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             ++events;
           }
           // TMEM half `buf` must have been read out by the row owners of tile i-2
-          if (i >= 2) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> 1) - 1) & 1, prm.status, &abort_flag);
+          if (i >= NB) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> nb_shift) - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
           if (!ok) break;
           tcgen05_fence_after();
           if (mtracing) { const long long now = clock64(); macc[0] += now - mlast; mlast = now; }
-          const uint32_t tb = tmem + buf * 256;
+          const uint32_t tb = tmem + buf * buf_cols;
           const uint32_t qb = base + L.q + st * q_stage_bytes;
           for (int kb = 0; kb < kq; ++kb) {
             const uint64_t ad = make_sdesc(qb + kb * 16384, 16, 1024, kSwizzle128);
@@ -251,22 +260,22 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       long long mlast = mtracing ? clock64() : 0;
       for (int j = 0; j < ntiles && ok; ++j) {
         const int head = (t_begin + j) / prm.tiles_per_head;
-        const int buf = j & 1;
+        const int buf = j & (NB - 1);
         if (head != head_prev) {
           ok = mbar_wait(bar_atfull, events & 1, prm.status, &abort_flag);
           if (!ok) break;
           head_prev = head;
           ++events;
         }
-        ok = mbar_wait(bar_pfull + 8 * buf, (j >> 1) & 1, prm.status, &abort_flag);
+        ok = mbar_wait(bar_pfull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
         if (mtracing) { const long long now = clock64(); macc[0] += now - mlast; mlast = now; }
-        const uint32_t tb = tmem + buf * 256;
+        const uint32_t tb = tmem + buf * buf_cols;
         // four 16-wide steps per call: one 64-feature block of p (TMEM) against one block of a^T
         for (int kb = 0; kb < kp; ++kb) {
           const uint64_t bd = make_sdesc(base + L.aT + kb * (d * 128), 16, 1024, kSwizzle128);
-          mma_ts_x4(tb + 128, tb + kb * 32, bd, 2, idesc2, kb > 0 ? 1u : 0u);
+          mma_ts_x4(tb + o_col, tb + kb * 32, bd, 2, idesc2, kb > 0 ? 1u : 0u);
         }
         mma_commit(bar_ofull + 8 * buf);
         const bool last_of_head = (j + 1 < ntiles) && ((t_begin + j + 1) / prm.tiles_per_head != head);
@@ -332,12 +341,50 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       long long tlast = tracing ? clock64() : 0;
 #define K3_STAMP(slot) \
   if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
-      for (int i = grp; i < ntiles && ok; i += 2) {
-        const int tile = t_begin + i;
+      // read-out of tile j: O / sum -> bf16 -> this thread's output row, 32 bytes per store
+      auto read_out = [&](int j, float inv) -> bool {
+        const int tile = t_begin + j;
         const int head = tile / prm.tiles_per_head;
         const int row0 = (tile % prm.tiles_per_head) * 128;
-        const int buf = i & 1, st = i % NS;
-        const uint32_t tb = tmem + buf * 256 + lane_off;
+        const int buf = j & (NB - 1);
+        const uint32_t tb = tmem + buf * buf_cols + lane_off + o_col;
+        if (!mbar_wait(bar_ofull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag)) return false;
+        tcgen05_fence_after();
+        K3_STAMP(3)
+        __nv_bfloat16* orow = prm.out + ((size_t)head * prm.N + row0 + row) * d;
+        for (int c = 0; c < d; c += 64) {
+          uint32_t ra[32], rb[32];
+          tmem_ld32(tb + c, ra);
+          tmem_ld32(tb + c + 32, rb);
+          tmem_wait_ld(ra);
+          tmem_wait_ld(rb);
+          if (c + 64 >= d) {
+            // everything this tile needs from TMEM is in registers: hand the buffer back before storing
+            tcgen05_fence_before();
+            mbar_arrive(bar_sfree + 8 * buf);
+          }
+#pragma unroll
+          for (int g8 = 0; g8 < 4; ++g8) {
+            const uint32_t* src = g8 < 2 ? ra : rb;
+            uint32_t v[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(src[(g8 & 1) * 16 + 2 * e]) * inv,
+                                                              __uint_as_float(src[(g8 & 1) * 16 + 2 * e + 1]) * inv);
+              v[e] = *reinterpret_cast<const uint32_t*>(&o2);
+            }
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(orow + c + g8 * 16),
+                         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                         : "memory");
+          }
+        }
+        K3_STAMP(4)
+        return true;
+      };
+      float inv_prev = 0.f;                            // four buffers: 1 / sum of the group's previous tile
+      for (int i = grp; i < ntiles && ok; i += 2) {
+        const int buf = i & (NB - 1), st = i % NS;
+        const uint32_t tb = tmem + buf * buf_cols + lane_off;
         float denom = 0.f, denom1 = 0.f;
         // count head changes the same way the other roles do (both groups see every tile index)
         for (int j = (i >= 2 ? i - 1 : 0); j <= i; ++j) {
@@ -345,7 +392,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           if (hj != head_prev) { head_prev = hj; ++events; }
         }
         if (kPerformer) {
-          ok = mbar_wait(bar_sfull + 8 * buf, (i >> 1) & 1, prm.status, &abort_flag);
+          ok = mbar_wait(bar_sfull + 8 * buf, (i >> nb_shift) & 1, prm.status, &abort_flag);
           if (!ok) break;
           tcgen05_fence_after();
           K3_STAMP(0)
@@ -412,7 +459,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           }
         } else {
           // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
-          if (i >= 2) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> 1) - 1) & 1, prm.status, &abort_flag);
+          if (i >= NB) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> nb_shift) - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
           if (!ok) break;
@@ -448,41 +495,17 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         mbar_arrive(bar_pfull + 8 * buf);
         K3_STAMP(2)
 
-        // ---- O / denom -> bf16 -> this thread's output row, 32 bytes per store
-        ok = mbar_wait(bar_ofull + 8 * buf, (i >> 1) & 1, prm.status, &abort_flag);
-        if (!ok) break;
-        tcgen05_fence_after();
-        K3_STAMP(3)
         const float inv = 1.f / fmaxf(denom + denom1, 1.17549435e-38f);
-        __nv_bfloat16* orow = prm.out + ((size_t)head * prm.N + row0 + row) * d;
-        for (int c = 0; c < d; c += 64) {
-          uint32_t ra[32], rb[32];
-          tmem_ld32(tb + 128 + c, ra);
-          tmem_ld32(tb + 128 + c + 32, rb);
-          tmem_wait_ld(ra);
-          tmem_wait_ld(rb);
-          if (c + 64 >= d) {
-            // everything this tile needs from TMEM is in registers: hand the half back before storing
-            tcgen05_fence_before();
-            mbar_arrive(bar_sfree + 8 * buf);
-          }
-#pragma unroll
-          for (int g8 = 0; g8 < 4; ++g8) {
-            const uint32_t* src = g8 < 2 ? ra : rb;
-            uint32_t v[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(src[(g8 & 1) * 16 + 2 * e]) * inv,
-                                                              __uint_as_float(src[(g8 & 1) * 16 + 2 * e + 1]) * inv);
-              v[e] = *reinterpret_cast<const uint32_t*>(&o2);
-            }
-            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(orow + c + g8 * 16),
-                         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-                         : "memory");
-          }
+        if (NB == 4) {
+          // two tiles of this group are in flight: read out the previous one, whose second product
+          // has had this tile's passes to finish
+          if (i >= 2) ok = read_out(i - 2, inv_prev);
+          inv_prev = inv;
+        } else {
+          ok = read_out(i, inv);
         }
-        K3_STAMP(4)
       }
+      if (NB == 4 && ok && ntiles > grp) (void)read_out(grp + 2 * ((ntiles - 1 - grp) / 2), inv_prev);
 #undef K3_STAMP
       if (tracing) {
         for (int sidx = 0; sidx < 6; ++sidx) prm.trace[((size_t)blockIdx.x * 3 + grp) * 8 + sidx] = tacc[sidx];
