@@ -9,7 +9,7 @@
 //   RNN         p = (elu(q) + 1) z / max z  straight from the Q tile, then the same second product.
 //
 // The per-feature summaries a_i, b_i (or z_i) come from stage 2.  A persistent CTA walks a
-// contiguous range of 128-row tiles; warp 0 feeds TMA, warps 1 and 3 issue the first and the second
+// contiguous range of 128-row tiles; warp 0 feeds Q tiles by TMA, warps 1 and 3 issue the first and the second
 // products, warp 2 rebuilds the bias operand when the head changes, and two groups of four warps
 // alternate tiles.  TMEM holds S/p and O of the tiles in flight: two 256-column buffers (S/p in
 // columns 0.., O in columns 128..) in general; four 128-column buffers (S/p in columns 0.., O in
@@ -171,21 +171,14 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   if (ntiles > 0) {
     if (warp == 0 && lane == 0) {
       // ============================================================ TMA producer
+      // Q tiles only: they do not depend on the head's operands, so the ring keeps running ahead
+      // across a change of head (a^T is reloaded by the operand builder, which waits for the drain)
       bool ok = true;
-      int head_prev = -1, events = 0;
       int issued = 0;
       for (int i = 0; i < ntiles && ok; ++i) {
         const int tile = t_begin + i;
         const int head = tile / prm.tiles_per_head;
         const int row0 = (tile % prm.tiles_per_head) * 128;
-        if (head != head_prev) {
-          if (events > 0) ok = mbar_wait(bar_drained, (events - 1) & 1, prm.status, &abort_flag);
-          if (!ok) break;
-          mbar_arrive_expect_tx(bar_atfull, (uint32_t)d * p * 2);
-          for (int kb = 0; kb < kp; ++kb) tma_load_3d(base + L.aT + kb * (d * 128), &tmAT, bar_atfull, kb * 64, 0, head);
-          head_prev = head;
-          ++events;
-        }
         const int st = i % NS;
         if (i >= NS) ok = mbar_wait(bar_qempty + 8 * st, ((i / NS) - 1) & 1, prm.status, &abort_flag);
         if (!ok) break;
@@ -295,6 +288,11 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (head == head_prev) continue;
         if (events > 0) ok = mbar_wait(bar_drained, (events - 1) & 1, prm.status, &abort_flag);
         if (!ok) break;
+        if (lane == 0) {
+          // a^T of the new head, the resident B operand of the second product
+          mbar_arrive_expect_tx(bar_atfull, (uint32_t)d * p * 2);
+          for (int kb = 0; kb < kp; ++kb) tma_load_3d(base + L.aT + kb * (d * 128), &tmAT, bar_atfull, kb * 64, 0, head);
+        }
         const float* wv = prm.weight + (size_t)head * p;
         float mx = -INFINITY;
         for (int f = lane; f < p; f += 32) mx = fmaxf(mx, wv[f]);
@@ -459,8 +457,9 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           }
         } else {
           // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
-          if (i >= NB) ok = mbar_wait(bar_sfree + 8 * buf, ((i >> nb_shift) - 1) & 1, prm.status, &abort_flag);
-          if (ok) ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
+          // (no wait for the buffer: this thread has itself read out the tile that used it before, and
+          // the second product starts only when all 128 owners have said so)
+          ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
           if (!ok) break;
           K3_STAMP(0)
@@ -475,13 +474,19 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
               uint32_t v[4];
               asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(a));
+              // the eight scale factors of these features: two 16-byte loads (every lane reads the same words)
+              const float4 s0 = *reinterpret_cast<const float4*>(sc + col);
+              const float4 s1 = *reinterpret_cast<const float4*>(sc + col + 4);
+              const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const __nv_bfloat162 qq = *reinterpret_cast<const __nv_bfloat162*>(&v[e]);
-                const float x0 = __bfloat162float(qq.x), x1 = __bfloat162float(qq.y);
-                const float f0 = (x0 > 0.f ? x0 + 1.f : __expf(x0)) * sc[col + 2 * e];
-                const float f1 = (x1 > 0.f ? x1 + 1.f : __expf(x1)) * sc[col + 2 * e + 1];
-                denom += f0 + f1;
+                // a bf16 is the upper half of an fp32
+                const float x0 = __uint_as_float(v[e] << 16), x1 = __uint_as_float(v[e] & 0xffff0000u);
+                // elu(x) + 1 = max(x, 0) + exp(min(x, 0))
+                const float f0 = (fmaxf(x0, 0.f) + ex2_approx(fminf(x0, 0.f) * kLog2e)) * scv[2 * e];
+                const float f1 = (fmaxf(x1, 0.f) + ex2_approx(fminf(x1, 0.f) * kLog2e)) * scv[2 * e + 1];
+                denom += f0;
+                denom1 += f1;
                 const __half2 hh = __floats2half2_rn(f0, f1);
                 h[ch * 4 + e] = *reinterpret_cast<const uint32_t*>(&hh);
               }
