@@ -90,8 +90,11 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
 /*
  * flurka_forward_host -- the same operation (Eq. (2)) on HOST buffers (same shapes and element types).
  * Copies the inputs to the device (cudaMemcpyAsync; pinned host memory makes them asynchronous),
- * runs flurka_forward, copies `out` back and synchronises `stream` before returning.  Device staging
- * buffers are allocated by the library on first use and re-used while they are large enough.
+ * runs flurka_forward, copies `out` back and synchronises `stream` before returning.  Larger calls go
+ * through the heads in up to eight groups, so that the output of one group is copied back (on a second,
+ * library-owned stream) while the inputs of the next are copied in; flurka_last_status() then covers all
+ * groups, flurka_debug_copy() the last one.  Device staging buffers are allocated by the library on
+ * first use and re-used while they are large enough.
  */
 int flurka_forward_host(const void* Q, const void* K, const void* V, const void* E, const void* F,
                         const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,

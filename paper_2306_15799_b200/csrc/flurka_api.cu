@@ -3,6 +3,8 @@
 #include "flurka.h"
 
 #include <cuda_runtime.h>
+
+#include <algorithm>
 #include <stdint.h>
 
 #include "simt_kernels.cuh"
@@ -73,6 +75,10 @@ struct State {
   // host-buffer entry point: device staging
   void* stage = nullptr;
   size_t stage_bytes = 0;
+  cudaStream_t out_stream = nullptr;   // device-to-host copies of finished head groups
+  cudaEvent_t group_done[8] = {};      // one per head group of a host-buffer call
+  cudaEvent_t out_done = nullptr;
+  bool keep_status = false;            // later head groups of one host-buffer call keep the status words
   StageTimer timer;
   TensorMaps maps;
 };
@@ -221,7 +227,9 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   const bool performer = pr.kernel == FLURKA_PERFORMER;
   int cuda_err = 0;
   // one memset: the K', V' accumulators (the kernels add into them), the status words and the counters
-  cudaError_t e = cudaMemsetAsync(ws + L.kpvp, 0, L.status + L.status_bytes - L.kpvp, st);
+  // (a later head group of a host-buffer call leaves the status words, which only ever gain bits, and
+  // the counters, which stage 2 hands back at zero)
+  cudaError_t e = cudaMemsetAsync(ws + L.kpvp, 0, (g.keep_status ? L.status : L.status + L.status_bytes) - L.kpvp, st);
   if (e != cudaSuccess) return cuda_fail(e);
   g.timer.mark(0, st);
   int rc;
@@ -361,20 +369,55 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
   const size_t qn = pr.qkv_elems() * pr.esize(), en = pr.ef_elems() * pr.esize(),
                wn = pr.w_elems() * pr.esize();
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(dQ, Q, qn, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemcpyAsync(dK, K, qn, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaMemcpyAsync(dV, V, qn, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
   if ((e = cudaMemcpyAsync(dE, E, en, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
   if ((e = cudaMemcpyAsync(dF, F, en, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
   if (wn && (e = cudaMemcpyAsync(dW, W, wn, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(e);
-  rc = flurka_forward(dQ, dK, dV, dE, dF, wn ? dW : nullptr, variant, B, H, N, d, k, m, dO, stream);
-  if (rc) {
-    cudaStreamSynchronize(st);
-    return rc;
+
+  // The heads are independent, so the call works through them in up to eight groups: while the
+  // inputs of one group travel to the device, the output of the group before travels back on a second
+  // stream (the link is full duplex), and the compute of a group hides under the copies.
+  const int heads = pr.BH();
+  int groups = (int)std::min<size_t>(8, qn >> 20);           // at least 1 MiB of Q per group
+  groups = std::max(1, std::min(groups, heads));
+  if (groups > 1 && !g.out_stream) {
+    if ((e = cudaStreamCreateWithFlags(&g.out_stream, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+    for (int i = 0; i < 8; ++i)
+      if ((e = cudaEventCreateWithFlags(&g.group_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventCreateWithFlags(&g.out_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
   }
-  if ((e = cudaMemcpyAsync(out, dO, qn, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
-  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e);
+  const size_t head_bytes = (size_t)N * d * pr.esize();
+  rc = FLURKA_OK;
+  for (int gi = 0; gi < groups && rc == FLURKA_OK; ++gi) {
+    const int h0 = (int)((long long)heads * gi / groups), h1 = (int)((long long)heads * (gi + 1) / groups);
+    const size_t off = (size_t)h0 * head_bytes, len = (size_t)(h1 - h0) * head_bytes;
+    if ((e = cudaMemcpyAsync(dQ + off, (const char*)Q + off, len, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dK + off, (const char*)K + off, len, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dV + off, (const char*)V + off, len, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+      rc = cuda_fail(e);
+      break;
+    }
+    g.keep_status = gi > 0;
+    rc = flurka_forward(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, 1, h1 - h0, N, d, k, m,
+                        dO + off, stream);
+    g.keep_status = false;
+    if (rc) break;
+    if (groups == 1) {
+      if ((e = cudaMemcpyAsync(out, dO, qn, cudaMemcpyDeviceToHost, st)) != cudaSuccess) rc = cuda_fail(e);
+    } else {
+      if ((e = cudaEventRecord(g.group_done[gi], st)) != cudaSuccess ||
+          (e = cudaStreamWaitEvent(g.out_stream, g.group_done[gi], 0)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)out + off, dO + off, len, cudaMemcpyDeviceToHost, g.out_stream)) != cudaSuccess)
+        rc = cuda_fail(e);
+    }
+  }
+  if (groups > 1) {
+    // the caller's stream also waits for the copies on the second stream
+    if (cudaEventRecord(g.out_done, g.out_stream) == cudaSuccess) cudaStreamWaitEvent(st, g.out_done, 0);
+  }
+  e = cudaStreamSynchronize(st);
+  if (rc) return rc;
+  if (e != cudaSuccess) return cuda_fail(e);
   return FLURKA_OK;
 }
 

@@ -91,6 +91,28 @@ def test_host_entry_point_matches_device_entry_point():
     assert torch.equal(host_out, dev_out) or float((host_out.float() - dev_out.float()).abs().max()) < 2e-2
 
 
+@pytest.mark.parametrize("variant,H", [(PERFORMER, 4), (RNN, 3)])
+def test_host_entry_point_in_head_groups(variant, H):
+    """Large enough (4 MiB / 3 MiB of Q) for the host entry point to work through the heads in groups,
+    copying finished groups back while the next ones are copied in; twice, to re-use its staging."""
+    w = _wl("host_groups", variant, "bf16", 2, H, 4096, 64, 64, 64, 42)
+    inputs = synth.make_inputs(w)
+    dev_out = pu.run_gpu(w, inputs).cpu()
+    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in inputs.items()}
+    for _ in range(2):
+        host_out = binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"],
+                                               pinned["W"], w.variant)
+        assert binding.flurka_last_status() == 0
+        # a group of heads is split over CTAs differently from the whole batch, so sums are taken in
+        # another order and intermediate roundings differ: outputs agree to a few bf16 ulps (2^-7 each)
+        diff = (host_out.float() - dev_out.float()).abs()
+        assert bool((diff <= 4 * 2.0 ** -7 * dev_out.float().abs() + 2e-3).all())
+    got = host_out.double().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            pu.assert_close(got[b, h], pu.oracle_head(inputs, w, b, h), "bf16", "host entry point, head (%d,%d)" % (b, h))
+
+
 def test_caller_workspace_and_too_small_workspace():
     w = _wl("ws_rnn_bf16", RNN, "bf16", 1, 2, 256, 64, 64, 0, 51)
     inputs = synth.make_inputs(w)
