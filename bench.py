@@ -326,12 +326,21 @@ def main():
         stage_bytes = [2 * BH * N * d * s + 2 * k * N * s + 2 * BH * k * d * 4,
                        2 * BH * k * d * 4 + m * d * s + BH * p * (d * 2 + 4),
                        2 * BH * N * d * s + m * d * s + BH * p * (d * 2 + 4)]
+        # exponentials go through the special-function unit: 16 per clock per SM, 148 SMs, at the
+        # maximum SM clock (nominal unit count x clock; there is no measured figure for this unit)
+        stage_exps = [0, k * p * BH, N * p * BH]
+        exp_peak = 16.0 * 148 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6      # 1965 MHz: the B200's maximum SM clock
         names = ["down_projection", "key_side", "query_side"]
         dom = max(range(3), key=lambda i: stage_ms[i])
         dt = stage_ms[dom] * 1e-3
         tf_t = stage_flops[dom] / (tf_peak * 1e12)
         hb_t = stage_bytes[dom] / (peaks["hbm_gbs"] * 1e9)
-        if hb_t >= tf_t:
+        ex_t = stage_exps[dom] / exp_peak
+        if ex_t >= max(hb_t, tf_t):
+            roofline = {"bound": "alu", "achieved": stage_exps[dom] / dt / 1e9, "peak": exp_peak / 1e9, "unit": "Gexp/s",
+                        "frac_tensor": stage_flops[dom] / dt / 1e12 / tf_peak,
+                        "frac_hbm": stage_bytes[dom] / dt / 1e9 / peaks["hbm_gbs"]}
+        elif hb_t >= tf_t:
             roofline = {"bound": "hbm", "achieved": stage_bytes[dom] / dt / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         else:
             roofline = {"bound": "tensor", "achieved": stage_flops[dom] / dt / 1e12, "peak": tf_peak, "unit": "TFLOP/s"}
@@ -340,7 +349,7 @@ def main():
             roofline[other_key] = roofline["achieved"] / tf_other
         roofline["traffic"] = recorded_traffic(names[dom], w)
         roofline["kernel"] = names[dom]
-        roofline["peak_source"] = "of " + peaks["source"] + (
+        roofline["peak_source"] = "nominal: 16 exp/clk/SM x 148 SMs x max SM clock" if roofline["bound"] == "alu" else "of " + peaks["source"] + (
             " (sustained GEMM figure: timed inside a long loop)" if sustained and roofline["bound"] == "tensor" else "")
         roofline["stage_ms"] = dict(zip(names, stage_ms))
 
