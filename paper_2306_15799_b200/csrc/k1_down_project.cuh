@@ -9,14 +9,6 @@
 // thread issues tcgen05.mma (M=128, N=ncols, K=16) into fp32 TMEM accumulators; when the range is
 // done four warps move the accumulators to shared memory and add them to the fp32 workspace with
 // TMA reduce-add, so partial sums from different CTAs meet in L2.
-//
-// Pairs.  The main loop is limited by how fast L2 fills shared memory (64 KB per chunk and CTA), and
-// half of that is the E slab, which the CTA of the neighbouring column group loads as well.  When the
-// number of column groups is even and the tile has two M-tiles, neighbouring column groups form a
-// cluster of two: each CTA loads only one 128-row half of the E slab by TMA and four otherwise idle
-// warps push that half into the partner's shared memory (st.shared::cluster), so every CTA takes
-// 48 KB per chunk from L2 instead of 64.  A stage is free again when the MMAs of BOTH CTAs have read
-// it (each CTA's tcgen05.commit arrives on the stage's barrier in both CTAs).
 #pragma once
 
 #include "tc_common.cuh"
@@ -28,7 +20,6 @@ struct K1Params {
   int nsplit;      // CTAs along the sequence
   int col_groups;  // ceil(BH * d / 256)
   int k_halves;    // ceil(k / 256)
-  int pair;        // 1: launched as clusters of two CTAs that share the E slabs (see above)
   int* status;
   unsigned long long* trace;   // optional [gridDim.x][4] nanosecond stamps: start, set up, accumulated, done
 };
@@ -37,32 +28,6 @@ constexpr int kK1Stages = 3;
 constexpr int kK1StageBytes = 65536;                  // 32 KB of E rows + 32 KB of K/V slabs
 constexpr int kK1SmemBytes = kK1Stages * kK1StageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 constexpr int kK1Threads = 192;
-
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t cluster_cta_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// address of the same shared-memory location in another CTA of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
-  uint32_t a;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(local_addr), "r"(rank));
-  return a;
-}
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// tcgen05.commit that arrives on the barrier at this offset in every CTA of `mask`
-__device__ __forceinline__ void mma_commit_multicast(uint32_t bar, uint16_t mask) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"(mask) : "memory");
-}
 
 __global__ void __launch_bounds__(kK1Threads, 1)
 k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmF,
@@ -75,8 +40,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const uint32_t bar_full = bar_base;                 // [3]
   const uint32_t bar_empty = bar_base + 24;           // [3]
   const uint32_t bar_accum = bar_base + 48;
-  const uint32_t bar_peer = bar_base + 56;            // [3]  the partner's half of the E slab has arrived
-  const uint32_t tmem_slot = bar_base + 80;
+  const uint32_t tmem_slot = bar_base + 64;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
 
@@ -99,15 +63,12 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const int c_end = (int)(((long long)(s + 1) * chunks_total) / p.nsplit);
   const int nchunks = c_end - c_begin;
   const uint32_t tmem_cols = mt == 2 ? 512u : 256u;
-  const bool pair = p.pair != 0;                            // host guarantees mt == 2 and an even number of column groups
-  const uint32_t rank = pair ? cluster_cta_rank() : 0u;     // = cg & 1: which half of the E slab this CTA loads
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int i = 0; i < kK1Stages; ++i) {
       mbar_init(bar_full + 8 * i, 1);
-      mbar_init(bar_empty + 8 * i, pair ? 2 : 1);           // pairs: the MMAs of both CTAs have read the stage
-      mbar_init(bar_peer + 8 * i, 4);                       // one arrival per pushing warp of the partner
+      mbar_init(bar_empty + 8 * i, 1);
     }
     mbar_init(bar_accum, 1);
     fence_mbar_init();
@@ -126,7 +87,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   }
   __syncthreads();
   const uint32_t tmem = tmem_base_shared;
-  if (pair) cluster_sync_all();                             // the partner's barriers exist before anybody arrives on them
   if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 1] = global_timer_ns();
 
   if (nchunks > 0) {
@@ -136,7 +96,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
       const CUtensorMap* tmX = t ? &tmV : &tmK;
       prefetch_tmap(tmP);
       prefetch_tmap(tmX);
-      const uint32_t tx_bytes = (uint32_t)((pair ? 1 : mt) * 16384 + nb * 8192);
+      const uint32_t tx_bytes = (uint32_t)(mt * 16384 + nb * 8192);
       const int dblocks = p.d >> 6;                         // 64-column slabs per head
       int issued = 0;
       bool ok = true;
@@ -148,11 +108,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
         const uint32_t b_dst = a_dst + 32768;
         const int n0 = (c_begin + it) << 6;
         mbar_arrive_expect_tx(bar_full + 8 * st, tx_bytes);
-        if (pair) {
-          tma_load_2d(a_dst + rank * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + (int)rank * 128);
-        } else {
-          for (int m = 0; m < mt; ++m) tma_load_2d(a_dst + m * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + m * 128);
-        }
+        for (int m = 0; m < mt; ++m) tma_load_2d(a_dst + m * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + m * 128);
         for (int b = 0; b < nb; ++b) {
           const int slab = cg * 4 + b;                       // global 64-column slab index
           const int head = slab / dblocks, dc = slab % dblocks;
@@ -172,10 +128,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
       for (int it = 0; it < nchunks; ++it) {
         const int st = it % kK1Stages;
         ok = mbar_wait(bar_full + 8 * st, (it / kK1Stages) & 1, p.status, &abort_flag);
-        if (ok && pair) {
-          ok = mbar_wait_cluster(bar_peer + 8 * st, (it / kK1Stages) & 1, p.status, &abort_flag);
-          asm volatile("fence.proxy.async;" ::: "memory");   // the partner's generic-proxy stores, now read by the MMAs
-        }
         if (!ok) break;
         tcgen05_fence_after();
         const uint32_t a_base = smem_base + st * kK1StageBytes;
@@ -188,39 +140,13 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
           const uint64_t ad = make_sdesc(a_base + m * 16384, 16, 1024, kSwizzle128);
           mma_ss_x4(tmem + m * 256, ad, bd, 2, 128, idesc, it > 0 ? 1u : 0u);
         }
-        if (pair) mma_commit_multicast(bar_empty + 8 * st, (uint16_t)3);
-        else mma_commit(bar_empty + 8 * st);
+        mma_commit(bar_empty + 8 * st);
       }
       if (ok) mma_commit(bar_accum);
     } else if (warp >= 2) {
       // ------------------------------------------------ epilogue: TMEM -> smem -> TMA reduce-add
       const int q = warp & 3;                                // TMEM lane quadrant of this warp
-      bool ok = true;
-      if (pair) {
-        // ---------------------------------------------- push this CTA's half of every E slab to the partner
-        const uint32_t peer = rank ^ 1u;
-        const int tid4 = (warp - 2) * 32 + lane;             // 0..127: 8 x 16 bytes each per chunk
-        for (int it = 0; it < nchunks && ok; ++it) {
-          const int st = it % kK1Stages;
-          // the partner's copy of this stage must have been read by its MMAs (and ours by ours)
-          if (it >= kK1Stages) ok = mbar_wait(bar_empty + 8 * st, ((it / kK1Stages) - 1) & 1, p.status, &abort_flag);
-          if (ok) ok = mbar_wait(bar_full + 8 * st, (it / kK1Stages) & 1, p.status, &abort_flag);
-          if (!ok) break;
-          const uint32_t src = smem_base + st * kK1StageBytes + rank * 16384;
-          const uint32_t dst = map_to_cta(src, peer);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint32_t off = (uint32_t)(j * 128 + tid4) * 16u;
-            uint32_t v0, v1, v2, v3;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(src + off));
-            st_cluster_v4(dst + off, v0, v1, v2, v3);
-          }
-          asm volatile("fence.proxy.async;" ::: "memory");   // the partner's MMAs read what we wrote
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_peer + 8 * st, peer));
-        }
-      }
-      if (ok) ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
+      bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
       if (warp == 2 && lane == 0) grid_launch_dependents();   // only the epilogue is left
       if (p.trace && warp == 2 && lane == 0) p.trace[4 * blockIdx.x + 2] = global_timer_ns();
       if (ok) {
@@ -263,8 +189,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   }
   tcgen05_fence_before();
   __syncthreads();
-  // nobody leaves while the partner may still write into this CTA's shared memory or arrive on its barriers
-  if (pair) cluster_sync_all();
   if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 3] = global_timer_ns();
   if (warp == 1) tmem_dealloc(tmem, tmem_cols);
 }

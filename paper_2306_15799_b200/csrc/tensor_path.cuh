@@ -140,22 +140,7 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
     attr_set = true;
   }
   const int grid = 2 * p.k_halves * p.col_groups * p.nsplit;
-  // neighbouring column groups pair up (cluster of two) when every tile has two M-tiles
-  p.pair = (p.col_groups % 2 == 0 && k % 256 == 0) ? 1 : 0;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)grid, 1, 1);
-  cfg.blockDim = dim3(kK1Threads, 1, 1);
-  cfg.dynamicSmemBytes = kK1SmemBytes;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = p.pair ? 2u : 1u;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, k1_down_project, tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
-  if (le != cudaSuccess) { *cuda_err = (int)le; (void)cudaGetLastError(); return -6; }
+  k1_down_project<<<grid, kK1Threads, kK1SmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
