@@ -160,7 +160,7 @@ TENSOR_CASES = [
     _wl("tc_perf_d64_k320_m256_n128", PERFORMER, "bf16", 1, 2, 128, 64, 320, 256, 109),
     _wl("tc_perf_d128_k448_m128", PERFORMER, "bf16", 2, 1, 256, 128, 448, 128, 110),
     _wl("tc_rnn_d128_k512_n128", RNN, "bf16", 1, 1, 128, 128, 512, 0, 111),
-    # two and four 256-column groups with 256-row tiles: stage 1 runs as pairs of CTAs sharing E slabs
+    # two and four 256-column groups with 256-row tiles in stage 1
     _wl("tc_perf_d64_k256_pairs", PERFORMER, "bf16", 2, 4, 1024, 64, 256, 128, 113),
     _wl("tc_rnn_d128_k512_pairs", RNN, "bf16", 2, 4, 512, 128, 512, 0, 114),
 ]
