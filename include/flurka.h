@@ -79,7 +79,7 @@ typedef enum {
  *
  * Shape limits: B, H, N >= 1, B*H <= 65535; 1 <= d <= 128; 1 <= k <= 4096; PERFORMER: m >= 1.
  * Pointers 16-byte aligned.  The tensor-core path additionally needs bf16, d in {64, 128},
- * N % 128 == 0, k % 64 == 0 with k <= 512, and (PERFORMER) m in {64, 128, 192, 256}; other shapes run
+ * N % 8 == 0, k % 64 == 0 with k <= 512, and (PERFORMER) m in {64, 128, 192, 256}; other shapes run
  * on the SIMT path.  The call enqueues work and returns; it never synchronises.  Scratch comes from the
  * workspace set by flurka_set_workspace(), or from one the library allocates (and re-uses) on first need.
  */

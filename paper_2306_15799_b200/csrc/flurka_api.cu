@@ -115,7 +115,7 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 bool tensor_path_ok(const Problem& pr) {
   if (pr.fp32) return false;
   if (pr.d != 64 && pr.d != 128) return false;
-  if (pr.N % 128) return false;
+  if (pr.N % 8) return false;       // row pitch of E, F (N elements) must be a multiple of 16 bytes for TMA
   if (pr.k % 64 || pr.k > 512) return false;
   if (pr.kernel == FLURKA_PERFORMER && (pr.m % 64 || pr.m > 256)) return false;
   return tensor_path_built();

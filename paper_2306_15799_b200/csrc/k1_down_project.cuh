@@ -58,7 +58,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const int total_cols = p.BH * p.d;
   const int ncols = min(256, total_cols - cg * 256);        // multiple of 64
   const int nb = ncols >> 6;                                // 64-column slabs
-  const int chunks_total = p.N >> 6;
+  const int chunks_total = (p.N + 63) >> 6;                 // a ragged last chunk is zero-filled by TMA
   const int c_begin = (int)(((long long)s * chunks_total) / p.nsplit);
   const int c_end = (int)(((long long)(s + 1) * chunks_total) / p.nsplit);
   const int nchunks = c_end - c_begin;

@@ -28,7 +28,7 @@ namespace flurka {
 
 struct K3Params {
   int N, d, p, BH;          // p = feature dimension (m, or d for RNN)
-  int tiles_per_head;       // N / 128
+  int tiles_per_head;       // ceil(N / 128): TMA zero-fills the rows of a ragged last tile, their outputs are not stored
   int total_tiles;
   const float* weight;      // [BH][p]  b_i or z_i
   __nv_bfloat16* out;       // [BH][N][d]
@@ -350,6 +350,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         tcgen05_fence_after();
         K3_STAMP(3)
         __nv_bfloat16* orow = prm.out + ((size_t)head * prm.N + row0 + row) * d;
+        const bool in_range = row0 + row < prm.N;        // rows past the end of the sequence exist only in the tile
         for (int c = 0; c < d; c += 64) {
           uint32_t ra[32], rb[32];
           tmem_ld32(tb + c, ra);
@@ -371,6 +372,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                                                               __uint_as_float(src[(g8 & 1) * 16 + 2 * e + 1]) * inv);
               v[e] = *reinterpret_cast<const uint32_t*>(&o2);
             }
+            if (in_range)
             asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(orow + c + g8 * 16),
                          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
                          : "memory");

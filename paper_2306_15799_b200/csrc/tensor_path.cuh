@@ -130,7 +130,7 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
   p.N = N; p.d = d; p.k = k; p.BH = BH;
   p.col_groups = (BH * d + 255) / 256;
   p.k_halves = (k + 255) / 256;
-  p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, N / 64);
+  p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, (N + 63) / 64);
   p.status = status;
   p.trace = nullptr;
   static bool attr_set = false;
@@ -252,7 +252,7 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
   }
   K3Params prm;
   prm.N = N; prm.d = d; prm.p = p; prm.BH = BH;
-  prm.tiles_per_head = N / 128;
+  prm.tiles_per_head = (N + 127) / 128;
   prm.total_tiles = prm.tiles_per_head * BH;
   prm.weight = weight;
   prm.out = reinterpret_cast<__nv_bfloat16*>(out);

@@ -160,6 +160,10 @@ TENSOR_CASES = [
     _wl("tc_perf_d64_k320_m256_n128", PERFORMER, "bf16", 1, 2, 128, 64, 320, 256, 109),
     _wl("tc_perf_d128_k448_m128", PERFORMER, "bf16", 2, 1, 256, 128, 448, 128, 110),
     _wl("tc_rnn_d128_k512_n128", RNN, "bf16", 1, 1, 128, 128, 512, 0, 111),
+    # sequence lengths that are not multiples of the 64-wide chunks of stage 1 or the 128-row tiles of stage 3
+    _wl("tc_perf_d64_n1000", PERFORMER, "bf16", 1, 3, 1000, 64, 128, 256, 115),
+    _wl("tc_rnn_d128_n200", RNN, "bf16", 2, 1, 200, 128, 64, 0, 116),
+    _wl("tc_perf_d128_n72", PERFORMER, "bf16", 1, 2, 72, 128, 64, 64, 117),
     # two and four 256-column groups with 256-row tiles in stage 1
     _wl("tc_perf_d64_k256_pairs", PERFORMER, "bf16", 2, 4, 1024, 64, 256, 128, 113),
     _wl("tc_rnn_d128_k512_pairs", RNN, "bf16", 2, 4, 512, 128, 512, 0, 114),
@@ -233,7 +237,7 @@ def test_auto_picks_tensor_path_when_the_shape_allows():
     w = TENSOR_CASES[0]
     pu.check_all_heads(w)
     assert binding.flurka_last_path() == binding.PATH_TENSOR
-    odd = _wl("auto_simt", PERFORMER, "bf16", 1, 1, 200, 64, 64, 64, 108)      # N % 128 != 0
+    odd = _wl("auto_simt", PERFORMER, "bf16", 1, 1, 204, 64, 64, 64, 108)      # N % 8 != 0
     pu.check_all_heads(odd)
     assert binding.flurka_last_path() == binding.PATH_SIMT
 
