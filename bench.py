@@ -191,6 +191,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--heads", default="", help="B,H override: a smaller batch of the same workload (profiling)")
     ap.add_argument("--no-load", action="store_true", help="skip the sustained-load phase before timing (profiling)")
+    ap.add_argument("--layout", default="bhnd", choices=["bhnd", "bnhd"],
+                    help="Q, K, V, out as [B,H,N,d] (default) or [B,N,H,d]")
     args = ap.parse_args()
     w = configs.get(args.config)
     if args.heads:
@@ -220,7 +222,11 @@ def main():
     # every rank draws its own batch (weak scaling over B*H); same recipe, rank-offset seed
     wr = rank_workload(w, rank)
     host = synth.make_inputs(wr)
-    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in host.items()}
+    laid_out = dict(host)
+    if args.layout == "bnhd":
+        for n in ("Q", "K", "V"):
+            laid_out[n] = host[n].transpose(1, 2).contiguous()
+    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in laid_out.items()}
     dev = {n: (t.cuda(non_blocking=True) if t is not None else None) for n, t in pinned.items()}
     out = torch.empty_like(dev["Q"])
     host_out = torch.empty_like(pinned["Q"]).pin_memory()
@@ -233,7 +239,7 @@ def main():
 
     def step():
         binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant,
-                               out=out, stream=stream)
+                               out=out, stream=stream, layout=args.layout)
 
     def barrier():
         if world > 1:
@@ -289,12 +295,12 @@ def main():
     # ---- end to end: host buffers in, host buffer out, through the host entry point
     e2e_steps = max(1, min(args.steps, 5))
     binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
-                                w.variant, out=host_out, stream=stream)
+                                w.variant, out=host_out, stream=stream, layout=args.layout)
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
-                                    w.variant, out=host_out, stream=stream)
+                                    w.variant, out=host_out, stream=stream, layout=args.layout)
     torch.cuda.synchronize()
     e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
     status = binding.flurka_last_status()
@@ -360,6 +366,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": w.name, "variant": "performer" if w.variant == configs.PERFORMER else "rnn",
                        "B": w.B, "H": w.H, "N": w.N, "d": w.d, "k": w.k, "m": w.m, "io": w.io, "path": path_taken,
+                       "layout": args.layout,
                        "parallelism": "replicated batches over B*H, no collective" if world > 1 else "single GPU",
                        "l2": "inputs (%.0f MB) exceed L2" % (in_bytes / 1e6) if flush is None
                              else "L2 flushed between steps (252 MiB write)"},

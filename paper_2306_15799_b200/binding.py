@@ -92,15 +92,21 @@ def version() -> int:
     return load().flurka_version()
 
 
-def _variant_word(variant: int, dtype: torch.dtype) -> int:
+LAYOUT_BNHD = 0x200   # or-ed into the variant word: Q, K, V, out are [B,N,H,d]
+
+
+def _variant_word(variant: int, dtype: torch.dtype, layout: str = "bhnd") -> int:
+    if layout not in ("bhnd", "bnhd"):
+        raise ValueError("flurka: layout must be 'bhnd' or 'bnhd'")
+    word = variant | (LAYOUT_BNHD if layout == "bnhd" else 0)
     if dtype == torch.bfloat16:
-        return variant | IO_BF16
+        return word | IO_BF16
     if dtype == torch.float32:
-        return variant | IO_FP32
+        return word | IO_FP32
     raise TypeError("flurka: tensors must be bfloat16 or float32, got %s" % dtype)
 
 
-def _check(Q, K, V, E, F, W, variant, out, device_type):
+def _check(Q, K, V, E, F, W, variant, out, device_type, layout="bhnd"):
     for name, t in (("Q", Q), ("K", K), ("V", V), ("E", E), ("F", F), ("out", out)):
         if t.device.type != device_type:
             raise ValueError("flurka: %s must live on %s" % (name, device_type))
@@ -109,8 +115,11 @@ def _check(Q, K, V, E, F, W, variant, out, device_type):
         if t.dtype != Q.dtype:
             raise TypeError("flurka: %s has dtype %s, Q has %s" % (name, t.dtype, Q.dtype))
     if Q.dim() != 4 or K.shape != Q.shape or V.shape != Q.shape or out.shape != Q.shape:
-        raise ValueError("flurka: Q, K, V, out must all be [B,H,N,d]")
-    B, H, N, d = Q.shape
+        raise ValueError("flurka: Q, K, V, out must all be [B,H,N,d] (or [B,N,H,d] with layout='bnhd')")
+    if layout == "bnhd":
+        B, N, H, d = Q.shape
+    else:
+        B, H, N, d = Q.shape
     if E.dim() != 2 or E.shape[1] != N or F.shape != E.shape:
         raise ValueError("flurka: E, F must be [k,N]")
     k = E.shape[0]
@@ -129,28 +138,29 @@ def _stream_ptr(stream):
     return ctypes.c_void_p(stream.cuda_stream)
 
 
-def flurka_forward(Q, K, V, E, F, W, variant, out=None, stream=None):
-    """O = phi(Q)(phi(EK)^T FV) / phi(Q)(phi(EK)^T 1) on device tensors; asynchronous on `stream`."""
+def flurka_forward(Q, K, V, E, F, W, variant, out=None, stream=None, layout="bhnd"):
+    """O = phi(Q)(phi(EK)^T FV) / phi(Q)(phi(EK)^T 1) on device tensors; asynchronous on `stream`.
+    layout: 'bhnd' for [B,H,N,d] tensors, 'bnhd' for [B,N,H,d]."""
     if out is None:
         out = torch.empty_like(Q)
-    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cuda")
+    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cuda", layout)
     rc = load().flurka_forward(
         Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
-        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, layout),
         B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
     if rc:
         raise FlurkaError(rc, "flurka_forward")
     return out
 
 
-def flurka_forward_host(Q, K, V, E, F, W, variant, out=None, stream=None):
+def flurka_forward_host(Q, K, V, E, F, W, variant, out=None, stream=None, layout="bhnd"):
     """The same on host (ideally pinned) tensors: copies in, computes, copies out, synchronises."""
     if out is None:
         out = torch.empty_like(Q, pin_memory=True)
-    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cpu")
+    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cpu", layout)
     rc = load().flurka_forward_host(
         Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
-        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, layout),
         B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
     if rc:
         raise FlurkaError(rc, "flurka_forward_host")

@@ -17,7 +17,9 @@ using namespace flurka;
 struct Problem {
   int kernel;      // FLURKA_PERFORMER / FLURKA_RNN
   bool fp32;       // element type of the I/O tensors
+  bool bnhd;       // Q, K, V, out are [B,N,H,d] (heads merged into the row) instead of [B,H,N,d]
   int B, H, N, d, k, m;
+  int seq_major_heads() const { return bnhd ? H : 0; }   // what head_view() takes
   int BH() const { return B * H; }
   int p() const { return kernel == FLURKA_PERFORMER ? m : d; }   // feature dimension
   size_t esize() const { return fp32 ? 4 : 2; }
@@ -93,15 +95,17 @@ int cuda_fail(cudaError_t e) {
 
 int parse_problem(int variant, int B, int H, int N, int d, int k, int m, Problem* pr) {
   const int kernel = variant & 0xff;
-  const int io = variant & ~0xff;
+  const int io = variant & 0x100;
+  const int layout = variant & 0x200;
   if (kernel != FLURKA_PERFORMER && kernel != FLURKA_RNN) return FLURKA_ERR_VARIANT;
-  if (io != FLURKA_IO_BF16 && io != FLURKA_IO_FP32) return FLURKA_ERR_VARIANT;
+  if (variant & ~0x3ff) return FLURKA_ERR_VARIANT;
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || k <= 0) return FLURKA_ERR_SHAPE;
   if (d > 128 || k > 4096) return FLURKA_ERR_SHAPE;
   if (kernel == FLURKA_PERFORMER && m <= 0) return FLURKA_ERR_SHAPE;
   if ((long long)B * H > 65535) return FLURKA_ERR_SHAPE;
   pr->kernel = kernel;
   pr->fp32 = io == FLURKA_IO_FP32;
+  pr->bnhd = layout == FLURKA_LAYOUT_BNHD;
   pr->B = B; pr->H = H; pr->N = N; pr->d = d; pr->k = k;
   pr->m = kernel == FLURKA_PERFORMER ? m : 0;
   return FLURKA_OK;
@@ -169,7 +173,7 @@ int launch_simt_down_project(const Problem& pr, const void* K, const void* V, co
   nsplit = (pr.N + chunk - 1) / chunk;
   dim3 grid(jt, pr.BH(), 2 * nsplit);
   simt_down_project<T><<<grid, 256, 0, st>>>((const T*)K, (const T*)V, (const T*)E, (const T*)F, kpvp,
-                                            pr.BH(), pr.N, pr.d, pr.k, nsplit, chunk);
+                                            pr.BH(), pr.N, pr.d, pr.k, nsplit, chunk, pr.seq_major_heads());
   ++*launches;
   return FLURKA_OK;
 }
@@ -200,7 +204,7 @@ int launch_simt_query_side(const Problem& pr, const void* Q, const void* W, cons
     if (e != cudaSuccess) return cuda_fail(e);
   }
   simt_query_side<T, P><<<grid, 256, smem, st>>>((const T*)Q, (const T*)W, weight, a32, (T*)out, pr.N,
-                                                 pr.d, pr.p());
+                                                 pr.d, pr.p(), pr.seq_major_heads());
   ++*launches;
   return FLURKA_OK;
 }
@@ -234,7 +238,7 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   g.timer.mark(0, st);
   int rc;
   if (tc1) {
-    rc = launch_k1(g.maps, K, V, E, F, kpvp, pr.BH(), pr.N, pr.d, pr.k, status, st, &cuda_err);
+    rc = launch_k1(g.maps, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err);
     if (rc) { g.last_cuda_error = cuda_err; return rc; }
     ++*launches;
   } else {
@@ -254,7 +258,8 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   }
   g.timer.mark(2, st);
   if (tc3) {
-    rc = launch_k3(g.maps, performer, Q, W, aT16, weight, out, pr.BH(), pr.N, pr.d, pr.p(), status, st, &cuda_err);
+    rc = launch_k3(g.maps, performer, Q, W, aT16, weight, out, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.p(),
+                   status, st, &cuda_err);
     if (rc) { g.last_cuda_error = cuda_err; return rc; }
     ++*launches;
   } else {
@@ -377,7 +382,8 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
   // The heads are independent, so the call works through them in up to eight groups: while the
   // inputs of one group travel to the device, the output of the group before travels back on a second
   // stream (the link is full duplex), and the compute of a group hides under the copies.
-  const int heads = pr.BH();
+  // (units that are contiguous in memory: heads for [B,H,N,d], batches for [B,N,H,d])
+  const int heads = pr.bnhd ? pr.B : pr.BH();
   int groups = (int)std::min<size_t>(8, qn >> 20);           // at least 1 MiB of Q per group
   groups = std::max(1, std::min(groups, heads));
   if (groups > 1 && !g.out_stream) {
@@ -386,7 +392,7 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
       if ((e = cudaEventCreateWithFlags(&g.group_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaEventCreateWithFlags(&g.out_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
   }
-  const size_t head_bytes = (size_t)N * d * pr.esize();
+  const size_t head_bytes = (size_t)N * d * pr.esize() * (pr.bnhd ? H : 1);
   rc = FLURKA_OK;
   for (int gi = 0; gi < groups && rc == FLURKA_OK; ++gi) {
     const int h0 = (int)((long long)heads * gi / groups), h1 = (int)((long long)heads * (gi + 1) / groups);
@@ -398,8 +404,8 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
       break;
     }
     g.keep_status = gi > 0;
-    rc = flurka_forward(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, 1, h1 - h0, N, d, k, m,
-                        dO + off, stream);
+    rc = flurka_forward(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, pr.bnhd ? h1 - h0 : 1,
+                        pr.bnhd ? H : h1 - h0, N, d, k, m, dO + off, stream);
     g.keep_status = false;
     if (rc) break;
     if (groups == 1) {

@@ -17,6 +17,7 @@ namespace flurka {
 
 struct K1Params {
   int N, d, k, BH;
+  int H;           // > 0: K, V are [B,N,H,d] (the tensor map has rows of H*d elements); 0: [B,H,N,d]
   int nsplit;      // CTAs along the sequence
   int col_groups;  // ceil(BH * d / 256)
   int k_halves;    // ceil(k / 256)
@@ -112,7 +113,8 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
         for (int b = 0; b < nb; ++b) {
           const int slab = cg * 4 + b;                       // global 64-column slab index
           const int head = slab / dblocks, dc = slab % dblocks;
-          tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, dc * 64, n0, head);
+          if (p.H > 0) tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, (head % p.H) * p.d + dc * 64, n0, head / p.H);
+          else tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, dc * 64, n0, head);
         }
         ++issued;
       }

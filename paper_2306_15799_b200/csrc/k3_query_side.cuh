@@ -28,6 +28,7 @@ namespace flurka {
 
 struct K3Params {
   int N, d, p, BH;          // p = feature dimension (m, or d for RNN)
+  int H;                    // > 0: Q and out are [B,N,H,d] (the Q tensor map has rows of H*d elements); 0: [B,H,N,d]
   int tiles_per_head;       // ceil(N / 128): TMA zero-fills the rows of a ragged last tile, their outputs are not stored
   int total_tiles;
   const float* weight;      // [BH][p]  b_i or z_i
@@ -184,7 +185,11 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (!ok) break;
         mbar_arrive_expect_tx(bar_qfull + 8 * st, q_stage_bytes);
         for (int kb = 0; kb < kq; ++kb)
-          tma_load_3d(base + L.q + st * q_stage_bytes + kb * 16384, &tmQ, bar_qfull + 8 * st, kb * 64, row0, head);
+          if (prm.H > 0)
+            tma_load_3d(base + L.q + st * q_stage_bytes + kb * 16384, &tmQ, bar_qfull + 8 * st,
+                        (head % prm.H) * d + kb * 64, row0, head / prm.H);
+          else
+            tma_load_3d(base + L.q + st * q_stage_bytes + kb * 16384, &tmQ, bar_qfull + 8 * st, kb * 64, row0, head);
         ++issued;
       }
       if (!ok) {
@@ -349,7 +354,9 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (!mbar_wait(bar_ofull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag)) return false;
         tcgen05_fence_after();
         K3_STAMP(3)
-        __nv_bfloat16* orow = prm.out + ((size_t)head * prm.N + row0 + row) * d;
+        __nv_bfloat16* orow = prm.H > 0
+            ? prm.out + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * d
+            : prm.out + ((size_t)head * prm.N + row0 + row) * d;
         const bool in_range = row0 + row < prm.N;        // rows past the end of the sequence exist only in the tile
         for (int c = 0; c < d; c += 64) {
           uint32_t ra[32], rb[32];

@@ -21,6 +21,23 @@
 
 namespace flurka {
 
+// Where head bh of a [B,H,N,d] tensor (H == 0) or of a [B,N,H,d] tensor (H = number of heads) starts,
+// and the distance between consecutive sequence positions of that head, in elements.
+struct HeadView {
+  size_t base, row_stride;
+};
+__host__ __device__ __forceinline__ HeadView head_view(int bh, int H, int N, int d) {
+  HeadView v;
+  if (H > 0) {
+    v.base = ((size_t)(bh / H) * N * H + (size_t)(bh % H)) * d;
+    v.row_stride = (size_t)H * d;
+  } else {
+    v.base = (size_t)bh * N * d;
+    v.row_stride = (size_t)d;
+  }
+  return v;
+}
+
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 __device__ __forceinline__ void store_out(float* p, float v) { *p = v; }
@@ -36,7 +53,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 simt_down_project(const T* __restrict__ Kin, const T* __restrict__ Vin, const T* __restrict__ E,
                   const T* __restrict__ F, float* __restrict__ KpVp, int BH, int N, int d, int k,
-                  int nsplit, int chunk) {
+                  int nsplit, int chunk, int seq_major_heads) {
   constexpr int TJ = 32, TN = 32;
   __shared__ float Ps[TJ][TN + 1];
   __shared__ float Xs[TN][128];
@@ -46,7 +63,8 @@ simt_down_project(const T* __restrict__ Kin, const T* __restrict__ Vin, const T*
   const int bh = blockIdx.y;
   const int j0 = blockIdx.x * TJ;
   const T* __restrict__ P = t ? F : E;
-  const T* __restrict__ X = (t ? Vin : Kin) + (size_t)bh * N * d;
+  const HeadView hv = head_view(bh, seq_major_heads, N, d);
+  const T* __restrict__ X = (t ? Vin : Kin) + hv.base;
   float* __restrict__ out = KpVp + ((size_t)t * BH + bh) * (size_t)k * d;
 
   const int n_begin = s * chunk;
@@ -69,7 +87,7 @@ simt_down_project(const T* __restrict__ Kin, const T* __restrict__ Vin, const T*
     for (int idx = threadIdx.x; idx < TN * 128; idx += 256) {
       const int nn = idx >> 7, c = idx & 127;
       const int n = n0 + nn;
-      Xs[nn][c] = (n < n_end && c < d) ? to_f32(X[(size_t)n * d + c]) : 0.f;
+      Xs[nn][c] = (n < n_end && c < d) ? to_f32(X[(size_t)n * hv.row_stride + c]) : 0.f;
     }
     __syncthreads();
 #pragma unroll 4
@@ -194,7 +212,7 @@ simt_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, float* __
 template <typename T, bool kPerformer>
 __global__ void __launch_bounds__(256)
 simt_query_side(const T* __restrict__ Q, const T* __restrict__ W, const float* __restrict__ weight,
-                const float* __restrict__ a32, T* __restrict__ out, int N, int d, int p) {
+                const float* __restrict__ a32, T* __restrict__ out, int N, int d, int p, int seq_major_heads) {
   extern __shared__ float smem[];
   float* Ws = smem;                  // [32][d+1]
   float* As = smem + 32 * (d + 1);   // [32][d]
@@ -204,13 +222,14 @@ simt_query_side(const T* __restrict__ Q, const T* __restrict__ W, const float* _
   const int bh = blockIdx.y;
   const int n0 = blockIdx.x * 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const T* __restrict__ Qh = Q + (size_t)bh * N * d;
+  const HeadView hv = head_view(bh, seq_major_heads, N, d);
+  const T* __restrict__ Qh = Q + hv.base;
   const float* __restrict__ ah = a32 + (size_t)bh * p * d;
   const float* __restrict__ wh = weight + (size_t)bh * p;
 
   for (int idx = threadIdx.x; idx < 32 * d; idx += 256) {
     const int r = idx / d, c = idx % d;
-    qs[r][c] = (n0 + r < N) ? to_f32(Qh[(size_t)(n0 + r) * d + c]) : 0.f;
+    qs[r][c] = (n0 + r < N) ? to_f32(Qh[(size_t)(n0 + r) * hv.row_stride + c]) : 0.f;
   }
   float run_max[4], run_sum[4], acc[4][4];
 #pragma unroll
@@ -280,7 +299,7 @@ simt_query_side(const T* __restrict__ Q, const T* __restrict__ W, const float* _
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
       const int c = lane + 32 * b;
-      if (c < d) store_out(out + ((size_t)bh * N + n) * d + c, acc[r][b] * inv);
+      if (c < d) store_out(out + hv.base + (size_t)n * hv.row_stride + c, acc[r][b] * inv);
     }
   }
 }

@@ -110,11 +110,14 @@ inline int k1_choose_nsplit(int units, int chunks) {
 }
 
 // ---- stage 1: K' = E K, V' = F V into kpvp (already zeroed) ----------------------------------
+// H > 0: K, V are [B,N,H,d] (H heads merged into the row); H == 0: [B,H,N,d]
 inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E, const void* F, float* kpvp,
-                     int BH, int N, int d, int k, int* status, cudaStream_t st, int* cuda_err) {
+                     int BH, int H, int N, int d, int k, int* status, cudaStream_t st, int* cuda_err) {
   const unsigned long long dE[2] = {(unsigned long long)N, (unsigned long long)k};
   const unsigned bE[2] = {64, 128};
-  const unsigned long long dX[3] = {(unsigned long long)d, (unsigned long long)N, (unsigned long long)BH};
+  // [B,N,H,d] is a 3-D tensor too: rows of H*d elements, head h at columns h*d .. h*d+d-1
+  const unsigned long long dX[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
+                                    (unsigned long long)(H > 0 ? BH / H : BH)};
   const unsigned bX[3] = {64, 64, 1};
   const unsigned long long dO[3] = {(unsigned long long)d, (unsigned long long)k, (unsigned long long)2 * BH};
   const unsigned bO[3] = {32, 32, 1};
@@ -127,7 +130,7 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
     return -6;
   }
   K1Params p;
-  p.N = N; p.d = d; p.k = k; p.BH = BH;
+  p.N = N; p.d = d; p.k = k; p.BH = BH; p.H = H;
   p.col_groups = (BH * d + 255) / 256;
   p.k_halves = (k + 255) / 256;
   p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, (N + 63) / 64);
@@ -231,9 +234,10 @@ inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const vo
 
 // ---- stage 3: O from Q, W and the key-side summaries ------------------------------------------
 inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* W, const __half* aT16,
-                     const float* weight, void* out, int BH, int N, int d, int p, int* status, cudaStream_t st,
+                     const float* weight, void* out, int BH, int H, int N, int d, int p, int* status, cudaStream_t st,
                      int* cuda_err) {
-  const unsigned long long dQ[3] = {(unsigned long long)d, (unsigned long long)N, (unsigned long long)BH};
+  const unsigned long long dQ[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
+                                    (unsigned long long)(H > 0 ? BH / H : BH)};
   const unsigned bQ[3] = {64, 128, 1};
   const unsigned long long dA[3] = {(unsigned long long)p, (unsigned long long)d, (unsigned long long)BH};
   const unsigned bA[3] = {64, (unsigned)d, 1};
@@ -251,7 +255,7 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
     }
   }
   K3Params prm;
-  prm.N = N; prm.d = d; prm.p = p; prm.BH = BH;
+  prm.N = N; prm.d = d; prm.p = p; prm.BH = BH; prm.H = H;
   prm.tiles_per_head = (N + 127) / 128;
   prm.total_tiles = prm.tiles_per_head * BH;
   prm.weight = weight;

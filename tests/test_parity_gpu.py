@@ -255,3 +255,49 @@ def test_tensor_path_with_large_and_small_logits(scale):
     assert np.isfinite(out).all()
     for h in range(w.H):
         pu.assert_close(out[0, h], pu.oracle_head(inputs, w, 0, h), "bf16", "scaled x%g head %d" % (scale, h))
+
+
+# ------------------------------------------------------------------------------- [B,N,H,d] tensors
+BNHD_CASES = [
+    (_wl("bnhd_tc_perf", PERFORMER, "bf16", 2, 3, 640, 64, 128, 256, 121), binding.PATH_TENSOR),
+    (_wl("bnhd_tc_rnn_d128", RNN, "bf16", 1, 4, 384, 128, 256, 0, 122), binding.PATH_TENSOR),
+    (_wl("bnhd_tc_perf_8groups", PERFORMER, "bf16", 2, 8, 512, 64, 256, 64, 123), binding.PATH_TENSOR),
+    (_wl("bnhd_simt_perf_fp32", PERFORMER, "fp32", 2, 3, 200, 24, 20, 40, 124), binding.PATH_SIMT),
+    (_wl("bnhd_simt_rnn_bf16", RNN, "bf16", 1, 2, 300, 64, 48, 0, 125), binding.PATH_SIMT),
+]
+
+
+@pytest.mark.parametrize("w,path", BNHD_CASES, ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_heads_merged_into_the_row(w, path):
+    """Q, K, V, out as [B,N,H,d]: the same inputs, transposed, must give the transposed output of the
+    oracle (which works head by head)."""
+    inputs = synth.make_inputs(w)
+    dev = pu.to_device(inputs)
+    t = {n: dev[n].transpose(1, 2).contiguous() for n in ("Q", "K", "V")}
+    prev = binding.flurka_set_path(path)
+    try:
+        out = binding.flurka_forward(t["Q"], t["K"], t["V"], dev["E"], dev["F"], dev["W"], w.variant, layout="bnhd")
+        torch.cuda.synchronize()
+        assert binding.flurka_last_status() == 0
+        assert binding.flurka_last_path() == path
+    finally:
+        binding.flurka_set_path(prev)
+    assert out.shape == (w.B, w.N, w.H, w.d)
+    got = out.transpose(1, 2).cpu().double().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            pu.assert_close(got[b, h], pu.oracle_head(inputs, w, b, h), w.io, "%s head (%d,%d)" % (w.name, b, h))
+
+
+def test_heads_merged_into_the_row_host_entry():
+    w = _wl("bnhd_host", PERFORMER, "bf16", 4, 2, 4096, 64, 64, 64, 126)      # 4 MiB of Q: four groups of one batch
+    inputs = synth.make_inputs(w)
+    pinned = {n: (inputs[n].transpose(1, 2).contiguous().pin_memory() if n in ("Q", "K", "V") else
+                  (inputs[n].pin_memory() if inputs[n] is not None else None)) for n in inputs}
+    out = binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
+                                      w.variant, layout="bnhd")
+    assert binding.flurka_last_status() == 0
+    got = out.transpose(1, 2).double().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            pu.assert_close(got[b, h], pu.oracle_head(inputs, w, b, h), "bf16", "host, head (%d,%d)" % (b, h))
