@@ -10,7 +10,7 @@
 //
 // The per-feature summaries a_i, b_i (or z_i) come from stage 2.  A persistent CTA walks a
 // contiguous range of 128-row tiles; warp 0 feeds Q tiles by TMA, warps 1 and 3 issue the first and the second
-// products, warp 2 rebuilds the bias operand when the head changes, and two groups of four warps
+// products, warp 2 reloads a^T and rebuilds the bias operand when the head changes, and two groups of four warps
 // alternate tiles.  TMEM holds S/p and O of the tiles in flight: two 256-column buffers (S/p in
 // columns 0.., O in columns 128..) in general; four 128-column buffers (S/p in columns 0.., O in
 // columns 64.., which S has vacated by then) when d = 64 and p <= 128.  With four buffers each group
