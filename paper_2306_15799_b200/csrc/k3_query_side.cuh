@@ -335,7 +335,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const int row = q4 * 32 + lane;                  // row of the tile this thread owns
       const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
       const float kLog2e = 1.4426950408889634f;
-      int head_prev = -1, events = 0;
+      int events = 0;
       bool ok = true;
       // optional cycle accounting of one thread per group: 0 wait for S (or Q), 1 pass 1,
       // 2 pass 2 + hand-over, 3 wait for O, 4 normalise + store
@@ -345,10 +345,8 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 #define K3_STAMP(slot) \
   if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
       // read-out of tile j: O / sum -> bf16 -> this thread's output row, 32 bytes per store
-      auto read_out = [&](int j, float inv) -> bool {
-        const int tile = t_begin + j;
-        const int head = tile / prm.tiles_per_head;
-        const int row0 = (tile % prm.tiles_per_head) * 128;
+      // (head and first row of the tile are tracked by the caller: no divisions on this path)
+      auto read_out = [&](int j, float inv, int head, int row0) -> bool {
         const int buf = j & (NB - 1);
         const uint32_t tb = tmem + buf * buf_cols + lane_off + o_col;
         if (!mbar_wait(bar_ofull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag)) return false;
@@ -389,15 +387,18 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         return true;
       };
       float inv_prev = 0.f;                            // four buffers: 1 / sum of the group's previous tile
+      // head and tile-within-head of this group's current tile, advanced by two tiles per iteration;
+      // the previous tile's pair is kept for the late read-out
+      const int head_first = t_begin / prm.tiles_per_head;
+      int head_i = (t_begin + grp) / prm.tiles_per_head, tih = (t_begin + grp) % prm.tiles_per_head;
+      int head_o = head_i, row0_o = 0;
+      const int ns_mask = NS - 1, ns_shift = NS == 4 ? 2 : 1;   // NS is 2 or 4
       for (int i = grp; i < ntiles && ok; i += 2) {
-        const int buf = i & (NB - 1), st = i % NS;
+        const int buf = i & (NB - 1), st = i & ns_mask;
         const uint32_t tb = tmem + buf * buf_cols + lane_off;
         float denom = 0.f, denom1 = 0.f;
-        // count head changes the same way the other roles do (both groups see every tile index)
-        for (int j = (i >= 2 ? i - 1 : 0); j <= i; ++j) {
-          const int hj = (t_begin + j) / prm.tiles_per_head;
-          if (hj != head_prev) { head_prev = hj; ++events; }
-        }
+        const int head = head_i, row0 = tih * 128;
+        events = head - head_first + 1;                // heads met so far, the way the other roles count them
         if (kPerformer) {
           ok = mbar_wait(bar_sfull + 8 * buf, (i >> nb_shift) & 1, prm.status, &abort_flag);
           if (!ok) break;
@@ -469,7 +470,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           // (no wait for the buffer: this thread has itself read out the tile that used it before, and
           // the second product starts only when all 128 owners have said so)
           ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
-          if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
+          if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i >> ns_shift) & 1, prm.status, &abort_flag);
           if (!ok) break;
           K3_STAMP(0)
           const uint32_t qb = base + L.q + st * q_stage_bytes;
@@ -513,13 +514,17 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (NB == 4) {
           // two tiles of this group are in flight: read out the previous one, whose second product
           // has had this tile's passes to finish
-          if (i >= 2) ok = read_out(i - 2, inv_prev);
+          if (i >= 2) ok = read_out(i - 2, inv_prev, head_o, row0_o);
           inv_prev = inv;
+          head_o = head;
+          row0_o = row0;
         } else {
-          ok = read_out(i, inv);
+          ok = read_out(i, inv, head, row0);
         }
+        tih += 2;
+        while (tih >= prm.tiles_per_head) { tih -= prm.tiles_per_head; ++head_i; }
       }
-      if (NB == 4 && ok && ntiles > grp) (void)read_out(grp + 2 * ((ntiles - 1 - grp) / 2), inv_prev);
+      if (NB == 4 && ok && ntiles > grp) (void)read_out(grp + 2 * ((ntiles - 1 - grp) / 2), inv_prev, head_o, row0_o);
 #undef K3_STAMP
       if (tracing) {
         for (int sidx = 0; sidx < 6; ++sidx) prm.trace[((size_t)blockIdx.x * 3 + grp) * 8 + sidx] = tacc[sidx];
