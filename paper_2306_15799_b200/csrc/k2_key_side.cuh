@@ -78,6 +78,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   const uint32_t bar_w = sm_stage + 65536;
   const uint32_t bar_mma = bar_w + 8;
   const uint32_t bar_stage = bar_w + 16;
+  const uint32_t bar_kp = bar_w + 24;             // RNN: a piece of K' has arrived
   const uint32_t tmem_slot = bar_w + 32;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
@@ -107,6 +108,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     mbar_init(bar_w, 1);
     mbar_init(bar_mma, 1);
     mbar_init(bar_stage, 1);
+    mbar_init(bar_kp, 1);
     fence_mbar_init();
   }
   if (warp == 4) {
@@ -298,39 +300,53 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     }
   } else {
     if (tid == 0) stage_chunk(Vp, jc_begin);
-    // RNN: f_ij = elu(k'_ji) + 1.  All threads stage 64 rows of K' in shared memory (coalesced), then
-    // the thread that owns feature i walks down column i (row stride d + 1 words: no bank conflicts).
-    float* stage = reinterpret_cast<float*>(base_ptr + (sm_op - base));
+    // RNN: f_ij = elu(k'_ji) + 1.  K' arrives by bulk copy, in pieces of up to 96 KB, in the operand
+    // area (unused until the conversion of V'); the thread that owns feature i walks down column i
+    // (consecutive lanes read consecutive words).  Two threads share a feature: warps w and w + 4 see
+    // the same TMEM lanes and take alternate groups of 32 keys.
+    const float* stage = reinterpret_cast<const float*>(base_ptr + (sm_op - base));
     const uint32_t tb = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    for (int jc = 0; jc < (k >> 6); ++jc) {
-      __syncthreads();
-      for (int idx = tid * 4; idx < 64 * d; idx += kK2Threads * 4) {
-        const int r = idx / d, c = idx % d;
-        const float4 v = *reinterpret_cast<const float4*>(Kp + (size_t)(jc * 64 + r) * d + c);
-        float* dst = stage + r * (d + 1) + c;
-        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    const int piece_rows = ((3 * 32768) / (d * 4)) & ~63;       // 384 rows at d = 64, 192 at d = 128
+    const int col = feat < p ? feat : 0;
+    uint32_t kp_phase = 0;
+    for (int r0 = 0; r0 < k && ok; r0 += piece_rows) {
+      const int rows = min(piece_rows, k - r0);
+      __syncthreads();                                            // the previous piece has been read
+      if (tid == 0) {
+        mbar_arrive_expect_tx(bar_kp, (uint32_t)rows * d * 4);
+        bulk_load(sm_op, Kp + (size_t)r0 * d, (uint32_t)rows * d * 4, bar_kp);
       }
-      __syncthreads();
-      if (warp < 4) {
-        const int col = feat < p ? feat : 0;
+      {
+        bool mine = true;
+        if (warp == 4) mine = mbar_wait(bar_kp, kp_phase, prm.status, &abort_flag);
+        ok = __syncthreads_and(mine) != 0;
+        kp_phase ^= 1;
+      }
+      if (!ok) break;
+      for (int g = warp >> 2; g < (rows >> 5); g += 2) {
+        uint32_t h[16];
+        const float* src = stage + (size_t)(g * 32) * d + col;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t h[16];
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float x0 = stage[(half * 32 + 2 * e) * (d + 1) + col];
-            const float x1 = stage[(half * 32 + 2 * e + 1) * (d + 1) + col];
-            const float f0 = x0 > 0.f ? x0 + 1.f : __expf(x0);
-            const float f1 = x1 > 0.f ? x1 + 1.f : __expf(x1);
-            const __half2 hh = __floats2half2_rn(f0, f1);
-            const float2 back = __half22float2(hh);
-            zsum += back.x + back.y;
-            h[e] = *reinterpret_cast<const uint32_t*>(&hh);
-          }
-          tmem_st16(tb + jc * 32 + half * 16, h);
+        for (int e = 0; e < 16; ++e) {
+          const float x0 = src[(2 * e) * d];
+          const float x1 = src[(2 * e + 1) * d];
+          const float f0 = fmaxf(x0, 0.f) + __expf(fminf(x0, 0.f));      // elu(x) + 1
+          const float f1 = fmaxf(x1, 0.f) + __expf(fminf(x1, 0.f));
+          const __half2 hh = __floats2half2_rn(f0, f1);
+          const float2 back = __half22float2(hh);
+          zsum += back.x + back.y;
+          h[e] = *reinterpret_cast<const uint32_t*>(&hh);
         }
+        tmem_st16(tb + ((r0 + g * 32) >> 1), h);
       }
     }
+    // the two threads of a feature add up their sums
+    __shared__ float zpart[128];
+    if (warp >= 4) zpart[(warp & 3) * 32 + lane] = zsum;
+    tmem_wait_st();
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp < 4) zsum += zpart[warp * 32 + lane];
     if (warp < 4) {
       if (feat < p) prm.weight[(size_t)head * p + feat] = zsum;
       tmem_wait_st();
