@@ -386,7 +386,7 @@ def main():
             import oracle
             oracle.build()
             t1 = oracle_sample(wr, host, 1)                        # warm + calibrate
-            heads = max(1, int(15.0 / max(t1, 1e-3)))              # about 15 s of CPU work (heads repeat)
+            heads = max(1, int(25.0 / max(t1, 1e-3)))              # 10 to 25 s of CPU work (the first, cold pass over-estimates)
             tt = oracle_sample(wr, host, heads)
             line["cpu_baseline"] = {"value": heads * w.N / tt, "unit": UNIT, "cores": oracle.threads(),
                                     "kind": "oracle",
