@@ -27,7 +27,9 @@
  * Errors.  Every function returns FLURKA_OK (0) or a negative flurka_status; on error NOTHING has been
  * launched or copied.  No exceptions, no abort, nothing is printed.
  *
- * Threads.  One call at a time per process (the workspace and the descriptor cache are shared).
+ * Threads and devices.  One call at a time per device (each device has its own workspace, staging
+ * buffers and descriptor cache, looked up by the device that is current at the call; the settings
+ * made by flurka_set_path, flurka_set_cta_limit and flurka_set_stage_timing are process-wide).
  */
 #ifndef FLURKA_H_
 #define FLURKA_H_
@@ -84,7 +86,11 @@ typedef enum {
  * Pointers 16-byte aligned.  The tensor-core path additionally needs bf16, d in {64, 128},
  * N % 8 == 0, k % 64 == 0 with k <= 512, and (PERFORMER) m in {64, 128, 192, 256}; other shapes run
  * on the SIMT path.  The call enqueues work and returns; it never synchronises.  Scratch comes from the
- * workspace set by flurka_set_workspace(), or from one the library allocates (and re-uses) on first need.
+ * workspace set by flurka_set_workspace(), or from one the library obtains on first need and re-uses:
+ * when a later problem needs more, the old block is released and a larger one obtained in stream order
+ * on `stream` (cudaFreeAsync / cudaMallocAsync), so calls that share the library-owned workspace must
+ * be ordered one after the other by the caller, and a call that grows it should not sit inside a
+ * stream capture (hand over a workspace with flurka_set_workspace() for that).
  */
 int flurka_forward(const void* Q, const void* K, const void* V, const void* E, const void* F,
                    const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
@@ -107,8 +113,9 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
  * fp32 projections K', V' (Eq. (2)'s E K and F V), the key-side feature summaries and a status word. */
 size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m);
 
-/* Hands the library a caller-owned device workspace (256-byte aligned). NULL/0 returns to the
- * library-owned one. The caller keeps it alive until the last call using it has finished. */
+/* Hands the library a caller-owned device workspace (256-byte aligned) for the current device.
+ * NULL/0 returns to the library-owned one. The caller keeps it alive until the last call using it
+ * has finished. */
 int flurka_set_workspace(void* dev_ptr, size_t bytes);
 
 /* Forces an execution path for later calls (flurka_path_t); returns the previous one. */
@@ -135,7 +142,7 @@ int flurka_last_launches(void);
 int flurka_debug_copy(int which, void* dev_dst, size_t bytes, void* stream);
 
 /* Synchronises the device and returns the status word the kernels of the last call left behind:
- * 0 = clean; bit 0 = a bounded wait gave up (results invalid); bit 1 = an index check failed. */
+ * 0 = clean; bit 0 = a bounded wait gave up (results invalid). */
 int flurka_last_status(void);
 
 /* cudaError_t (as int) behind the most recent FLURKA_ERR_CUDA. */
@@ -172,10 +179,12 @@ int flurka_version(void);
  *
  * Arguments, layouts, element types and error codes are those of flurka_forward; inputs and `out`
  * are still the caller's device buffers.  Differences:
- *   - a problem whose flurka_workspace_bytes() exceeds FLURKA_STATIC_SCRATCH_BYTES is refused with
- *     FLURKA_ERR_TOO_LARGE and nothing is launched;
+ *   - a problem whose flurka_static_scratch_need() exceeds FLURKA_STATIC_SCRATCH_BYTES is refused
+ *     with FLURKA_ERR_TOO_LARGE and nothing is launched (that need is a little below
+ *     flurka_workspace_bytes(), which also reserves room only the tensor-core kernels use);
  *   - it always runs the fp32 CUDA-core kernels (flurka_set_path is ignored), and it does not feed
- *     flurka_debug_copy / flurka_last_status / flurka_last_path;
+ *     flurka_debug_copy / flurka_last_status / flurka_last_path / flurka_last_stage_ms, which keep
+ *     describing the last flurka_forward;
  *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current); make that first call outside any stream capture;
  *   - all calls share the one array and it keeps what the last call left there.  The call itself
@@ -183,6 +192,9 @@ int flurka_version(void);
  *     streams, or this one next to another thread's) race on it: serialise them.
  */
 #define FLURKA_STATIC_SCRATCH_BYTES (8u << 20)
+/* Bytes of the built-in array flurka_forward_static_scratch would use for this problem (0 on invalid
+ * arguments).  (Like the entry point itself, without a counterpart in the paper.) */
+size_t flurka_static_scratch_need(int variant, int B, int H, int N, int d, int k, int m);
 int flurka_forward_static_scratch(const void* Q, const void* K, const void* V, const void* E,
                                   const void* F, const void* W, int variant, int B, int H, int N,
                                   int d, int k, int m, void* out, void* stream);

@@ -20,7 +20,7 @@ EXPORTS = [
     "flurka_forward", "flurka_forward_host", "flurka_workspace_bytes", "flurka_set_workspace",
     "flurka_set_path", "flurka_set_cta_limit", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
     "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
-    "flurka_strerror", "flurka_version", "flurka_forward_static_scratch",
+    "flurka_strerror", "flurka_version", "flurka_forward_static_scratch", "flurka_static_scratch_need",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -61,6 +61,8 @@ def load() -> ctypes.CDLL:
     lib.flurka_forward_static_scratch.argtypes = fwd_args
     lib.flurka_workspace_bytes.restype = sz
     lib.flurka_workspace_bytes.argtypes = [ci] * 7
+    lib.flurka_static_scratch_need.restype = sz
+    lib.flurka_static_scratch_need.argtypes = [ci] * 7
     lib.flurka_set_workspace.restype = ci
     lib.flurka_set_workspace.argtypes = [vp, sz]
     lib.flurka_set_path.restype = ci
@@ -169,6 +171,11 @@ def flurka_forward_host(Q, K, V, E, F, W, variant, out=None, stream=None, layout
 
 def flurka_workspace_bytes(variant, io_dtype, B, H, N, d, k, m) -> int:
     return int(load().flurka_workspace_bytes(_variant_word(variant, io_dtype), B, H, N, d, k, m))
+
+
+def flurka_static_scratch_need(variant, io_dtype, B, H, N, d, k, m) -> int:
+    """Bytes of the built-in scratch array flurka_forward_static_scratch would use (0: invalid arguments)."""
+    return int(load().flurka_static_scratch_need(_variant_word(variant, io_dtype), B, H, N, d, k, m))
 
 
 def flurka_set_workspace(buf) -> None:

@@ -29,15 +29,16 @@ struct Problem {
 };
 
 // Workspace layout (all offsets 256-byte aligned):
+//   status  int32[4] at offset 0 whatever the problem, then one arrival counter per
+//           (head, 128-feature tile) of stage 2
 //   kpvp    fp32 [2][BH][k][d]     K' then V'
-//   status  int32[4], then one arrival counter per (head, 128-feature tile) of stage 2
-//           (kpvp and status are adjacent: one memset per forward clears both)
+//           (status and kpvp are adjacent: one memset per forward clears both)
 //   weight  fp32 [BH][p]           b_i (PERFORMER) or z_i (RNN)
 //   a32     fp32 [BH][p][d]        key-side summary, feature-major
 //   aT16    fp16 [BH][d][p]        the same, transposed, as the tensor-core B operand
 //   part    fp32 partial results of a key-split stage 2 (tensor-core path only)
 struct Layout {
-  size_t kpvp, weight, a32, aT16, status, status_bytes, part, total;
+  size_t status, status_bytes, kpvp, kpvp_end, weight, a32, aT16, part, total;
 };
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -47,9 +48,9 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 Layout make_layout(const Problem& pr, bool with_split_scratch = true) {
   Layout L;
   size_t off = 0;
-  L.kpvp = off;   off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
   L.status_bytes = 16 + (with_split_scratch ? (size_t)pr.BH() * ((pr.p() + 127) / 128) * 4 : 0);
   L.status = off; off = align256(off + L.status_bytes);
+  L.kpvp = off;   L.kpvp_end = off + (size_t)2 * pr.BH() * pr.k * pr.d * 4; off = align256(L.kpvp_end);
   L.weight = off; off = align256(off + (size_t)pr.BH() * pr.p() * 4);
   L.a32 = off;    off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 4);
   L.aT16 = off;   off = align256(off + (size_t)pr.BH() * pr.p() * pr.d * 2);
@@ -61,15 +62,15 @@ Layout make_layout(const Problem& pr, bool with_split_scratch = true) {
   return L;
 }
 
-struct State {
+// Everything that belongs to one GPU: scratch, staging, streams, events, tensor maps and the record
+// of the last forward.  Slot = CUDA device ordinal of the device that is current at the call.
+struct DeviceState {
   void* user_ws = nullptr;
   size_t user_ws_bytes = 0;
   void* own_ws = nullptr;
   size_t own_ws_bytes = 0;
-  int path = FLURKA_PATH_AUTO;
   int last_path = 0;
   int last_launches = 0;
-  int last_cuda_error = 0;
   // most recent forward (for flurka_debug_copy / flurka_last_status)
   bool have_last = false;
   Problem last_problem{};
@@ -80,15 +81,29 @@ struct State {
   cudaStream_t out_stream = nullptr;   // device-to-host copies of finished head groups
   cudaEvent_t group_done[8] = {};      // one per head group of a host-buffer call
   cudaEvent_t out_done = nullptr;
-  bool keep_status = false;            // later head groups of one host-buffer call keep the status words
   StageTimer timer;
-  TensorMaps maps;
+  TensorContext tc;
 };
 
-State g;
+constexpr int kMaxDevices = 64;
+DeviceState g_dev[kMaxDevices];
+
+// Process-wide settings
+int g_path = FLURKA_PATH_AUTO;
+bool g_stage_timing = false;
+int g_last_cuda_error = 0;
+
+// The slot of the current device (slot 0 when there is no usable device: the calls that reach
+// this without one only touch host-side fields).
+DeviceState& dev_state() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); dev = 0; }
+  if (dev < 0 || dev >= kMaxDevices) dev = 0;
+  return g_dev[dev];
+}
 
 int cuda_fail(cudaError_t e) {
-  g.last_cuda_error = (int)e;
+  g_last_cuda_error = (int)e;
   (void)cudaGetLastError();
   return FLURKA_ERR_CUDA;
 }
@@ -122,34 +137,38 @@ bool tensor_path_ok(const Problem& pr) {
   if (pr.N % 8) return false;       // row pitch of E, F (N elements) must be a multiple of 16 bytes for TMA
   if (pr.k % 64 || pr.k > 512) return false;
   if (pr.kernel == FLURKA_PERFORMER && (pr.m % 64 || pr.m > 256)) return false;
-  return tensor_path_built();
+  return true;
 }
 
-int get_workspace(size_t need, char** ws) {
-  if (g.user_ws) {
-    if (g.user_ws_bytes < need) return FLURKA_ERR_WORKSPACE;
-    *ws = (char*)g.user_ws;
+// The library-owned workspace grows in stream order: the old block is released and the new one
+// obtained on the call's stream, so nothing waits on the host and earlier work queued on that
+// stream still finds its block.
+int get_workspace(DeviceState& ds, size_t need, cudaStream_t st, char** ws) {
+  if (ds.user_ws) {
+    if (ds.user_ws_bytes < need) return FLURKA_ERR_WORKSPACE;
+    *ws = (char*)ds.user_ws;
     return FLURKA_OK;
   }
-  if (g.own_ws_bytes < need) {
-    if (g.own_ws) {
-      cudaError_t e = cudaDeviceSynchronize();
+  if (ds.own_ws_bytes < need) {
+    if (ds.own_ws) {
+      cudaError_t e = cudaFreeAsync(ds.own_ws, st);
       if (e != cudaSuccess) return cuda_fail(e);
-      cudaFree(g.own_ws);
-      g.own_ws = nullptr;
-      g.own_ws_bytes = 0;
+      ds.own_ws = nullptr;
+      ds.own_ws_bytes = 0;
+      ds.have_last = false;
     }
-    cudaError_t e = cudaMalloc(&g.own_ws, need);
-    if (e != cudaSuccess) { cuda_fail(e); return FLURKA_ERR_WORKSPACE; }
-    g.own_ws_bytes = need;
+    cudaError_t e = cudaMallocAsync(&ds.own_ws, need, st);
+    if (e != cudaSuccess) { cuda_fail(e); ds.own_ws = nullptr; return FLURKA_ERR_WORKSPACE; }
+    ds.own_ws_bytes = need;
   }
-  *ws = (char*)g.own_ws;
+  *ws = (char*)ds.own_ws;
   return FLURKA_OK;
 }
 
 int check_device() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return FLURKA_ERR_DEVICE; }
+  if (dev < 0 || dev >= kMaxDevices) return FLURKA_ERR_DEVICE;
   int major = 0;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -218,11 +237,13 @@ int key_side_dispatch(const Problem& pr, const float* kpvp, const void* W, float
 }
 
 // The three stages in order.  tc1 / tc3 choose the tensor-core kernel for stage 1 / stage 3
-// (bf16 only); tc2 (which needs tc3) does the same for stage 2.
+// (bf16 only); tc2 (which needs tc3) does the same for stage 2.  `timer` (may be NULL) gets an
+// event before and after each stage.  `keep_status`: the status words are left as they are (a
+// later head group of one host-buffer call; they only ever gain bits).
 template <typename T>
 int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
                  const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc2,
-                 bool tc3, int* launches) {
+                 bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status, int* launches) {
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
   float* a32 = (float*)(ws + L.a32);
@@ -230,53 +251,46 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   int* status = (int*)(ws + L.status);
   const bool performer = pr.kernel == FLURKA_PERFORMER;
   int cuda_err = 0;
-  // one memset: the K', V' accumulators (the kernels add into them), the status words and the counters
-  // (a later head group of a host-buffer call leaves the status words, which only ever gain bits, and
-  // the counters, which stage 2 hands back at zero)
-  cudaError_t e = cudaMemsetAsync(ws + L.kpvp, 0, (g.keep_status ? L.status : L.status + L.status_bytes) - L.kpvp, st);
+  // one memset: the status words, the arrival counters and the K', V' accumulators the kernels add into
+  const size_t clear_from = L.status + (keep_status ? 16 : 0);
+  cudaError_t e = cudaMemsetAsync(ws + clear_from, 0, L.kpvp_end - clear_from, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  g.timer.mark(0, st);
+  if (timer) timer->mark(0, st);
   int rc;
   if (tc1) {
-    rc = launch_k1(g.maps, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err);
-    if (rc) { g.last_cuda_error = cuda_err; return rc; }
+    rc = launch_k1(*tc, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err);
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
     ++*launches;
   } else {
     rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
     if (rc) return rc;
   }
-  g.timer.mark(1, st);
+  if (timer) timer->mark(1, st);
   if (tc2) {
     float* part = L.total > L.part ? (float*)(ws + L.part) : nullptr;
-    rc = launch_k2(g.maps, performer, kpvp, W, weight, aT16, part, status + 4, pr.BH(), pr.d, pr.k, pr.p(), status, st,
+    rc = launch_k2(*tc, performer, kpvp, W, weight, aT16, part, status + 4, pr.BH(), pr.d, pr.k, pr.p(), status, st,
                    &cuda_err);
-    if (rc) { g.last_cuda_error = cuda_err; return rc; }
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
     ++*launches;
   } else {
     rc = key_side_dispatch<T>(pr, kpvp, W, weight, tc3 ? nullptr : a32, tc3 ? aT16 : nullptr, st, launches);
     if (rc) return rc;
   }
-  g.timer.mark(2, st);
+  if (timer) timer->mark(2, st);
   if (tc3) {
-    rc = launch_k3(g.maps, performer, Q, W, aT16, weight, out, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.p(),
+    rc = launch_k3(*tc, performer, Q, W, aT16, weight, out, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.p(),
                    status, st, &cuda_err);
-    if (rc) { g.last_cuda_error = cuda_err; return rc; }
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
     ++*launches;
   } else {
     rc = performer ? launch_simt_query_side<T, true>(pr, Q, W, weight, a32, out, st, launches)
                    : launch_simt_query_side<T, false>(pr, Q, W, weight, a32, out, st, launches);
     if (rc) return rc;
   }
-  g.timer.mark(3, st);
+  if (timer) timer->mark(3, st);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return FLURKA_OK;
-}
-
-template <typename T>
-int run_simt(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
-             const void* E, const void* F, const void* W, void* out, cudaStream_t st, int* launches) {
-  return run_pipeline<T>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, false, launches);
 }
 
 int validate_pointers(const Problem& pr, const void* Q, const void* K, const void* V, const void* E,
@@ -294,6 +308,55 @@ int validate_pointers(const Problem& pr, const void* Q, const void* K, const voi
   return FLURKA_OK;
 }
 
+// flurka_forward proper.  `reserve` (>= the problem's own need, or 0) is the workspace size to ask
+// for, so that a caller that runs several problems in a row gets one block that fits them all.
+int forward_device(const void* Q, const void* K, const void* V, const void* E, const void* F, const void* W,
+                   int variant, int B, int H, int N, int d, int k, int m, void* out, void* stream,
+                   bool keep_status, size_t reserve) {
+  Problem pr;
+  int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
+  if (rc) return rc;
+  rc = validate_pointers(pr, Q, K, V, E, F, W, out);
+  if (rc) return rc;
+  int path = g_path;
+  const bool tensor_ok = tensor_path_ok(pr);
+  if (path >= FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
+  if (path == FLURKA_PATH_AUTO) path = tensor_ok ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
+  rc = check_device();
+  if (rc) return rc;
+  DeviceState& ds = dev_state();
+  const Layout L = make_layout(pr);
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = nullptr;
+  rc = get_workspace(ds, std::max(L.total, reserve), st, &ws);
+  if (rc) return rc;
+  int launches = 0;
+  ds.timer.on = g_stage_timing;
+  StageTimer* timer = g_stage_timing ? &ds.timer : nullptr;
+  if (timer) {
+    rc = timer->create();
+    if (rc != cudaSuccess) return cuda_fail((cudaError_t)rc);
+  }
+  if (pr.fp32) {
+    rc = run_pipeline<float>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, false, &ds.tc, timer, keep_status,
+                             &launches);
+  } else {
+    const bool tc1 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE1;
+    const bool tc2 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE23;
+    const bool tc3 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE3 || tc2;
+    rc = run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, tc1, tc2, tc3, &ds.tc, timer,
+                                     keep_status, &launches);
+  }
+  if (rc) return rc;
+  ds.timer.have = g_stage_timing;
+  ds.last_path = path;
+  ds.last_launches = launches;
+  ds.have_last = true;
+  ds.last_problem = pr;
+  ds.last_ws = ws;
+  return FLURKA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -301,39 +364,7 @@ extern "C" {
 int flurka_forward(const void* Q, const void* K, const void* V, const void* E, const void* F,
                    const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
                    void* stream) {
-  Problem pr;
-  int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
-  if (rc) return rc;
-  rc = validate_pointers(pr, Q, K, V, E, F, W, out);
-  if (rc) return rc;
-  int path = g.path;
-  const bool tensor_ok = tensor_path_ok(pr);
-  if (path >= FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
-  if (path == FLURKA_PATH_AUTO) path = tensor_ok ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
-  rc = check_device();
-  if (rc) return rc;
-  const Layout L = make_layout(pr);
-  char* ws = nullptr;
-  rc = get_workspace(L.total, &ws);
-  if (rc) return rc;
-  cudaStream_t st = (cudaStream_t)stream;
-  int launches = 0;
-  if (pr.fp32) {
-    rc = run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
-  } else {
-    const bool tc1 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE1;
-    const bool tc2 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE23;
-    const bool tc3 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE3 || tc2;
-    rc = run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, tc1, tc2, tc3, &launches);
-  }
-  if (rc) return rc;
-  g.timer.have = g.timer.on;
-  g.last_path = path;
-  g.last_launches = launches;
-  g.have_last = true;
-  g.last_problem = pr;
-  g.last_ws = ws;
-  return FLURKA_OK;
+  return forward_device(Q, K, V, E, F, W, variant, B, H, N, d, k, m, out, stream, /*keep_status=*/false, 0);
 }
 
 int flurka_forward_host(const void* Q, const void* K, const void* V, const void* E, const void* F,
@@ -346,23 +377,24 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
   if (pr.kernel == FLURKA_PERFORMER && !W) return FLURKA_ERR_NULL;
   rc = check_device();
   if (rc) return rc;
+  DeviceState& ds = dev_state();
   const size_t qb = align256(pr.qkv_elems() * pr.esize());
   const size_t eb = align256(pr.ef_elems() * pr.esize());
   const size_t wb = align256(pr.w_elems() * pr.esize());
   const size_t need = 4 * qb + 2 * eb + wb;
-  if (g.stage_bytes < need) {
-    if (g.stage) {
+  if (ds.stage_bytes < need) {
+    if (ds.stage) {
       cudaError_t e = cudaDeviceSynchronize();
       if (e != cudaSuccess) return cuda_fail(e);
-      cudaFree(g.stage);
-      g.stage = nullptr;
-      g.stage_bytes = 0;
+      cudaFree(ds.stage);
+      ds.stage = nullptr;
+      ds.stage_bytes = 0;
     }
-    cudaError_t e = cudaMalloc(&g.stage, need);
+    cudaError_t e = cudaMalloc(&ds.stage, need);
     if (e != cudaSuccess) { cuda_fail(e); return FLURKA_ERR_WORKSPACE; }
-    g.stage_bytes = need;
+    ds.stage_bytes = need;
   }
-  char* base = (char*)g.stage;
+  char* base = (char*)ds.stage;
   char* dQ = base;
   char* dK = dQ + qb;
   char* dV = dK + qb;
@@ -386,11 +418,21 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
   const int heads = pr.bnhd ? pr.B : pr.BH();
   int groups = (int)std::min<size_t>(8, qn >> 20);           // at least 1 MiB of Q per group
   groups = std::max(1, std::min(groups, heads));
-  if (groups > 1 && !g.out_stream) {
-    if ((e = cudaStreamCreateWithFlags(&g.out_stream, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+  if (groups > 1 && !ds.out_stream) {
+    if ((e = cudaStreamCreateWithFlags(&ds.out_stream, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
     for (int i = 0; i < 8; ++i)
-      if ((e = cudaEventCreateWithFlags(&g.group_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaEventCreateWithFlags(&g.out_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaEventCreateWithFlags(&ds.group_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventCreateWithFlags(&ds.out_done, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+  }
+  // The groups need not be equal (12 heads in 8 groups: 1, 2, 1, 2, ...).  One workspace that fits the
+  // largest group is obtained before the first group runs, so it never moves between groups; the
+  // status words sit at its start for every group size.
+  size_t reserve = 0;
+  for (int gi = 0; gi < groups; ++gi) {
+    const int cnt = (int)((long long)heads * (gi + 1) / groups) - (int)((long long)heads * gi / groups);
+    Problem sub = pr;
+    if (pr.bnhd) sub.B = cnt; else { sub.B = 1; sub.H = cnt; }
+    reserve = std::max(reserve, make_layout(sub).total);
   }
   const size_t head_bytes = (size_t)N * d * pr.esize() * (pr.bnhd ? H : 1);
   rc = FLURKA_OK;
@@ -403,23 +445,21 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
       rc = cuda_fail(e);
       break;
     }
-    g.keep_status = gi > 0;
-    rc = flurka_forward(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, pr.bnhd ? h1 - h0 : 1,
-                        pr.bnhd ? H : h1 - h0, N, d, k, m, dO + off, stream);
-    g.keep_status = false;
+    rc = forward_device(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, pr.bnhd ? h1 - h0 : 1,
+                        pr.bnhd ? H : h1 - h0, N, d, k, m, dO + off, stream, /*keep_status=*/gi > 0, reserve);
     if (rc) break;
     if (groups == 1) {
       if ((e = cudaMemcpyAsync(out, dO, qn, cudaMemcpyDeviceToHost, st)) != cudaSuccess) rc = cuda_fail(e);
     } else {
-      if ((e = cudaEventRecord(g.group_done[gi], st)) != cudaSuccess ||
-          (e = cudaStreamWaitEvent(g.out_stream, g.group_done[gi], 0)) != cudaSuccess ||
-          (e = cudaMemcpyAsync((char*)out + off, dO + off, len, cudaMemcpyDeviceToHost, g.out_stream)) != cudaSuccess)
+      if ((e = cudaEventRecord(ds.group_done[gi], st)) != cudaSuccess ||
+          (e = cudaStreamWaitEvent(ds.out_stream, ds.group_done[gi], 0)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)out + off, dO + off, len, cudaMemcpyDeviceToHost, ds.out_stream)) != cudaSuccess)
         rc = cuda_fail(e);
     }
   }
   if (groups > 1) {
     // the caller's stream also waits for the copies on the second stream
-    if (cudaEventRecord(g.out_done, g.out_stream) == cudaSuccess) cudaStreamWaitEvent(st, g.out_done, 0);
+    if (cudaEventRecord(ds.out_done, ds.out_stream) == cudaSuccess) cudaStreamWaitEvent(st, ds.out_done, 0);
   }
   e = cudaStreamSynchronize(st);
   if (rc) return rc;
@@ -436,15 +476,16 @@ size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, in
 int flurka_set_workspace(void* dev_ptr, size_t bytes) {
   if (dev_ptr && ((uintptr_t)dev_ptr & 255)) return FLURKA_ERR_ALIGN;
   if (dev_ptr && bytes == 0) return FLURKA_ERR_WORKSPACE;
-  g.user_ws = dev_ptr;
-  g.user_ws_bytes = dev_ptr ? bytes : 0;
-  g.have_last = false;
+  DeviceState& ds = dev_state();
+  ds.user_ws = dev_ptr;
+  ds.user_ws_bytes = dev_ptr ? bytes : 0;
+  ds.have_last = false;
   return FLURKA_OK;
 }
 
 int flurka_set_path(int path) {
-  const int prev = g.path;
-  if (path >= FLURKA_PATH_AUTO && path <= FLURKA_PATH_TENSOR_STAGE23) g.path = path;
+  const int prev = g_path;
+  if (path >= FLURKA_PATH_AUTO && path <= FLURKA_PATH_TENSOR_STAGE23) g_path = path;
   return prev;
 }
 
@@ -454,13 +495,14 @@ int flurka_set_cta_limit(int max_ctas) {
   return prev;
 }
 
-int flurka_last_path(void) { return g.last_path; }
-int flurka_last_launches(void) { return g.last_launches; }
+int flurka_last_path(void) { return dev_state().last_path; }
+int flurka_last_launches(void) { return dev_state().last_launches; }
 
 int flurka_debug_copy(int which, void* dev_dst, size_t bytes, void* stream) {
   if (!dev_dst) return FLURKA_ERR_NULL;
-  if (!g.have_last) return FLURKA_ERR_WORKSPACE;
-  const Problem& pr = g.last_problem;
+  DeviceState& ds = dev_state();
+  if (!ds.have_last) return FLURKA_ERR_WORKSPACE;
+  const Problem& pr = ds.last_problem;
   const Layout L = make_layout(pr);
   const size_t kd = (size_t)pr.BH() * pr.k * pr.d * 4;
   size_t off = 0, size = 0;
@@ -473,46 +515,40 @@ int flurka_debug_copy(int which, void* dev_dst, size_t bytes, void* stream) {
     default: return FLURKA_ERR_VARIANT;
   }
   if (bytes != size) return FLURKA_ERR_SHAPE;
-  cudaError_t e = cudaMemcpyAsync(dev_dst, g.last_ws + off, size, cudaMemcpyDeviceToDevice,
+  cudaError_t e = cudaMemcpyAsync(dev_dst, ds.last_ws + off, size, cudaMemcpyDeviceToDevice,
                                   (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
   return FLURKA_OK;
 }
 
 int flurka_last_status(void) {
-  if (!g.have_last) return 0;
-  const Layout L = make_layout(g.last_problem);
+  DeviceState& ds = dev_state();
+  if (!ds.have_last) return 0;
+  const Layout L = make_layout(ds.last_problem);
   int words[4] = {0, 0, 0, 0};
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) return cuda_fail(e);
-  e = cudaMemcpy(words, g.last_ws + L.status, 16, cudaMemcpyDeviceToHost);
+  e = cudaMemcpy(words, ds.last_ws + L.status, 16, cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e);
   return words[0];
 }
 
-int flurka_last_cuda_error(void) { return g.last_cuda_error; }
+int flurka_last_cuda_error(void) { return g_last_cuda_error; }
 
 int flurka_set_stage_timing(int on) {
-  if (on) {
-    for (int i = 0; i < 4; ++i) {
-      if (!g.timer.ev[i]) {
-        cudaError_t e = cudaEventCreate(&g.timer.ev[i]);
-        if (e != cudaSuccess) return cuda_fail(e);
-      }
-    }
-  }
-  g.timer.on = on != 0;
-  g.timer.have = false;
+  g_stage_timing = on != 0;
+  for (int i = 0; i < kMaxDevices; ++i) g_dev[i].timer.have = false;
   return FLURKA_OK;
 }
 
 int flurka_last_stage_ms(float* ms3) {
   if (!ms3) return FLURKA_ERR_NULL;
-  if (!g.timer.have) return FLURKA_ERR_WORKSPACE;
-  cudaError_t e = cudaEventSynchronize(g.timer.ev[3]);
+  DeviceState& ds = dev_state();
+  if (!ds.timer.have) return FLURKA_ERR_WORKSPACE;
+  cudaError_t e = cudaEventSynchronize(ds.timer.ev[3]);
   if (e != cudaSuccess) return cuda_fail(e);
   for (int i = 0; i < 3; ++i) {
-    e = cudaEventElapsedTime(&ms3[i], g.timer.ev[i], g.timer.ev[i + 1]);
+    e = cudaEventElapsedTime(&ms3[i], ds.timer.ev[i], ds.timer.ev[i + 1]);
     if (e != cudaSuccess) return cuda_fail(e);
   }
   return FLURKA_OK;
@@ -536,6 +572,12 @@ const char* flurka_strerror(int code) {
 
 int flurka_version(void) { return FLURKA_VERSION; }
 
+size_t flurka_static_scratch_need(int variant, int B, int H, int N, int d, int k, int m) {
+  Problem pr;
+  if (parse_problem(variant, B, H, N, d, k, m, &pr)) return 0;
+  return make_layout(pr, /*with_split_scratch=*/false).total;
+}
+
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------
@@ -548,7 +590,6 @@ namespace {
 
 static __device__ __align__(256) unsigned char g_static_scratch[FLURKA_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
 char* g_static_scratch_addr[kMaxDevices] = {};
 
 int static_scratch_address(char** out) {
@@ -577,6 +618,7 @@ extern "C" int flurka_forward_static_scratch(const void* Q, const void* K, const
   if (rc) return rc;
   rc = validate_pointers(pr, Q, K, V, E, F, W, out);
   if (rc) return rc;
+  // the CUDA-core kernels' scratch: no partial results of a split key side
   const Layout L = make_layout(pr, /*with_split_scratch=*/false);
   if (L.total > (size_t)FLURKA_STATIC_SCRATCH_BYTES) return FLURKA_ERR_TOO_LARGE;
   rc = check_device();
@@ -585,9 +627,13 @@ extern "C" int flurka_forward_static_scratch(const void* Q, const void* K, const
   rc = static_scratch_address(&ws);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  // The array still holds the previous call's contents: run_simt zeroes the K', V' accumulators
-  // and the status words before the kernels add into them.
+  // The array still holds the previous call's contents: the pipeline zeroes the status words and the
+  // K', V' accumulators before the kernels add into them.  No stage timing and no record of the call
+  // is kept: flurka_last_stage_ms and the other flurka_last_* queries keep describing flurka_forward.
   int launches = 0;
-  if (pr.fp32) return run_simt<float>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
-  return run_simt<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, &launches);
+  if (pr.fp32)
+    return run_pipeline<float>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, false, nullptr, nullptr, false,
+                               &launches);
+  return run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, false, nullptr, nullptr,
+                                     false, &launches);
 }

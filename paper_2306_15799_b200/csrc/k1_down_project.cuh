@@ -22,7 +22,6 @@ struct K1Params {
   int col_groups;  // ceil(BH * d / 256)
   int k_halves;    // ceil(k / 256)
   int* status;
-  unsigned long long* trace;   // optional [gridDim.x][4] nanosecond stamps: start, set up, accumulated, done
 };
 
 constexpr int kK1Stages = 3;
@@ -46,7 +45,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   __shared__ uint32_t tmem_base_shared;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x] = global_timer_ns();
 
   // ---- which piece of the problem
   int idx = blockIdx.x;
@@ -88,7 +86,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   }
   __syncthreads();
   const uint32_t tmem = tmem_base_shared;
-  if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 1] = global_timer_ns();
 
   if (nchunks > 0) {
     if (warp == 0 && lane == 0) {
@@ -150,7 +147,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
       const int q = warp & 3;                                // TMEM lane quadrant of this warp
       bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
       if (warp == 2 && lane == 0) grid_launch_dependents();   // only the epilogue is left
-      if (p.trace && warp == 2 && lane == 0) p.trace[4 * blockIdx.x + 2] = global_timer_ns();
       if (ok) {
         tcgen05_fence_after();
         const uint32_t stage_buf = smem_base + (warp - 2) * 32768;   // 8 x 4 KB, pipeline is drained
@@ -191,7 +187,6 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (p.trace && threadIdx.x == 0) p.trace[4 * blockIdx.x + 3] = global_timer_ns();
   if (warp == 1) tmem_dealloc(tmem, tmem_cols);
 }
 

@@ -37,7 +37,6 @@ struct K2Params {
   float* weight;            // [BH][p]      b_i (PERFORMER) or z_i (RNN)
   __half* aT16;             // [BH][d][p]   a^T
   int* status;
-  long long* trace;         // optional [gridDim.x][8] cycle sums of thread 0 (see K2_STAMP)
   int nsplit;               // CTAs per (head, feature tile) along the keys (1..4; PERFORMER only)
   float* part;              // nsplit > 1: [BH * ftiles][nsplit][d + 2][128]  max, sum, accumulator columns
   int* counters;            // nsplit > 1: [BH * ftiles], zero on entry, zero again on exit
@@ -84,11 +83,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   __shared__ uint32_t tmem_base_shared;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
-  long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  long long tlast = clock64();
-  const bool tracing = prm.trace != nullptr && tid == 0;
-#define K2_STAMP(slot) \
-  if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
   const int d = prm.d, k = prm.k, p = prm.p;
   const int nsplit = prm.nsplit;
   const int sp = blockIdx.x % nsplit;                         // which part of the keys
@@ -142,7 +136,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   const uint32_t tmem = tmem_base_shared;
   bool ok = true;
   uint32_t mma_phase = 0;
-  K2_STAMP(0)
   // everything above (and the W tile on its way) is independent of stage 1
   grid_dependency_wait();
 
@@ -239,7 +232,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       // the staging buffer has been read out: start the next copy (the next K' chunk, or the first
       // V' chunk of the second product) under this chunk's MMAs
       if (tid == 0) stage_chunk(jc + 1 < nchunks ? Kp : Vp, jc + 1 < nchunks ? jc_begin + jc + 1 : jc_begin);
-      K2_STAMP(1)
       if (tid == 128) {
         tcgen05_fence_after();
         const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, (uint32_t)rows);
@@ -258,7 +250,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       }
       // the operand tiles are rewritten for the next chunk: wait until the MMAs have read them
       wait_mma();
-      K2_STAMP(2)
     }
   }
 
@@ -354,7 +345,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
     }
   }
   __syncthreads();
-  K2_STAMP(3)
 
   // ---- a = weights x V', streamed in chunks of up to 128 keys; V' = hi + lo in fp16, MN-major slabs
   {
@@ -382,7 +372,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
       fence_proxy_async_smem();
       __syncthreads();
       if (tid == 0 && jc + 1 < nchunks) stage_chunk(Vp, jc_begin + jc + 1);
-      K2_STAMP(4)
       if (tid == 128) {
         tcgen05_fence_after();
         // B: 64-column slabs 16384 B apart, 8-key groups 1024 B apart, 16 keys = 2048 B per step;
@@ -397,7 +386,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
         mma_commit(bar_mma);
       }
       wait_mma();
-      K2_STAMP(5)
     }
   }
 
@@ -489,11 +477,6 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   }
   tcgen05_fence_before();
   __syncthreads();
-  K2_STAMP(6)
-#undef K2_STAMP
-  if (tracing) {
-    for (int sidx = 0; sidx < 8; ++sidx) prm.trace[(size_t)blockIdx.x * 8 + sidx] = tacc[sidx];
-  }
   if (warp == 4) tmem_dealloc(tmem, 512);
 }
 

@@ -34,7 +34,6 @@ struct K3Params {
   const float* weight;      // [BH][p]  b_i or z_i
   __nv_bfloat16* out;       // [BH][N][d]
   int* status;
-  long long* trace;         // optional [gridDim.x][3][8] cycle sums: two row-owner groups, then the issuers
 };
 
 constexpr int kK3Threads = 384;
@@ -204,9 +203,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         const uint32_t idesc1 = make_idesc(kFmtBF16, 0, 0, 128, (uint32_t)p);
         bool ok = mbar_wait(bar_wfull, 0, prm.status, &abort_flag);
         int head_prev = -1, events = 0;
-        const bool mtracing = prm.trace != nullptr;
-        long long macc[2] = {0, 0};
-        long long mlast = mtracing ? clock64() : 0;
         for (int i = 0; i < ntiles && ok; ++i) {
           const int head = (t_begin + i) / prm.tiles_per_head;
           const int buf = i & (NB - 1), st = i % NS;
@@ -221,7 +217,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i / NS) & 1, prm.status, &abort_flag);
           if (!ok) break;
           tcgen05_fence_after();
-          if (mtracing) { const long long now = clock64(); macc[0] += now - mlast; mlast = now; }
           const uint32_t tb = tmem + buf * buf_cols;
           const uint32_t qb = base + L.q + st * q_stage_bytes;
           for (int kb = 0; kb < kq; ++kb) {
@@ -237,11 +232,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           }
           mma_commit(bar_sfull + 8 * buf);
           mma_commit(bar_qempty + 8 * st);         // the Q tile is free once these MMAs have read it
-          if (mtracing) { const long long now = clock64(); macc[1] += now - mlast; mlast = now; }
-        }
-        if (mtracing) {
-          prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 0] = macc[0];
-          prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 1] = macc[1];
         }
       }
     } else if (warp == 3 && lane == 0) {
@@ -253,9 +243,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const uint32_t idesc2 = make_idesc(kFmtF16, 0, 0, 128, (uint32_t)d);
       bool ok = true;
       int head_prev = -1, events = 0;
-      const bool mtracing = prm.trace != nullptr;
-      long long macc[2] = {0, 0};
-      long long mlast = mtracing ? clock64() : 0;
       for (int j = 0; j < ntiles && ok; ++j) {
         const int head = (t_begin + j) / prm.tiles_per_head;
         const int buf = j & (NB - 1);
@@ -268,7 +255,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         ok = mbar_wait(bar_pfull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag);
         if (!ok) break;
         tcgen05_fence_after();
-        if (mtracing) { const long long now = clock64(); macc[0] += now - mlast; mlast = now; }
         const uint32_t tb = tmem + buf * buf_cols;
         // four 16-wide steps per call: one 64-feature block of p (TMEM) against one block of a^T
         for (int kb = 0; kb < kp; ++kb) {
@@ -278,11 +264,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         mma_commit(bar_ofull + 8 * buf);
         const bool last_of_head = (j + 1 < ntiles) && ((t_begin + j + 1) / prm.tiles_per_head != head);
         if (last_of_head) mma_commit(bar_drained);
-        if (mtracing) { const long long now = clock64(); macc[1] += now - mlast; mlast = now; }
-      }
-      if (mtracing) {
-        prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 2] = macc[0];
-        prm.trace[((size_t)blockIdx.x * 3 + 2) * 8 + 3] = macc[1];
       }
     } else if (warp == 2) {
       // ============================================================ per-head operand builder
@@ -337,13 +318,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const float kLog2e = 1.4426950408889634f;
       int events = 0;
       bool ok = true;
-      // optional cycle accounting of one thread per group: 0 wait for S (or Q), 1 pass 1,
-      // 2 pass 2 + hand-over, 3 wait for O, 4 normalise + store
-      const bool tracing = prm.trace != nullptr && q4 == 0 && lane == 0;
-      long long tacc[6] = {0, 0, 0, 0, 0, 0};
-      long long tlast = tracing ? clock64() : 0;
-#define K3_STAMP(slot) \
-  if (tracing) { const long long now = clock64(); tacc[slot] += now - tlast; tlast = now; }
       // read-out of tile j: O / sum -> bf16 -> this thread's output row, 32 bytes per store
       // (head and first row of the tile are tracked by the caller: no divisions on this path)
       auto read_out = [&](int j, float inv, int head, int row0) -> bool {
@@ -351,7 +325,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         const uint32_t tb = tmem + buf * buf_cols + lane_off + o_col;
         if (!mbar_wait(bar_ofull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag)) return false;
         tcgen05_fence_after();
-        K3_STAMP(3)
         __nv_bfloat16* orow = prm.H > 0
             ? prm.out + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * d
             : prm.out + ((size_t)head * prm.N + row0 + row) * d;
@@ -383,7 +356,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                          : "memory");
           }
         }
-        K3_STAMP(4)
         return true;
       };
       float inv_prev = 0.f;                            // four buffers: 1 / sum of the group's previous tile
@@ -403,7 +375,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           ok = mbar_wait(bar_sfull + 8 * buf, (i >> nb_shift) & 1, prm.status, &abort_flag);
           if (!ok) break;
           tcgen05_fence_after();
-          K3_STAMP(0)
           // Two passes over the row with double-buffered TMEM loads: while one 32-column chunk is
           // being worked on, the next one is already in flight.
           // pass 1: row maximum
@@ -432,7 +403,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           }
           mx = fmaxf(fmax3(mx, mx1, mx2), mx3);
           const float shift = mx * kLog2e;
-          K3_STAMP(1)
           // pass 2: p = 2^(S log2e - shift), fp16 pairs back into columns [c/2, c/2+16)
           for (int c = 0; c < p; c += 64) {
             uint32_t h[16];
@@ -472,7 +442,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i >> ns_shift) & 1, prm.status, &abort_flag);
           if (!ok) break;
-          K3_STAMP(0)
           const uint32_t qb = base + L.q + st * q_stage_bytes;
           const float* sc = reinterpret_cast<const float*>(base_ptr + L.scale);
           for (int c = 0; c < d; c += 32) {
@@ -508,7 +477,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         tmem_wait_st();
         tcgen05_fence_before();
         mbar_arrive(bar_pfull + 8 * buf);
-        K3_STAMP(2)
 
         const float inv = 1.f / fmaxf(denom + denom1, 1.17549435e-38f);
         if (NB == 4) {
@@ -525,10 +493,6 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         while (tih >= prm.tiles_per_head) { tih -= prm.tiles_per_head; ++head_i; }
       }
       if (NB == 4 && ok && ntiles > grp) (void)read_out(grp + 2 * ((ntiles - 1 - grp) / 2), inv_prev, head_o, row0_o);
-#undef K3_STAMP
-      if (tracing) {
-        for (int sidx = 0; sidx < 6; ++sidx) prm.trace[((size_t)blockIdx.x * 3 + grp) * 8 + sidx] = tacc[sidx];
-      }
     }
   }
   tcgen05_fence_before();

@@ -17,12 +17,20 @@ struct StageTimer {
   bool on = false;
   bool have = false;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  // creates the events on the current device on first use; returns a cudaError_t as int
+  int create() {
+    for (int i = 0; i < 4; ++i) {
+      if (!ev[i]) {
+        cudaError_t e = cudaEventCreate(&ev[i]);
+        if (e != cudaSuccess) return (int)e;
+      }
+    }
+    return 0;
+  }
   void mark(int i, cudaStream_t st) {
     if (on && ev[i]) cudaEventRecord(ev[i], st);
   }
 };
-
-inline bool tensor_path_built() { return true; }
 
 // ---------------------------------------------------------------------------------------------
 // cuTensorMapEncodeTiled is fetched from the driver at run time, so the library links against
@@ -81,20 +89,33 @@ struct TensorMaps {
   CachedMap E, F, K, V, kpvp, Q, W, W2, aT;
 };
 
+// Per-device context of the tensor-core kernels: the cached tensor maps (their pointers are device
+// addresses), the SM count, and whether the kernels' shared-memory limits have been raised there.
+struct TensorContext {
+  TensorMaps maps;
+  int sms = 0;
+  bool k1_attr = false;
+  int sm_total() {
+    if (!sms) {
+      int dev = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      if (sms <= 0) sms = 148;
+    }
+    return sms;
+  }
+  // SMs the persistent kernels may use (the test knob caps it)
+  int sm_count();
+};
+
 // 0 = use every SM; otherwise the persistent kernels are launched with at most this many CTAs
 inline int& cta_limit() {
   static int limit = 0;
   return limit;
 }
 
-inline int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
+inline int TensorContext::sm_count() {
+  const int n = sm_total();
   const int lim = cta_limit();
   return (lim > 0 && lim < n) ? lim : n;
 }
@@ -102,8 +123,8 @@ inline int sm_count() {
 // Sequence splits of stage 1: as few as fill the machine once.  Every split adds a full copy of
 // the output to the fp32 reduction (measured: the reduce-add traffic of all CTAs drains at about
 // 2.5 TB/s after the last MMA, so more, shorter CTAs lose more in that tail than they gain).
-inline int k1_choose_nsplit(int units, int chunks) {
-  int ns = sm_count() / units;
+inline int k1_choose_nsplit(int sms, int units, int chunks) {
+  int ns = sms / units;
   if (ns < 1) ns = 1;
   if (ns > chunks) ns = chunks;
   return ns;
@@ -111,8 +132,9 @@ inline int k1_choose_nsplit(int units, int chunks) {
 
 // ---- stage 1: K' = E K, V' = F V into kpvp (already zeroed) ----------------------------------
 // H > 0: K, V are [B,N,H,d] (H heads merged into the row); H == 0: [B,H,N,d]
-inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E, const void* F, float* kpvp,
+inline int launch_k1(TensorContext& tc, const void* K, const void* V, const void* E, const void* F, float* kpvp,
                      int BH, int H, int N, int d, int k, int* status, cudaStream_t st, int* cuda_err) {
+  TensorMaps& tm = tc.maps;
   const unsigned long long dE[2] = {(unsigned long long)N, (unsigned long long)k};
   const unsigned bE[2] = {64, 128};
   // [B,N,H,d] is a 3-D tensor too: rows of H*d elements, head h at columns h*d .. h*d+d-1
@@ -133,14 +155,12 @@ inline int launch_k1(TensorMaps& tm, const void* K, const void* V, const void* E
   p.N = N; p.d = d; p.k = k; p.BH = BH; p.H = H;
   p.col_groups = (BH * d + 255) / 256;
   p.k_halves = (k + 255) / 256;
-  p.nsplit = k1_choose_nsplit(2 * p.col_groups * p.k_halves, (N + 63) / 64);
+  p.nsplit = k1_choose_nsplit(tc.sm_count(), 2 * p.col_groups * p.k_halves, (N + 63) / 64);
   p.status = status;
-  p.trace = nullptr;
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!tc.k1_attr) {
     cudaError_t e = cudaFuncSetAttribute(k1_down_project, cudaFuncAttributeMaxDynamicSharedMemorySize, kK1SmemBytes);
     if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
-    attr_set = true;
+    tc.k1_attr = true;
   }
   const int grid = 2 * p.k_halves * p.col_groups * p.nsplit;
   k1_down_project<<<grid, kK1Threads, kK1SmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
@@ -170,15 +190,8 @@ inline cudaError_t launch_after_predecessor(void (*fn)(KArgs...), int grid, int 
 
 // Key splits of stage 2: with few (head, feature tile) pairs the keys are divided over up to four
 // CTAs per pair, as long as all of them fit on the machine at once.
-inline int k2_nsplit(bool performer, int BH, int k, int p) {
+inline int k2_nsplit(int sms, bool performer, int BH, int k, int p) {
   if (!performer) return 1;
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
-  }
   const int units = BH * ((p + 127) / 128);
   const int chunks = (k + kK2Chunk - 1) / kK2Chunk;
   int ns = sms / units;
@@ -198,9 +211,10 @@ inline size_t k2_part_floats(bool performer, int BH, int d, int k, int p) {
 }
 
 // ---- stage 2: per-feature summaries a (fp16, transposed) and weights b / z from K', V' --------
-inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const void* W, float* weight,
+inline int launch_k2(TensorContext& tc, bool performer, const float* kpvp, const void* W, float* weight,
                      __half* aT16, float* part, int* counters, int BH, int d, int k, int p, int* status,
                      cudaStream_t st, int* cuda_err) {
+  TensorMaps& tm = tc.maps;
   if (performer) {
     const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
     const unsigned bW[2] = {64, 128};
@@ -216,8 +230,7 @@ inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const vo
   prm.weight = weight;
   prm.aT16 = aT16;
   prm.status = status;
-  prm.trace = nullptr;
-  prm.nsplit = (part && counters) ? k2_nsplit(performer, BH, k, p) : 1;
+  prm.nsplit = (part && counters) ? k2_nsplit(tc.sm_total(), performer, BH, k, p) : 1;
   prm.part = part;
   prm.counters = counters;
   auto fn = performer ? k2_key_side<true> : k2_key_side<false>;
@@ -233,9 +246,10 @@ inline int launch_k2(TensorMaps& tm, bool performer, const float* kpvp, const vo
 }
 
 // ---- stage 3: O from Q, W and the key-side summaries ------------------------------------------
-inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* W, const __half* aT16,
+inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const void* W, const __half* aT16,
                      const float* weight, void* out, int BH, int H, int N, int d, int p, int* status, cudaStream_t st,
                      int* cuda_err) {
+  TensorMaps& tm = tc.maps;
   const unsigned long long dQ[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
                                     (unsigned long long)(H > 0 ? BH / H : BH)};
   const unsigned bQ[3] = {64, 128, 1};
@@ -261,12 +275,11 @@ inline int launch_k3(TensorMaps& tm, bool performer, const void* Q, const void* 
   prm.weight = weight;
   prm.out = reinterpret_cast<__nv_bfloat16*>(out);
   prm.status = status;
-  prm.trace = nullptr;
   const K3Smem L = k3_smem_plan(d, p, performer);
   auto fn = performer ? k3_query_side<true> : k3_query_side<false>;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
-  int grid = sm_count();
+  int grid = tc.sm_count();
   if (grid > prm.total_tiles) grid = prm.total_tiles;
   // the RNN kernel ignores tmW; pass any valid map
   e = launch_after_predecessor(fn, grid, kK3Threads, L.total, st, tm.Q.map, performer ? tm.W.map : tm.Q.map,

@@ -37,17 +37,33 @@ def compare(got, ref, io):
     return rel, mx
 
 
+def bf16_half_ulp(ref):
+    """Half a unit in the last place of bfloat16 at each |ref| (8 significand bits): what rounding the
+    exact value to bfloat16 can cost by itself."""
+    a = np.maximum(np.abs(np.asarray(ref, dtype=np.float64)), 2.0 ** -126)
+    return 2.0 ** (np.floor(np.log2(a)) - 8)
+
+
 def assert_close(got, ref, io, what=""):
+    """The parity gate.  bf16: rel-Frobenius <= 1e-2 and max-abs <= 5e-2, element by element.  Only an
+    element whose own bfloat16 rounding can already cost more than 5e-2 (|ref| >= 16: half an ulp is
+    0.0625) gets half an ulp + 2.5e-2 instead; such elements are counted and printed."""
     rel, mx = compare(got, ref, io)
     if io == "fp32":
         assert rel <= FP32_REL, "%s: rel-Fro %.3e > %.1e (max-abs %.3e)" % (what, rel, FP32_REL, mx)
     else:
-        floor = bf16_floor(ref)
         assert rel <= BF16_REL_FRO, "%s: rel-Fro %.3e > %.1e" % (what, rel, BF16_REL_FRO)
-        # The output's own bf16 rounding (half an ulp: 0.031 for |O| in [8,16), 0.0625 in [16,32)) is
-        # part of any bf16 result; the bound applies on top of what exceeds 5e-2 by rounding alone.
-        bound = max(BF16_MAX_ABS, floor + 0.5 * BF16_MAX_ABS)
-        assert mx <= bound, "%s: max-abs %.3e > %.3e (bf16 rounding floor %.3e)" % (what, mx, bound, floor)
+        diff = np.abs(np.asarray(got, dtype=np.float64) - ref)
+        half_ulp = bf16_half_ulp(ref)
+        wide = half_ulp >= BF16_MAX_ABS
+        bound = np.where(wide, half_ulp + 0.5 * BF16_MAX_ABS, BF16_MAX_ABS)
+        bad = diff > bound
+        assert not bad.any(), "%s: max-abs %.3e > %.1e at %d elements (worst excess %.3e; %d elements on the widened bound)" % (
+            what, mx, BF16_MAX_ABS, int(bad.sum()), float((diff - bound).max()), int(wide.sum()))
+        if wide.any():
+            print("%s: %d of %d elements have |ref| >= 16 (bf16 half-ulp 0.0625 > 5e-2) and use half-ulp + 2.5e-2; "
+                  "max-abs over the others %.3e" % (what, int(wide.sum()), wide.size,
+                                                    float(diff[~wide].max()) if (~wide).any() else 0.0))
     return rel, mx
 
 

@@ -30,7 +30,9 @@ def _check_full(w, heads, n_rows, seed=0):
     assert binding.flurka_last_status() == 0
     assert binding.flurka_last_path() == binding.PATH_TENSOR
     assert binding.flurka_last_launches() == 3
-    # convexity over the whole output, against the library's own fp32 V'
+    # convexity over the whole output, against the library's fp32 V' (itself compared with the oracle's
+    # for every sampled head below)
+    Kp = binding.flurka_debug_copy(0, (w.B, w.H, w.k, w.d))
     Vp = binding.flurka_debug_copy(1, (w.B, w.H, w.k, w.d))
     torch.cuda.synchronize()
     lo = Vp.min(dim=2, keepdim=True).values
@@ -44,7 +46,11 @@ def _check_full(w, heads, n_rows, seed=0):
     for (b, h) in heads:
         rows = np.sort(rng.choice(w.N, size=n_rows, replace=False))
         rows[0], rows[-1] = 0, w.N - 1                                    # first and last row of the head
-        ref = pu.oracle_head(inputs, w, b, h, rows=rows)
+        ref, inter = pu.oracle_head(inputs, w, b, h, rows=rows, intermediates=True)
+        # the full-size projections K' = E K, V' = F V of this head, element by element
+        for mine, theirs, nm in ((Kp[b, h], inter["Kp"], "K'"), (Vp[b, h], inter["Vp"], "V'")):
+            err = np.abs(mine.cpu().double().numpy() - theirs).max()
+            assert err < 3e-5 * max(1.0, np.abs(theirs).max()), "%s %s head (%d,%d): %.3e" % (w.name, nm, b, h, err)
         got = out[b, h].cpu()[torch.from_numpy(rows)].double().numpy()
         rel, mx = pu.assert_close(got, ref, w.io, "%s head (%d,%d)" % (w.name, b, h))
         worst = (max(worst[0], rel), max(worst[1], mx))
@@ -60,7 +66,7 @@ def test_c3_full_size():
 
 
 def test_c4_full_size():
-    _check_full(configs.C4, heads=[(0, 5)], n_rows=384)
+    _check_full(configs.C4, heads=[(0, 0), (0, 5), (0, 7)], n_rows=384)
 
 
 @pytest.mark.parametrize("k,m", configs.C5_GRID, ids=lambda v: str(v))

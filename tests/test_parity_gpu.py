@@ -113,6 +113,28 @@ def test_host_entry_point_in_head_groups(variant, H):
             pu.assert_close(got[b, h], pu.oracle_head(inputs, w, b, h), "bf16", "host entry point, head (%d,%d)" % (b, h))
 
 
+@pytest.mark.parametrize("variant,heads", [(PERFORMER, 12), (PERFORMER, 10), (RNN, 12)])
+def test_host_entry_point_with_unequal_head_groups(variant, heads):
+    """1 MiB of Q per head, so the host entry point takes 12 (10) heads in eight groups of 1 and 2 heads:
+    the workspace layout differs from group to group.  PERFORMER with k = 256 and so few heads per group
+    also splits the keys of stage 2 over two CTAs, whose arrival counters live next to the status words."""
+    w = _wl("host_uneven_groups", variant, "bf16", 1, heads, 8192, 64, 256, 256, 43 + heads)
+    inputs = synth.make_inputs(w)
+    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in inputs.items()}
+    # a small problem first, so that the library-owned workspace has to grow inside the big call
+    small = _wl("host_uneven_small", variant, "bf16", 1, 1, 256, 64, 64, 64, 44)
+    pu.run_gpu(small, synth.make_inputs(small))
+    for _ in range(2):
+        host_out = binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"],
+                                               pinned["W"], w.variant)
+        assert binding.flurka_last_status() == 0
+        assert binding.flurka_last_path() == binding.PATH_TENSOR
+    got = host_out.double().numpy()
+    assert np.isfinite(got).all()
+    for h in range(w.H):
+        pu.assert_close(got[0, h], pu.oracle_head(inputs, w, 0, h), "bf16", "host entry point, head %d of %d" % (h, heads))
+
+
 def test_caller_workspace_and_too_small_workspace():
     w = _wl("ws_rnn_bf16", RNN, "bf16", 1, 2, 256, 64, 64, 0, 51)
     inputs = synth.make_inputs(w)

@@ -57,6 +57,30 @@ def test_static_scratch_matches_forward_on_two_calls_in_a_row():
 
 
 @pytest.mark.gpu
+def test_static_scratch_leaves_the_stage_timing_of_flurka_forward_alone():
+    w = Workload("noalloc_timing", PERFORMER, "fp32", 1, 2, 256, 32, 32, 64, 905)
+    x = synth.make_inputs(w)
+    dev = pu.to_device(x)
+    out = torch.empty_like(dev["Q"])
+    binding.flurka_set_stage_timing(True)
+    try:
+        # with timing on but no flurka_forward yet, there is nothing to report, before and after
+        with pytest.raises(binding.FlurkaError):
+            binding.flurka_last_stage_ms()
+        binding.flurka_forward_static_scratch(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant, out)
+        torch.cuda.synchronize()
+        with pytest.raises(binding.FlurkaError):
+            binding.flurka_last_stage_ms()
+        binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant)
+        first = binding.flurka_last_stage_ms()
+        binding.flurka_forward_static_scratch(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant, out)
+        torch.cuda.synchronize()
+        assert binding.flurka_last_stage_ms() == first
+    finally:
+        binding.flurka_set_stage_timing(False)
+
+
+@pytest.mark.gpu
 def test_static_scratch_same_problem_twice_is_stable():
     w = Workload("noalloc_repeat", PERFORMER, "fp32", 1, 2, 256, 32, 32, 64, 904)
     x = synth.make_inputs(w)
@@ -79,8 +103,13 @@ def test_static_scratch_refuses_oversized_problems_without_a_device():
     # addresses that are never dereferenced: every check that can refuse runs before any access
     q, k, v, e, f, w, o = ((1 << 40) + (i << 34) for i in range(7))
     big = configs.C3
-    assert lib.flurka_workspace_bytes(0, big.B, big.H, big.N, big.d, big.k, big.m) > binding.STATIC_SCRATCH_BYTES
+    assert lib.flurka_static_scratch_need(0, big.B, big.H, big.N, big.d, big.k, big.m) > binding.STATIC_SCRATCH_BYTES
     rc = lib.flurka_forward_static_scratch(q, k, v, e, f, w, 0, big.B, big.H, big.N, big.d, big.k, big.m, o, None)
     assert rc == -9
+    # the threshold is the size query's: the largest head count that still fits is accepted as far as
+    # the device check (-7 without a GPU, 0 with one is not tried here: the addresses are fake), one more is refused
+    fits = max(h for h in range(1, 400) if lib.flurka_static_scratch_need(1, 1, h, 512, 64, 64, 0) <= binding.STATIC_SCRATCH_BYTES)
+    assert lib.flurka_static_scratch_need(1, 1, fits, 512, 64, 64, 0) <= lib.flurka_workspace_bytes(1, 1, fits, 512, 64, 64, 0)
+    assert lib.flurka_forward_static_scratch(q, k, v, e, f, None, 1, 1, fits + 1, 512, 64, 64, 0, o, None) == -9
     assert b"scratch" in lib.flurka_strerror(-9)
     assert lib.flurka_forward_static_scratch(None, k, v, e, f, w, 0, 1, 1, 8, 8, 4, 8, o, None) == -1
