@@ -180,44 +180,11 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", default="c3")
-    ap.add_argument("--impl", default="flurka", choices=["flurka", "reference"])
-    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--heads", default="", help="B,H override: a smaller batch of the same workload (profiling)")
-    ap.add_argument("--no-load", action="store_true", help="skip the sustained-load phase before timing (profiling)")
-    ap.add_argument("--layout", default="bhnd", choices=["bhnd", "bnhd"],
-                    help="Q, K, V, out as [B,H,N,d] (default) or [B,N,H,d]")
-    args = ap.parse_args()
-    w = configs.get(args.config)
-    if args.heads:
-        b, h = (int(x) for x in args.heads.split(","))
-        w = configs.shrink(w, name="%s_B%d_H%d" % (w.name, b, h), B=b, H=h)
-
-    if args.impl == "reference":
-        run_reference(args, w)
-        return
-
-    from paper_2306_15799_b200 import binding, build
-
-    rank, world, local = dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
-    torch.cuda.set_device(local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank == 0:
-        build.build()
-    if world > 1:
-        dist.barrier()
-    binding.load()
-    binding.flurka_set_path({"auto": binding.PATH_AUTO, "simt": binding.PATH_SIMT, "tensor": binding.PATH_TENSOR}[args.path])
+def measure(w, args, binding, rank, world, local, with_e2e=True):
+    """Times `args.steps` forward passes of workload `w` on this rank's GPU: CUDA events on the launch
+    stream around every step, a second pass with the library's per-stage events, the clocks sampled
+    meanwhile, and (optionally) the host-buffer entry point end to end."""
+    import torch.distributed as dist
 
     # every rank draws its own batch (weak scaling over B*H); same recipe, rank-offset seed
     wr = rank_workload(w, rank)
@@ -229,7 +196,6 @@ def main():
     pinned = {n: (t.pin_memory() if t is not None else None) for n, t in laid_out.items()}
     dev = {n: (t.cuda(non_blocking=True) if t is not None else None) for n, t in pinned.items()}
     out = torch.empty_like(dev["Q"])
-    host_out = torch.empty_like(pinned["Q"]).pin_memory()
     in_bytes = sum(t.numel() * t.element_size() for t in dev.values() if t is not None)
     flush = None
     if in_bytes < 2 * L2_BYTES:
@@ -273,9 +239,10 @@ def main():
             stops[i].record(stream)
     barrier()
     step_ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
-    total_ms = sum(step_ms)
-    launches = binding.flurka_last_launches() * args.steps
-    path_taken = {1: "simt", 2: "tensor"}.get(binding.flurka_last_path(), "?")
+    res = {"step_ms": step_ms, "total_ms": sum(step_ms), "in_bytes": in_bytes,
+           "out_bytes": out.numel() * out.element_size(), "flushed": flush is not None,
+           "launches": binding.flurka_last_launches() * args.steps,
+           "path": {1: "simt", 2: "tensor"}.get(binding.flurka_last_path(), "?")}
 
     # ---- per-stage durations (same inputs, events inside the library between the stages)
     binding.flurka_set_stage_timing(True)
@@ -288,76 +255,148 @@ def main():
             ms3 = binding.flurka_last_stage_ms()
             stage_ms = [a + b for a, b in zip(stage_ms, ms3)]
     binding.flurka_set_stage_timing(False)
-    stage_ms = [x / args.steps for x in stage_ms]
+    res["stage_ms"] = [x / args.steps for x in stage_ms]
     torch.cuda.synchronize()
-    clocks = sampler.stop()
+    res["clocks"] = sampler.stop()
 
     # ---- end to end: host buffers in, host buffer out, through the host entry point
-    e2e_steps = max(1, min(args.steps, 5))
-    binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
-                                w.variant, out=host_out, stream=stream, layout=args.layout)
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
+    res["e2e_ms"] = None
+    if with_e2e:
+        host_out = torch.empty_like(pinned["Q"]).pin_memory()
+        e2e_steps = max(1, min(args.steps, 5))
         binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
                                     w.variant, out=host_out, stream=stream, layout=args.layout)
-    torch.cuda.synchronize()
-    e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
-    status = binding.flurka_last_status()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
+                                        w.variant, out=host_out, stream=stream, layout=args.layout)
+        torch.cuda.synchronize()
+        res["e2e_ms"] = 1e3 * (time.perf_counter() - t0) / e2e_steps
+    res["status"] = binding.flurka_last_status()
+    res["host_inputs"] = (wr, host)
+    return res
 
-    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], world, device="cuda")
+
+def stage_work(w):
+    """Algorithmic FLOPs, bytes and exponentials of the three stages (all heads), and their names."""
+    N, d, k, m, BH, s = w.N, w.d, w.k, w.m, w.B * w.H, w.elem_bytes
+    perf = w.variant == configs.PERFORMER
+    p = m if perf else d
+    flops = [4 * N * k * d * BH,
+             (2 * k * d * m + 2 * k * m * d) * BH if perf else 2 * k * d * d * BH,
+             (2 * N * d * m + 2 * N * m * d) * BH if perf else 2 * N * d * d * BH]
+    byts = [2 * BH * N * d * s + 2 * k * N * s + 2 * BH * k * d * 4,
+            2 * BH * k * d * 4 + m * d * s + BH * p * (d * 2 + 4),
+            2 * BH * N * d * s + m * d * s + BH * p * (d * 2 + 4)]
+    exps = [0, k * p * BH, N * p * BH]
+    return ["down_projection", "key_side", "query_side"], flops, byts, exps
+
+
+def rooflines(w, res, peaks, steps, world, exp_rate):
+    """The `roofline` object (dominant kernel) and the `path_roofline` object (whole forward) of a run.
+
+    Both follow one definition: time at the roofline = max(FLOPs / measured dense bf16 peak, bytes / measured
+    HBM bandwidth); frac = that time / measured time.  The GEMM denominator is the burst figure; the fraction
+    against the seconds-long (power-capped) figure is given beside it."""
+    ms_per_step = res["total_ms"] / steps
+    names, sflops, sbytes, sexps = stage_work(w)
+    stage_ms = res["stage_ms"]
+    dom = max(range(3), key=lambda i: stage_ms[i])
+    dt = stage_ms[dom] * 1e-3
+    tf, tf_s, hbm = peaks["bf16_tflops"] * 1e12, peaks["bf16_tflops_sustained"] * 1e12, peaks["hbm_gbs"] * 1e9
+    t_tensor, t_hbm = sflops[dom] / tf, sbytes[dom] / hbm
+    if t_hbm >= t_tensor:
+        roofline = {"bound": "hbm", "achieved": sbytes[dom] / dt / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roofline = {"bound": "tensor", "achieved": sflops[dom] / dt / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+    roofline["frac"] = max(t_tensor, t_hbm) / dt
+    roofline["frac_sustained"] = max(sflops[dom] / tf_s, t_hbm) / dt
+    roofline["frac_tensor"] = t_tensor / dt
+    roofline["frac_hbm"] = t_hbm / dt
+    roofline["traffic"] = recorded_traffic(names[dom], w)
+    roofline["kernel"] = names[dom]
+    roofline["peak_source"] = "of " + peaks["source"] + " (burst GEMM figure)"
+    roofline["stage_ms"] = dict(zip(names, stage_ms))
+    if sexps[dom] and exp_rate:
+        # a third limit the FLOP / byte roofline does not count: the exponentials of this stage against the
+        # rate a loop of nothing but independent ex2.approx chains reaches on this GPU (measured in this run)
+        roofline["exp"] = {"achieved_gexp_s": sexps[dom] / dt / 1e9, "measured_peak_gexp_s": exp_rate,
+                           "frac": sexps[dom] / dt / 1e9 / exp_rate}
+    flops, byts = w.flops(), w.compulsory_bytes()
+    t_t, t_h = flops / tf, byts / hbm
+    path = {"flops": flops, "bytes": byts, "t_tensor_us": t_t * 1e6, "t_hbm_us": t_h * 1e6,
+            "frac": max(t_t, t_h) / (ms_per_step * 1e-3),
+            "frac_sustained": max(flops / tf_s, t_h) / (ms_per_step * 1e-3),
+            "tensor_peak_tflops": peaks["bf16_tflops"], "peak_source": "of " + peaks["source"] + " (burst GEMM figure)"}
+    return roofline, path
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="", help="workload (default: c3, followed by a c4 block under `also`)")
+    ap.add_argument("--impl", default="flurka", choices=["flurka", "reference"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-also", action="store_true", help="default run: skip the second target configuration (c4)")
+    ap.add_argument("--heads", default="", help="B,H override: a smaller batch of the same workload (profiling)")
+    ap.add_argument("--no-load", action="store_true", help="skip the sustained-load phase before timing (profiling)")
+    ap.add_argument("--layout", default="bhnd", choices=["bhnd", "bnhd"],
+                    help="Q, K, V, out as [B,H,N,d] (default) or [B,N,H,d]")
+    args = ap.parse_args()
+    default_run = args.config == ""
+    w = configs.get(args.config or "c3")
+    if args.heads:
+        b, h = (int(x) for x in args.heads.split(","))
+        w = configs.shrink(w, name="%s_B%d_H%d" % (w.name, b, h), B=b, H=h)
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2306_15799_b200 import binding, build
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    binding.load()
+    binding.flurka_set_path({"auto": binding.PATH_AUTO, "simt": binding.PATH_SIMT, "tensor": binding.PATH_TENSOR}[args.path])
+
+    res = measure(w, args, binding, rank, world, local)
+    total_ms, e2e_ms = max_over_ranks([res["total_ms"], res["e2e_ms"]], world, device="cuda")
+    res["total_ms"] = total_ms
     ms_per_step = total_ms / args.steps
+    wr, host = res.pop("host_inputs")
+
+    also = None
+    if default_run and not args.no_also and not args.heads:
+        # the second configuration the roofline target is stated on, timed the same way (no end-to-end
+        # leg, no oracle leg); every rank runs it, the slowest one counts
+        w4 = configs.get("c4")
+        r4 = measure(w4, args, binding, rank, world, local, with_e2e=False)
+        r4.pop("host_inputs")
+        r4["total_ms"] = max_over_ranks([r4["total_ms"]], world, device="cuda")[0]
+        also = (w4, r4)
 
     if rank == 0:
         peaks = measured_peaks()
+        exp_rate = binding.flurka_measure_ex2_rate()          # Gexp/s of a bare ex2.approx loop on this GPU, now
         tokens = w.tokens * world
         value = job_tokens_per_s(w, world, ms_per_step)
-        flops, byts = w.flops(), w.compulsory_bytes()
-        # The steps are timed after a 0.6 s load phase, i.e. inside a long power-capped loop, so the
-        # GEMM denominator is the seconds-long figure; with --no-load it is the burst figure.  The
-        # fraction against the other one is reported next to it.
-        sustained = not args.no_load
-        tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-        tf_other = peaks["bf16_tflops"] if sustained else peaks["bf16_tflops_sustained"]
-        other_key = "frac_burst" if sustained else "frac_sustained"
-        t_tensor = flops / (tf_peak * 1e12)
-        t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
-        roof_s = max(t_tensor, t_hbm)
-        # dominant stage and its own roofline (algorithmic work of that stage alone)
-        N, d, k, m, BH, s = w.N, w.d, w.k, w.m, w.B * w.H, w.elem_bytes
-        p = m if w.variant == configs.PERFORMER else d
-        stage_flops = [4 * N * k * d * BH,
-                       (2 * k * d * m + 2 * k * m * d) * BH if w.variant == configs.PERFORMER else 2 * k * d * d * BH,
-                       (2 * N * d * m + 2 * N * m * d) * BH if w.variant == configs.PERFORMER else 2 * N * d * d * BH]
-        stage_bytes = [2 * BH * N * d * s + 2 * k * N * s + 2 * BH * k * d * 4,
-                       2 * BH * k * d * 4 + m * d * s + BH * p * (d * 2 + 4),
-                       2 * BH * N * d * s + m * d * s + BH * p * (d * 2 + 4)]
-        # exponentials go through the special-function unit: 16 per clock per SM, 148 SMs, at the
-        # maximum SM clock (nominal unit count x clock; there is no measured figure for this unit)
-        stage_exps = [0, k * p * BH, N * p * BH]
-        exp_peak = 16.0 * 148 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6      # 1965 MHz: the B200's maximum SM clock
-        names = ["down_projection", "key_side", "query_side"]
-        dom = max(range(3), key=lambda i: stage_ms[i])
-        dt = stage_ms[dom] * 1e-3
-        tf_t = stage_flops[dom] / (tf_peak * 1e12)
-        hb_t = stage_bytes[dom] / (peaks["hbm_gbs"] * 1e9)
-        ex_t = stage_exps[dom] / exp_peak
-        if ex_t >= max(hb_t, tf_t):
-            roofline = {"bound": "alu", "achieved": stage_exps[dom] / dt / 1e9, "peak": exp_peak / 1e9, "unit": "Gexp/s",
-                        "frac_tensor": stage_flops[dom] / dt / 1e12 / tf_peak,
-                        "frac_hbm": stage_bytes[dom] / dt / 1e9 / peaks["hbm_gbs"]}
-        elif hb_t >= tf_t:
-            roofline = {"bound": "hbm", "achieved": stage_bytes[dom] / dt / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-        else:
-            roofline = {"bound": "tensor", "achieved": stage_flops[dom] / dt / 1e12, "peak": tf_peak, "unit": "TFLOP/s"}
-        roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        if roofline["bound"] == "tensor":
-            roofline[other_key] = roofline["achieved"] / tf_other
-        roofline["traffic"] = recorded_traffic(names[dom], w)
-        roofline["kernel"] = names[dom]
-        roofline["peak_source"] = "nominal: 16 exp/clk/SM x 148 SMs x max SM clock" if roofline["bound"] == "alu" else "of " + peaks["source"] + (
-            " (sustained GEMM figure: timed inside a long loop)" if sustained and roofline["bound"] == "tensor" else "")
-        roofline["stage_ms"] = dict(zip(names, stage_ms))
+        roofline, path_roofline = rooflines(w, res, peaks, args.steps, world, exp_rate)
+        clocks = res["clocks"]
+        step_ms = res["step_ms"]
 
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -365,23 +404,33 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.io == "bf16" else "f32",
             "data": "synthetic",
             "config": {"workload": w.name, "variant": "performer" if w.variant == configs.PERFORMER else "rnn",
-                       "B": w.B, "H": w.H, "N": w.N, "d": w.d, "k": w.k, "m": w.m, "io": w.io, "path": path_taken,
+                       "B": w.B, "H": w.H, "N": w.N, "d": w.d, "k": w.k, "m": w.m, "io": w.io, "path": res["path"],
                        "layout": args.layout,
                        "parallelism": "replicated batches over B*H, no collective" if world > 1 else "single GPU",
-                       "l2": "inputs (%.0f MB) exceed L2" % (in_bytes / 1e6) if flush is None
+                       "l2": "inputs (%.0f MB) exceed L2" % (res["in_bytes"] / 1e6) if not res["flushed"]
                              else "L2 flushed between steps (252 MiB write)"},
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"]},
             "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": out.numel() * out.element_size()},
-            "gpu_launches": launches,
+                    "h2d_bytes_per_step": res["in_bytes"], "d2h_bytes_per_step": res["out_bytes"]},
+            "gpu_launches": res["launches"],
             "roofline": roofline,
-            "path_roofline": {"flops": flops, "bytes": byts, "t_tensor_us": t_tensor * 1e6, "t_hbm_us": t_hbm * 1e6,
-                              "frac": roof_s / (ms_per_step * 1e-3),
-                              other_key: max(flops / (tf_other * 1e12), t_hbm) / (ms_per_step * 1e-3),
-                              "tensor_peak_tflops": tf_peak, "peak_source": "of " + peaks["source"]},
+            "path_roofline": path_roofline,
             "step_ms_min": min(step_ms), "step_ms_median": statistics.median(step_ms),
-            "device_status": status,
+            "device_status": res["status"],
         }
+        if also is not None:
+            w4, r4 = also
+            rf4, pr4 = rooflines(w4, r4, peaks, args.steps, world, exp_rate)
+            ms4 = r4["total_ms"] / args.steps
+            line["also"] = {w4.name: {
+                "value": job_tokens_per_s(w4, world, ms4), "unit": UNIT, "ms_per_step": ms4,
+                "step_ms_min": min(r4["step_ms"]), "step_ms_median": statistics.median(r4["step_ms"]),
+                "config": {"workload": w4.name, "variant": "performer", "B": w4.B, "H": w4.H, "N": w4.N, "d": w4.d,
+                           "k": w4.k, "m": w4.m, "io": w4.io, "path": r4["path"], "layout": args.layout,
+                           "l2": "inputs (%.0f MB) exceed L2" % (r4["in_bytes"] / 1e6)},
+                "clocks": {"sm_mhz": r4["clocks"]["sm_mhz"], "sm_max_mhz": r4["clocks"]["sm_max_mhz"],
+                           "reasons": r4["clocks"]["reasons"]},
+                "gpu_launches": r4["launches"], "roofline": rf4, "path_roofline": pr4, "device_status": r4["status"]}}
         if not args.no_cpu_baseline and world == 1:
             import oracle
             oracle.build()
@@ -393,6 +442,7 @@ def main():
                                     "sample": "%d head passes over the %d heads of %s, all %d rows each, %.1f s" % (heads, w.B * w.H, w.name, w.N, tt)}
         print(json.dumps(line), flush=True)
     if world > 1:
+        import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
 

@@ -158,6 +158,15 @@ int flurka_last_cuda_error(void);
 int flurka_set_stage_timing(int on);
 int flurka_last_stage_ms(float* ms3);
 
+/*
+ * Measurement aid for the roofline of the query side, whose N * m exponentials per head (the feature
+ * map phi(Q) of Section 2.1) go through the special-function unit, a limit that FLOP and byte counts
+ * do not show.  Runs a kernel of nothing but independent ex2.approx chains on every SM of the current
+ * device (default stream, a few milliseconds, synchronises) and writes the rate it reached, in 1e9
+ * exponentials per second, to the HOST double `gexp_per_s`.
+ */
+int flurka_measure_ex2_rate(double* gexp_per_s);
+
 /* Static, human-readable text for a flurka_status. */
 const char* flurka_strerror(int code);
 

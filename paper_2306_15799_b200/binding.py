@@ -21,6 +21,7 @@ EXPORTS = [
     "flurka_set_path", "flurka_set_cta_limit", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
     "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
     "flurka_strerror", "flurka_version", "flurka_forward_static_scratch", "flurka_static_scratch_need",
+    "flurka_measure_ex2_rate",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -82,6 +83,8 @@ def load() -> ctypes.CDLL:
     lib.flurka_strerror.restype = ctypes.c_char_p
     lib.flurka_strerror.argtypes = [ci]
     lib.flurka_version.restype = ci
+    lib.flurka_measure_ex2_rate.restype = ci
+    lib.flurka_measure_ex2_rate.argtypes = [ctypes.POINTER(ctypes.c_double)]
     _lib = lib
     return lib
 
@@ -230,6 +233,15 @@ def flurka_last_stage_ms():
     if rc:
         raise FlurkaError(rc, "flurka_last_stage_ms")
     return [float(x) for x in ms]
+
+
+def flurka_measure_ex2_rate() -> float:
+    """1e9 exponentials per second a bare ex2.approx loop reaches on the current GPU (synchronises)."""
+    v = ctypes.c_double(0.0)
+    rc = load().flurka_measure_ex2_rate(ctypes.byref(v))
+    if rc:
+        raise FlurkaError(rc, "flurka_measure_ex2_rate")
+    return float(v.value)
 
 
 def flurka_forward_static_scratch(Q, K, V, E, F, W, variant, out, stream=None):

@@ -572,6 +572,58 @@ const char* flurka_strerror(int code) {
 
 int flurka_version(void) { return FLURKA_VERSION; }
 
+// A loop of nothing but exponentials: eight independent ex2.approx chains per thread, every SM full.
+namespace {
+__global__ void ex2_rate_kernel(int iters, float* sink) {
+  float x[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) x[c] = -0.001f * (float)(threadIdx.x + c + 1);
+  for (int i = 0; i < iters; ++i) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) asm volatile("ex2.approx.ftz.f32 %0, %0;" : "+f"(x[c]));
+  }
+  float acc = 0.f;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) acc += x[c];
+  if (acc == -1.f) sink[0] = acc;       // never true (2^x > 0): keeps the chains alive
+}
+}  // namespace
+
+int flurka_measure_ex2_rate(double* gexp_per_s) {
+  if (!gexp_per_s) return FLURKA_ERR_NULL;
+  int rc = check_device();
+  if (rc) return rc;
+  DeviceState& ds = dev_state();
+  const int blocks = ds.tc.sm_total() * 8, threads = 256, iters = 4096;
+  float* sink = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaMalloc(&sink, sizeof(float));
+  if (e != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaEventCreate(&e0)) != cudaSuccess || (e = cudaEventCreate(&e1)) != cudaSuccess) {
+    cudaFree(sink);
+    if (e0) cudaEventDestroy(e0);
+    return cuda_fail(e);
+  }
+  float best_ms = 0.f;
+  for (int rep = 0; rep < 4; ++rep) {               // the first launch warms up
+    cudaEventRecord(e0, 0);
+    ex2_rate_kernel<<<blocks, threads>>>(iters, sink);
+    cudaEventRecord(e1, 0);
+    e = cudaEventSynchronize(e1);
+    if (e != cudaSuccess) break;
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && (best_ms == 0.f || ms < best_ms)) best_ms = ms;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaFree(sink);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (best_ms <= 0.f) return FLURKA_ERR_CUDA;
+  *gexp_per_s = (double)blocks * threads * 8.0 * iters / (best_ms * 1e-3) / 1e9;
+  return FLURKA_OK;
+}
+
 size_t flurka_static_scratch_need(int variant, int B, int H, int N, int d, int k, int m) {
   Problem pr;
   if (parse_problem(variant, B, H, N, d, k, m, &pr)) return 0;

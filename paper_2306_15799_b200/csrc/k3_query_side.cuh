@@ -11,12 +11,14 @@
 // The per-feature summaries a_i, b_i (or z_i) come from stage 2.  A persistent CTA walks a
 // contiguous range of 128-row tiles; warp 0 feeds Q tiles by TMA, warps 1 and 3 issue the first and the second
 // products, warp 2 reloads a^T and rebuilds the bias operand when the head changes, and two groups of four warps
-// alternate tiles.  TMEM holds S/p and O of the tiles in flight: two 256-column buffers (S/p in
-// columns 0.., O in columns 128..) in general; four 128-column buffers (S/p in columns 0.., O in
-// columns 64.., which S has vacated by then) when d = 64 and p <= 128.  With four buffers each group
-// has two tiles in flight and reads tile i-2 out after it has handed tile i to the second product,
-// so it never waits for a product it has just asked for.  Every thread of a group owns one output
-// row and writes it with 32-byte stores.
+// alternate tiles.  TMEM holds S/p and O of the tiles in flight: two 256-column buffers in general, four
+// 128-column buffers when d = 64 and p <= 128.  p overwrites S at half the width, block by block of 64
+// features, and the row owners hand every finished block to the second product.  With d = 64, O sits in
+// columns 64..127 of its buffer, which pass 2 has consumed after the first 128 features (blocks 2 and 3 of
+// p go to columns 128.. instead), so at m = 256 the second product of a tile runs under the second half
+// of its pass 2 and only its last block is left when the row owners start waiting for O.  With four
+// buffers each group has two tiles in flight and reads tile i-2 out after it has handed tile i to the
+// second product.  Every thread of a group owns one output row and writes it with 32-byte stores.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -63,7 +65,7 @@ __host__ __device__ inline K3Smem k3_smem_plan(int d, int p, bool performer) {
   s.q_stages = (d == 64) ? 4 : 2;
   s.q = off;    off += (uint32_t)s.q_stages * 128 * d * 2;
   s.scale = off; off += 1024;                                      // RNN: z_i / max z as floats
-  s.bars = off; off += 256;
+  s.bars = off; off += 512;
   s.total = off + 1024;                                            // alignment slack
   return s;
 }
@@ -86,14 +88,14 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const uint32_t bar_qfull = bars;            // [4]   Q tile landed
   const uint32_t bar_qempty = bars + 32;      // [4]   Q tile consumed (MMA commit, or 128 readers for RNN)
   const uint32_t bar_sfull = bars + 64;       // [4]   S ready in TMEM (PERFORMER)
-  const uint32_t bar_pfull = bars + 96;       // [4]   p written to TMEM by the 128 row owners
-  const uint32_t bar_ofull = bars + 128;      // [4]   O ready in TMEM
-  const uint32_t bar_sfree = bars + 160;      // [4]   TMEM buffer read out, may be overwritten
-  const uint32_t bar_wfull = bars + 192;      //       W resident
-  const uint32_t bar_drained = bars + 200;    //       every MMA of the previous head is complete
-  const uint32_t bar_atfull = bars + 208;     //       a^T of the new head resident
-  const uint32_t bar_biasready = bars + 216;  //       bias operand / scale vector of the new head built
-  const uint32_t tmem_slot = bars + 232;
+  const uint32_t bar_ofull = bars + 96;       // [4]   O ready in TMEM
+  const uint32_t bar_sfree = bars + 128;      // [4]   TMEM buffer read out, may be overwritten
+  const uint32_t bar_pfull = bars + 160;      // [4][4] a block of 64 features of p written to TMEM by the 128 row owners
+  const uint32_t bar_wfull = bars + 288;      //       W resident
+  const uint32_t bar_drained = bars + 296;    //       every MMA of the previous head is complete
+  const uint32_t bar_atfull = bars + 304;     //       a^T of the new head resident
+  const uint32_t bar_biasready = bars + 312;  //       bias operand / scale vector of the new head built
+  const uint32_t tmem_slot = bars + 320;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
 
@@ -112,7 +114,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
     }
     for (int i = 0; i < 4; ++i) {
       mbar_init(bar_sfull + 8 * i, 1);
-      mbar_init(bar_pfull + 8 * i, 128);
+      for (int q = 0; q < 4; ++q) mbar_init(bar_pfull + 8 * (4 * i + q), 128);
       mbar_init(bar_ofull + 8 * i, 1);
       mbar_init(bar_sfree + 8 * i, 128);
     }
@@ -154,7 +156,15 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const int NB = (d == 64 && p <= 128) ? 4 : 2;
   const int nb_shift = NB == 4 ? 2 : 1;
   const uint32_t buf_cols = 512u / NB;
-  const uint32_t o_col = NB == 4 ? 64u : 128u;
+  const uint32_t o_col = d == 64 ? 64u : 128u;
+  // O occupies columns [o_col, o_col + d) of the buffer.  Where that range overlaps S (PERFORMER), the
+  // second product may start only when pass 2 has consumed those columns: q_first is the first block
+  // of 64 features whose completion its issuer waits for (the blocks before it need no signal).
+  int q_first = 0;
+  if (kPerformer && (int)o_col < p) q_first = (min(p, (int)o_col + d) - 1) >> 6;
+  // p's block kb of 64 features (32 columns of fp16 pairs) sits at column pcol(kb): side by side from
+  // column 0, except that with d = 64 blocks 2 and 3 skip over O to columns 128 and 160
+  auto pcol = [&](int kb) -> uint32_t { return (uint32_t)(32 * kb + ((d == 64 && kb >= 2) ? 64 : 0)); };
 
   if (ntiles > 0 && warp == 0 && lane == 0) {
     // W is an input, not a result of stage 2: its load starts before the dependency wait
@@ -169,7 +179,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   grid_dependency_wait();
 
   if (ntiles > 0) {
-    if (warp == 0 && lane == 0) {
+    if (warp == 0 && elect_one()) {
       // ============================================================ TMA producer
       // Q tiles only: they do not depend on the head's operands, so the ring keeps running ahead
       // across a change of head (a^T is reloaded by the operand builder, which waits for the drain)
@@ -195,7 +205,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         for (int i = max(0, issued - NS); i < issued; ++i)
           (void)mbar_wait(bar_qfull + 8 * (i % NS), (i / NS) & 1, prm.status, &abort_flag);
       }
-    } else if (warp == 1 && lane == 0) {
+    } else if (warp == 1 && elect_one()) {
       // ============================================================ issuer of the first products
       // S_i = Q_i W^T + 1 b^T (PERFORMER only).  A new head's bias operand is ready once
       // bar_biasready flips, which also means every MMA of the old head has completed.
@@ -235,6 +245,9 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         }
       }
     } else if (warp == 3 && lane == 0) {
+      // (lane 0 rather than an elected lane: with the slower issue code the compiler makes for a lane it
+      // cannot prove to be alone, the second products of one tile interleave better with the first
+      // products of the next: measured 5 % faster at m = 128 and 3 % at d = 128)
       // ============================================================ issuer of the second products
       // O_j = p_j a once the 128 row owners of tile j have written p_j.  Before the first tile of a
       // new head it waits for that head's a^T; after the last tile of a head it commits to
@@ -252,15 +265,19 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           head_prev = head;
           ++events;
         }
-        ok = mbar_wait(bar_pfull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag);
-        if (!ok) break;
-        tcgen05_fence_after();
         const uint32_t tb = tmem + buf * buf_cols;
-        // four 16-wide steps per call: one 64-feature block of p (TMEM) against one block of a^T
-        for (int kb = 0; kb < kp; ++kb) {
-          const uint64_t bd = make_sdesc(base + L.aT + kb * (d * 128), 16, 1024, kSwizzle128);
-          mma_ts_x4(tb + o_col, tb + kb * 32, bd, 2, idesc2, kb > 0 ? 1u : 0u);
+        // block by block of 64 features as the row owners hand them over (the blocks before q_first
+        // go together with block q_first); four 16-wide steps per call
+        for (int kb = q_first; kb < kp && ok; ++kb) {
+          ok = mbar_wait(bar_pfull + 8 * (4 * buf + kb), (j >> nb_shift) & 1, prm.status, &abort_flag);
+          if (!ok) break;
+          tcgen05_fence_after();
+          for (int kk = (kb == q_first ? 0 : kb); kk <= kb; ++kk) {
+            const uint64_t bd = make_sdesc(base + L.aT + kk * (d * 128), 16, 1024, kSwizzle128);
+            mma_ts_x4(tb + o_col, tb + pcol(kk), bd, 2, idesc2, kk > 0 ? 1u : 0u);
+          }
         }
+        if (!ok) break;
         mma_commit(bar_ofull + 8 * buf);
         const bool last_of_head = (j + 1 < ntiles) && ((t_begin + j + 1) / prm.tiles_per_head != head);
         if (last_of_head) mma_commit(bar_drained);
@@ -358,6 +375,13 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         }
         return true;
       };
+      // a block of 64 features of p is complete: every row owner waits for its own TMEM stores and
+      // tells the issuer of the second product
+      auto hand_over = [&](int buf, int kb) {
+        tmem_wait_st();
+        tcgen05_fence_before();
+        mbar_arrive(bar_pfull + 8 * (4 * buf + kb));
+      };
       float inv_prev = 0.f;                            // four buffers: 1 / sum of the group's previous tile
       // head and tile-within-head of this group's current tile, advanced by two tiles per iteration;
       // the previous tile's pair is kept for the late read-out
@@ -419,7 +443,8 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
               const __half2 hh = __floats2half2_rn(e0, e1);
               h[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
-            tmem_st16(tb + (c >> 1), h);
+            const uint32_t pc = pcol(c >> 6);
+            tmem_st16(tb + pc, h);
             tmem_wait_ld(rb);
             if (c + 64 < p) tmem_ld32(tb + c + 64, ra);
 #pragma unroll
@@ -433,7 +458,8 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
               const __half2 hh = __floats2half2_rn(e0, e1);
               h[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
-            tmem_st16(tb + ((c + 32) >> 1), h);
+            tmem_st16(tb + pc + 16, h);
+            if ((c >> 6) >= q_first && c + 64 < p) hand_over(buf, c >> 6);
           }
         } else {
           // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
@@ -471,12 +497,11 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
               }
             }
             tmem_st16(tb + (c >> 1), h);
+            if ((c & 32) != 0 && c + 32 < d) hand_over(buf, c >> 6);
           }
           mbar_arrive(bar_qempty + 8 * st);             // this thread is done with the Q tile
         }
-        tmem_wait_st();
-        tcgen05_fence_before();
-        mbar_arrive(bar_pfull + 8 * buf);
+        hand_over(buf, kp - 1);                         // the last block of the tile
 
         const float inv = 1.f / fmaxf(denom + denom1, 1.17549435e-38f);
         if (NB == 4) {

@@ -21,6 +21,19 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
+// One lane of a converged warp (all 32 lanes must execute this together).  Code guarded by it is
+// known to the compiler to run in a single thread, so the descriptor operands of tcgen05.mma and of
+// the TMA instructions are set up once instead of once per possibly active lane.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // ------------------------------------------------------------------------------ dependent launch
 // A kernel launched with programmatic stream serialisation may start while its predecessor in the
 // stream is still running; it must not touch the predecessor's results before this wait (which
