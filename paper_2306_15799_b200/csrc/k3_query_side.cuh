@@ -49,7 +49,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 // shared-memory plan (byte offsets from a 1024-aligned base)
 struct K3Smem {
-  uint32_t w, ones, bias, aT, q, scale, bars, total;
+  uint32_t w, ones, bias, aT, q, ostage, scale, bars, total;
   int q_stages;
 };
 
@@ -64,6 +64,7 @@ __host__ __device__ inline K3Smem k3_smem_plan(int d, int p, bool performer) {
   off = (off + 1023u) & ~1023u;
   s.q_stages = (d == 64) ? 4 : 2;
   s.q = off;    off += (uint32_t)s.q_stages * 128 * d * 2;
+  s.ostage = off; off += (d == 64) ? 8 * 4096 : 0;                 // d = 64: a [32 x 64] bf16 output slab per row-owner warp
   s.scale = off; off += 1024;                                      // RNN: z_i / max z as floats
   s.bars = off; off += 512;
   s.total = off + 1024;                                            // alignment slack
@@ -73,7 +74,8 @@ __host__ __device__ inline K3Smem k3_smem_plan(int d, int p, bool performer) {
 template <bool kPerformer>
 __global__ void __launch_bounds__(kK3Threads, 1)
 k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmW,
-              const __grid_constant__ CUtensorMap tmAT, const K3Params prm) {
+              const __grid_constant__ CUtensorMap tmAT, const __grid_constant__ CUtensorMap tmO,
+              const K3Params prm) {
   using namespace tc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -335,13 +337,49 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
       const float kLog2e = 1.4426950408889634f;
       int events = 0;
       bool ok = true;
-      // read-out of tile j: O / sum -> bf16 -> this thread's output row, 32 bytes per store
+      // read-out of tile j: O / sum -> bf16 -> the output rows
       // (head and first row of the tile are tracked by the caller: no divisions on this path)
+      const uint32_t slab = base + L.ostage + (uint32_t)(warp - 4) * 4096u;
       auto read_out = [&](int j, float inv, int head, int row0) -> bool {
         const int buf = j & (NB - 1);
         const uint32_t tb = tmem + buf * buf_cols + lane_off + o_col;
         if (!mbar_wait(bar_ofull + 8 * buf, (j >> nb_shift) & 1, prm.status, &abort_flag)) return false;
         tcgen05_fence_after();
+        if (d == 64) {
+          // d = 64: the warp's 32 rows go through a 4 KB slab of shared memory (128-byte rows, 16-byte
+          // chunks swizzled like the tensor map expects, so the stores do not collide) and leave as one
+          // TMA store of whole lines; rows past the end of the sequence are clipped by the tensor map
+          if (lane == 0) bulk_wait_group_read0();          // the slab's previous store has been read
+          __syncwarp();
+          uint32_t ra[32], rb[32];
+          tmem_ld32(tb, ra);
+          tmem_ld32(tb + 32, rb);
+          tmem_wait_ld(ra);
+          tmem_wait_ld(rb);
+          tcgen05_fence_before();
+          mbar_arrive(bar_sfree + 8 * buf);                 // the buffer goes back before the rows are packed
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const uint32_t* src = g < 4 ? ra : rb;
+            uint32_t v[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(src[(g & 3) * 8 + 2 * e]) * inv,
+                                                              __uint_as_float(src[(g & 3) * 8 + 2 * e + 1]) * inv);
+              v[e] = *reinterpret_cast<const uint32_t*>(&o2);
+            }
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + lane * 128 + ((g ^ (lane & 7)) << 4)),
+                         "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && row0 + q4 * 32 < prm.N) {
+            if (prm.H > 0) tma_store_3d(&tmO, slab, (head % prm.H) * d, row0 + q4 * 32, head / prm.H);
+            else tma_store_3d(&tmO, slab, 0, row0 + q4 * 32, head);
+            bulk_commit_group();
+          }
+          return true;
+        }
         __nv_bfloat16* orow = prm.H > 0
             ? prm.out + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * d
             : prm.out + ((size_t)head * prm.N + row0 + row) * d;
@@ -518,6 +556,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         while (tih >= prm.tiles_per_head) { tih -= prm.tiles_per_head; ++head_i; }
       }
       if (NB == 4 && ok && ntiles > grp) (void)read_out(grp + 2 * ((ntiles - 1 - grp) / 2), inv_prev, head_o, row0_o);
+      if (lane == 0) bulk_wait_group0();                // this warp's output stores are complete
     }
   }
   tcgen05_fence_before();

@@ -86,7 +86,7 @@ inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int ran
 }
 
 struct TensorMaps {
-  CachedMap E, F, K, V, kpvp, Q, W, W2, aT;
+  CachedMap E, F, K, V, kpvp, Q, W, W2, aT, O;
 };
 
 // Per-device context of the tensor-core kernels: the cached tensor maps (their pointers are device
@@ -255,6 +255,11 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
   const unsigned bQ[3] = {64, 128, 1};
   const unsigned long long dA[3] = {(unsigned long long)p, (unsigned long long)d, (unsigned long long)BH};
   const unsigned bA[3] = {64, (unsigned)d, 1};
+  const unsigned bO[3] = {64, 32, 1};                 // d = 64: one row-owner warp's slab of the output
+  if (d == 64 && !encode_map(&tm.O, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, out, dQ, bO)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
   if (!encode_map(&tm.Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Q, dQ, bQ) ||
       !encode_map(&tm.aT, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, 3, aT16, dA, bA)) {
     *cuda_err = (int)cudaErrorInvalidValue;
@@ -281,9 +286,9 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   int grid = tc.sm_count();
   if (grid > prm.total_tiles) grid = prm.total_tiles;
-  // the RNN kernel ignores tmW; pass any valid map
+  // the RNN kernel ignores tmW and only d = 64 stores through tmO; pass any valid map otherwise
   e = launch_after_predecessor(fn, grid, kK3Threads, L.total, st, tm.Q.map, performer ? tm.W.map : tm.Q.map,
-                               tm.aT.map, prm);
+                               tm.aT.map, d == 64 ? tm.O.map : tm.Q.map, prm);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
