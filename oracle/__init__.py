@@ -77,6 +77,9 @@ class OracleLib:
         lib.flurka_oracle_features.restype = ci
         lib.flurka_oracle_features.argtypes = [_DP, ci, ci, _DP, ci, ci, ci, ci, _DP]
         lib.flurka_oracle_threads.restype = ci
+        if hasattr(lib, "flurka_oracle_fused_head"):
+            lib.flurka_oracle_fused_head.restype = ci
+            lib.flurka_oracle_fused_head.argtypes = [_DP] * 9 + [ci] * 7 + [_LP, ctypes.c_long] + [_DP] * 4
         self._lib = lib
 
     def threads(self) -> int:
@@ -129,6 +132,34 @@ class OracleLib:
             raise ValueError("flurka_oracle_head_quadratic failed: %d" % rc)
         return (out, Ahat) if weights else out
 
+    def fused_head(self, Xq, Xk, Xv, E, F, Wq, Wk, Wv, W, variant, *, stabilise=True, rows=None, intermediates=False):
+        """One head of Eq. (2) with its linear maps: Xq, Xk, Xv [N,dm] un-projected; Wq, Wk, Wv [dm,d]
+        (this head's); E, F [k,N]; W [m,d] or None.  Returns O [n_rows,d], or (O, dict(Kp, Vp, Q))."""
+        Xq, Xk, Xv, E, F, Wq, Wk, Wv, W = (_f64(x) for x in (Xq, Xk, Xv, E, F, Wq, Wk, Wv, W))
+        N, dm = Xq.shape
+        d = Wq.shape[1]
+        k = E.shape[0]
+        assert Xk.shape == (N, dm) and Xv.shape == (N, dm), "Xq, Xk, Xv must be [N, dm]"
+        assert Wq.shape == (dm, d) and Wk.shape == (dm, d) and Wv.shape == (dm, d), "Wq, Wk, Wv must be [dm, d]"
+        assert E.shape == (k, N) and F.shape == (k, N), "E, F must be [k, N]"
+        if variant == PERFORMER:
+            assert W is not None and W.shape[1] == d, "W must be [m, d]"
+            m = W.shape[0]
+        else:
+            m = 0
+        rows_arr, n_rows, rows_p = _rows(rows, N)
+        out = np.empty((n_rows, d), dtype=np.float64)
+        if intermediates:
+            Kp, Vp, Qh = np.empty((k, d)), np.empty((k, d)), np.empty((n_rows, d))
+        else:
+            Kp = Vp = Qh = None
+        rc = self._lib.flurka_oracle_fused_head(
+            _ptr(Xq), _ptr(Xk), _ptr(Xv), _ptr(E), _ptr(F), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(W), variant,
+            N, dm, d, k, m, 1 if stabilise else 0, rows_p, n_rows, _ptr(out), _ptr(Kp), _ptr(Vp), _ptr(Qh))
+        if rc:
+            raise ValueError("flurka_oracle_fused_head failed: %d" % rc)
+        return (out, {"Kp": Kp, "Vp": Vp, "Q": Qh}) if intermediates else out
+
     def features(self, X, W, variant, *, stabilise=False, scope_global=False):
         """phi applied to the rows of X [rows,d]. Returns [rows,m] (PERFORMER) or [rows,d] (RNN)."""
         X, W = _f64(X), _f64(W)
@@ -175,6 +206,10 @@ def head(*a, **kw):
 
 def head_quadratic(*a, **kw):
     return default().head_quadratic(*a, **kw)
+
+
+def fused_head(*a, **kw):
+    return default().fused_head(*a, **kw)
 
 
 def features(*a, **kw):

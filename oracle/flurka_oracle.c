@@ -13,7 +13,8 @@
  *                        the product in the associative (linear-cost) order.
  *                        The per-head linear maps W^Q, W^K, W^V are taken as
  *                        already applied to the inputs (legal by
- *                        associativity, (E1 K) W^K = E1 (K W^K)).
+ *                        associativity, (E1 K) W^K = E1 (K W^K)), except in
+ *                        flurka_oracle_fused_head, which writes them out.
  *   Section 2.1          E1, E2 are d_k x N (here: E, F of shape k x N).
  *                        Kernel attention phi(Q)(phi(K)^T V); random-feature
  *                        maps phi(x) = m^{-1/2} [psi_1(x) .. psi_m(x)] with
@@ -23,7 +24,7 @@
  *                        a_nj = phi(x_n).phi(y_j) / sum_j' phi(x_n).phi(y_j'),
  *                        i.e. rows are normalised; Eq. (2) elides this.
  *
- * Readings where the paper is silent (all stated again in the design notes):
+ * Readings where the paper is silent:
  *   - positive random features psi_i(x) = exp(w_i.x - |x|^2/2) (FAVOR+);
  *   - the non-random map is phi(x) = elu(x) + 1, alpha = 1, feature dim = d;
  *   - the normaliser sums over the k projected keys;
@@ -263,6 +264,95 @@ int flurka_oracle_head_quadratic(const double *Q, const double *K, const double 
   }
   free(Kp); free(Vp); free(Phik); free(Qs); free(Phiq);
   return fail ? -7 : 0;
+}
+
+/* Section 2.1 / Appendix B "Linear Transformations": Y = X Wm, X is rows x dm, Wm is dm x d. */
+static void linear_map(const double *X, int rows, int dm, const double *Wm, int d, double *Y) {
+#pragma omp parallel for schedule(static)
+  for (int r = 0; r < rows; ++r) {
+    double *y = Y + (size_t)r * d;
+    for (int c = 0; c < d; ++c) y[c] = 0.0;
+    for (int e = 0; e < dm; ++e) {
+      const double x = X[(size_t)r * dm + e];
+      const double *w = Wm + (size_t)e * d;
+      for (int c = 0; c < d; ++c) y[c] += x * w[c];
+    }
+  }
+}
+
+/*
+ * One head of Eq. (2) with its linear maps written out,
+ *     Head = phi(Xq W^Q) ( phi((E Xk) W^K)^T ((F Xv) W^V) ),   rows normalised as in Appendix D,
+ * in the order the equation and Appendix B's step list give: the un-projected keys and values
+ * (N x dm) are contracted along the sequence FIRST (k x dm), the per-head maps (dm x d) are
+ * applied to the k contracted rows, the queries are mapped as they are.  Then steps 2 to 4 of
+ * flurka_oracle_head.  Xq, Xk, Xv: [N,dm] (they may be the same array); Wq, Wk, Wv: [dm,d], this
+ * head's maps; rows / n_rows select query rows (NULL: all).  Optional outputs (may be NULL):
+ * Kp_out, Vp_out [k,d] = (E Xk) W^K and (F Xv) W^V; Q_out [n_rows,d] = Xq W^Q.
+ */
+int flurka_oracle_fused_head(const double *Xq, const double *Xk, const double *Xv,
+                             const double *E, const double *F, const double *Wq,
+                             const double *Wk, const double *Wv, const double *W, int variant,
+                             int N, int dm, int d, int k, int m, int stabilise,
+                             const long *rows, long n_rows, double *out, double *Kp_out,
+                             double *Vp_out, double *Q_out) {
+  int rc = check_args(Xq, Xk, Xv, E, F, W, variant, N, d, k, m, out);
+  if (rc) return rc;
+  if (!Wq || !Wk || !Wv) return -1;
+  if (dm <= 0) return -3;
+  if (!rows) n_rows = N;
+  if (n_rows < 0) return -3;
+  const int p = (variant == FLURKA_ORACLE_PERFORMER) ? m : d;
+  const long nq = n_rows > 0 ? n_rows : 1;
+
+  double *Kt = (double *)malloc((size_t)k * dm * sizeof(double));
+  double *Vt = (double *)malloc((size_t)k * dm * sizeof(double));
+  double *Kp = (double *)malloc((size_t)k * d * sizeof(double));
+  double *Vp = (double *)malloc((size_t)k * d * sizeof(double));
+  double *Phik = (double *)malloc((size_t)k * p * sizeof(double));
+  double *KV = (double *)calloc((size_t)p * d, sizeof(double));
+  double *z = (double *)calloc((size_t)p, sizeof(double));
+  double *Xs = gather_rows(Xq, dm, rows, nq);
+  double *Qs = (double *)malloc((size_t)nq * d * sizeof(double));
+  double *Phiq = (double *)malloc((size_t)nq * p * sizeof(double));
+  if (!Kt || !Vt || !Kp || !Vp || !Phik || !KV || !z || !Xs || !Qs || !Phiq) {
+    free(Kt); free(Vt); free(Kp); free(Vp); free(Phik); free(KV); free(z); free(Xs); free(Qs); free(Phiq);
+    return -7;
+  }
+
+  /* the low-rank contraction comes before the linear maps */
+  down_project(E, Xk, N, dm, k, Kt);
+  down_project(F, Xv, N, dm, k, Vt);
+  linear_map(Kt, k, dm, Wk, d, Kp);
+  linear_map(Vt, k, dm, Wv, d, Vp);
+  linear_map(Xs, (int)n_rows, dm, Wq, d, Qs);
+  /* feature maps, key-side summaries, ratio: as in flurka_oracle_head */
+  feature_map(Kp, k, d, W, m, variant, stabilise, /*one scalar per head*/ 1, Phik);
+  feature_map(Qs, (int)n_rows, d, W, m, variant, stabilise, /*one scalar per row*/ 0, Phiq);
+  for (int j = 0; j < k; ++j)
+    for (int i = 0; i < p; ++i) {
+      const double f = Phik[(size_t)j * p + i];
+      z[i] += f;
+      for (int c = 0; c < d; ++c) KV[(size_t)i * d + c] += f * Vp[(size_t)j * d + c];
+    }
+#pragma omp parallel for schedule(static)
+  for (long r = 0; r < n_rows; ++r) {
+    double den = 0.0;
+    double *o = out + (size_t)r * d;
+    for (int c = 0; c < d; ++c) o[c] = 0.0;
+    for (int i = 0; i < p; ++i) {
+      const double f = Phiq[(size_t)r * p + i];
+      den += f * z[i];
+      for (int c = 0; c < d; ++c) o[c] += f * KV[(size_t)i * d + c];
+    }
+    for (int c = 0; c < d; ++c) o[c] /= den;
+  }
+
+  if (Kp_out) memcpy(Kp_out, Kp, (size_t)k * d * sizeof(double));
+  if (Vp_out) memcpy(Vp_out, Vp, (size_t)k * d * sizeof(double));
+  if (Q_out) memcpy(Q_out, Qs, (size_t)n_rows * d * sizeof(double));
+  free(Kt); free(Vt); free(Kp); free(Vp); free(Phik); free(KV); free(z); free(Xs); free(Qs); free(Phiq);
+  return 0;
 }
 
 /*

@@ -273,6 +273,56 @@ def pin_forward_layout(orc):
                 assert _rel(O[b, h], ref) < 1e-11
 
 
+def _tiny_fused(seed, N=24, dm=10, d=6, k=5, m=12, scale=0.5):
+    r = _rng(seed)
+    Xq, Xk, Xv = (r.normal(size=(N, dm)) for _ in range(3))
+    Wq = r.normal(size=(dm, d)) * scale / math.sqrt(dm)
+    Wk = r.normal(size=(dm, d)) * scale / math.sqrt(dm)
+    Wv = r.normal(size=(dm, d)) / math.sqrt(dm)
+    E = r.normal(size=(k, N)) / math.sqrt(k)
+    F = r.normal(size=(k, N)) / math.sqrt(k)
+    W = r.normal(size=(m, d))
+    return Xq, Xk, Xv, E, F, Wq, Wk, Wv, W
+
+
+def pin_fused_maps_commute_with_the_contraction(orc):
+    """Eq. (2): (E1 K) W^K = E1 (K W^K).  The head with its linear maps written out, which contracts the
+    un-projected keys and values first, equals the plain head on inputs projected beforehand (numpy)."""
+    for variant in (PERFORMER, RNN):
+        for seed in (11, 12):
+            Xq, Xk, Xv, E, F, Wq, Wk, Wv, W = _tiny_fused(seed)
+            Wf = W if variant == PERFORMER else None
+            got, mid = orc.fused_head(Xq, Xk, Xv, E, F, Wq, Wk, Wv, Wf, variant, intermediates=True)
+            ref = orc.head_quadratic(Xq @ Wq, Xk @ Wk, Xv @ Wv, E, F, Wf, variant)
+            assert _rel(got, ref) < 1e-10, ("fused vs projected inputs", variant, _rel(got, ref))
+            assert _rel(mid["Kp"], E @ (Xk @ Wk)) < 1e-12 and _rel(mid["Vp"], F @ (Xv @ Wv)) < 1e-12
+            assert _rel(mid["Q"], Xq @ Wq) < 1e-12
+            rows = [3, 0, 17]
+            sub = orc.fused_head(Xq, Xk, Xv, E, F, Wq, Wk, Wv, Wf, variant, rows=rows)
+            assert _rel(sub, got[rows]) < 1e-12
+
+
+def pin_fused_special_cases(orc):
+    """Identity maps give back the plain head; one projected key gives O_n = (F Xv) W^V for every row;
+    the output is linear in Xv and does not change when Xq's rows the call does not select change."""
+    Q, K, V, E, F, W = _tiny(21, N=20, d=6, k=4, m=10)
+    eye = np.eye(6)
+    for variant, Wf in ((PERFORMER, W), (RNN, None)):
+        a = orc.fused_head(Q, K, V, E, F, eye, eye, eye, Wf, variant)
+        assert _rel(a, orc.head(Q, K, V, E, F, Wf, variant)) < 1e-11
+        Xq, Xk, Xv, E2, F2, Wq, Wk, Wv, W2 = _tiny_fused(22, k=1)
+        Wf2 = W2 if variant == PERFORMER else None
+        o = orc.fused_head(Xq, Xk, Xv, E2, F2, Wq, Wk, Wv, Wf2, variant)
+        assert np.allclose(o, np.broadcast_to((F2 @ Xv) @ Wv, o.shape), atol=1e-12)
+        Xq, Xk, Xv, E3, F3, Wq, Wk, Wv, W3 = _tiny_fused(23)
+        Wf3 = W3 if variant == PERFORMER else None
+        Xv2 = _rng(24).normal(size=Xv.shape)
+        lin = orc.fused_head(Xq, Xk, 2.0 * Xv - 3.0 * Xv2, E3, F3, Wq, Wk, Wv, Wf3, variant)
+        sep = 2.0 * orc.fused_head(Xq, Xk, Xv, E3, F3, Wq, Wk, Wv, Wf3, variant) \
+            - 3.0 * orc.fused_head(Xq, Xk, Xv2, E3, F3, Wq, Wk, Wv, Wf3, variant)
+        assert _rel(lin, sep) < 1e-11
+
+
 ALL_PINS = [
     pin_quadratic_equals_associative,
     pin_identity_projection,
@@ -286,6 +336,8 @@ ALL_PINS = [
     pin_feature_expectation,
     pin_softmax_limit,
     pin_forward_layout,
+    pin_fused_maps_commute_with_the_contraction,
+    pin_fused_special_cases,
 ]
 
 
@@ -315,6 +367,11 @@ MUTANTS = {
     "features_from_unprojected_keys": (
         "feature_map(Kp, k, d, W, m, variant, stabilise, /*scope_global=*/1, Phik);",
         "feature_map(K, k, d, W, m, variant, stabilise, /*scope_global=*/1, Phik);"),
+    "fused_value_map_is_key_map": ("linear_map(Vt, k, dm, Wv, d, Vp);", "linear_map(Vt, k, dm, Wk, d, Vp);"),
+    "fused_keys_from_value_input": ("down_project(E, Xk, N, dm, k, Kt);", "down_project(E, Xv, N, dm, k, Kt);"),
+    "fused_query_map_is_key_map": ("linear_map(Xs, (int)n_rows, dm, Wq, d, Qs);", "linear_map(Xs, (int)n_rows, dm, Wk, d, Qs);"),
+    "linear_map_transposed": ("y[c] += x * w[c];", "y[c] += x * Wm[(size_t)c * dm + e];"),
+    "fused_queries_contracted_too": ("double *Xs = gather_rows(Xq, dm, rows, nq);", "double *Xs = gather_rows(Xk, dm, rows, nq);"),
     "head_stride_wrong": ("const size_t head = (size_t)N * d;", "const size_t head = (size_t)N * d / 2 * 2 - d;"),
 }
 
