@@ -109,6 +109,35 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
                         const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
                         void* stream);
 
+/*
+ * flurka_forward_fused -- Eq. (2) with its per-head linear maps inside the call:
+ *
+ *     Head_h = phi(Xq W^Q_h) ( phi((E Xk) W^K_h)^T ((F Xv) W^V_h) ),  rows normalised as in Appendix D,
+ *     out    = Concat(Head_1 .. Head_H)                                           (Section 2)
+ *
+ * in the order Section 3 argues for and Appendix B's step list counts ("Linear Transformations":
+ * N d_m^2 + 2 d_k d_m^2 instead of 3 N d_m^2): the un-projected keys and values are contracted along
+ * the sequence first, W^K and W^V touch only the k contracted rows, W^Q maps the N queries.
+ *
+ *   Xq, Xk, Xv  device, [B,N,dm]   the layer's inputs before the maps (they may be one and the same buffer)
+ *   E, F        device, [k,N]      W  device, [m,d] (NULL for RNN)
+ *   Wq, Wk, Wv  device, [dm, H*d]  columns h*d .. h*d+d-1 are head h's map (x W, row vector times matrix)
+ *   variant     flurka_kernel_t | FLURKA_IO_BF16 / FLURKA_IO_FP32   (FLURKA_LAYOUT_BNHD is refused: the
+ *               layout is fixed)
+ *   out         device, [B,N,H,d] = [B,N,H*d], same element type; must not overlap an input
+ *
+ * Limits as for flurka_forward, and 1 <= dm <= 16384.  The tensor-core path needs what flurka_forward's
+ * needs and dm % 64 == 0; everything else runs on CUDA cores.  Asynchronous on `stream`; scratch (the
+ * inner problem's, the contracted rows and Xq W^Q as [B,N,H,d]) comes from the workspace as described
+ * for flurka_forward, flurka_fused_workspace_bytes() says how much.  Afterwards flurka_last_status,
+ * flurka_last_path, flurka_last_launches, flurka_debug_copy (K' and V' after the maps) and, with timing
+ * on, flurka_last_stage_ms (stage 0 = contraction and all three linear maps) describe this call.
+ */
+int flurka_forward_fused(const void* Xq, const void* Xk, const void* Xv, const void* E, const void* F,
+                         const void* Wq, const void* Wk, const void* Wv, const void* W, int variant, int B, int H,
+                         int N, int dm, int d, int k, int m, void* out, void* stream);
+size_t flurka_fused_workspace_bytes(int variant, int B, int H, int N, int dm, int d, int k, int m);
+
 /* Bytes of device scratch flurka_forward needs for this problem (0 on invalid arguments). Holds the
  * fp32 projections K', V' (Eq. (2)'s E K and F V), the key-side feature summaries and a status word. */
 size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m);

@@ -21,7 +21,7 @@ EXPORTS = [
     "flurka_set_path", "flurka_set_cta_limit", "flurka_last_path", "flurka_last_launches", "flurka_debug_copy",
     "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
     "flurka_strerror", "flurka_version", "flurka_forward_static_scratch", "flurka_static_scratch_need",
-    "flurka_measure_ex2_rate",
+    "flurka_measure_ex2_rate", "flurka_forward_fused", "flurka_fused_workspace_bytes",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -83,6 +83,10 @@ def load() -> ctypes.CDLL:
     lib.flurka_strerror.restype = ctypes.c_char_p
     lib.flurka_strerror.argtypes = [ci]
     lib.flurka_version.restype = ci
+    lib.flurka_forward_fused.restype = ci
+    lib.flurka_forward_fused.argtypes = [vp] * 9 + [ci] * 8 + [vp, vp]
+    lib.flurka_fused_workspace_bytes.restype = sz
+    lib.flurka_fused_workspace_bytes.argtypes = [ci] * 8
     lib.flurka_measure_ex2_rate.restype = ci
     lib.flurka_measure_ex2_rate.argtypes = [ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -170,6 +174,41 @@ def flurka_forward_host(Q, K, V, E, F, W, variant, out=None, stream=None, layout
     if rc:
         raise FlurkaError(rc, "flurka_forward_host")
     return out
+
+
+def flurka_forward_fused(Xq, Xk, Xv, E, F, Wq, Wk, Wv, W, variant, H, out=None, stream=None):
+    """Eq. (2) with its linear maps: Xq, Xk, Xv [B,N,dm] un-projected, Wq, Wk, Wv [dm,H*d]; out [B,N,H,d]."""
+    B, N, dm = Xq.shape
+    if Wq.dim() != 2 or Wq.shape[0] != dm or Wq.shape[1] % H:
+        raise ValueError("flurka: Wq, Wk, Wv must be [dm, H*d]")
+    d = Wq.shape[1] // H
+    if out is None:
+        out = torch.empty((B, N, H, d), dtype=Xq.dtype, device=Xq.device)
+    for name, t in (("Xq", Xq), ("Xk", Xk), ("Xv", Xv), ("E", E), ("F", F), ("Wq", Wq), ("Wk", Wk), ("Wv", Wv),
+                    ("out", out)):
+        if t.device.type != "cuda" or not t.is_contiguous() or t.dtype != Xq.dtype:
+            raise ValueError("flurka: %s must be a contiguous CUDA tensor of Xq's dtype" % name)
+    if Xk.shape != Xq.shape or Xv.shape != Xq.shape or Wk.shape != Wq.shape or Wv.shape != Wq.shape:
+        raise ValueError("flurka: Xq, Xk, Xv must be [B,N,dm] and Wq, Wk, Wv [dm,H*d]")
+    if E.dim() != 2 or E.shape[1] != N or F.shape != E.shape or tuple(out.shape) != (B, N, H, d):
+        raise ValueError("flurka: E, F must be [k,N] and out [B,N,H,d]")
+    k, m = E.shape[0], 0
+    if variant == PERFORMER:
+        if W is None or W.dim() != 2 or W.shape[1] != d or W.dtype != Xq.dtype or not W.is_contiguous() \
+                or W.device.type != "cuda":
+            raise ValueError("flurka: W must be a contiguous [m,d] tensor like Xq")
+        m = W.shape[0]
+    rc = load().flurka_forward_fused(
+        Xq.data_ptr(), Xk.data_ptr(), Xv.data_ptr(), E.data_ptr(), F.data_ptr(), Wq.data_ptr(), Wk.data_ptr(),
+        Wv.data_ptr(), W.data_ptr() if W is not None else None, _variant_word(variant, Xq.dtype),
+        B, H, N, dm, d, k, m, out.data_ptr(), _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_forward_fused")
+    return out
+
+
+def flurka_fused_workspace_bytes(variant, io_dtype, B, H, N, dm, d, k, m) -> int:
+    return int(load().flurka_fused_workspace_bytes(_variant_word(variant, io_dtype), B, H, N, dm, d, k, m))
 
 
 def flurka_workspace_bytes(variant, io_dtype, B, H, N, d, k, m) -> int:

@@ -54,6 +54,28 @@ class Workload:
         return 4 * self.B * self.H * self.N * self.d * s + 2 * self.k * self.N * s + self.m * self.d * s
 
 
+@dataclass(frozen=True)
+class FusedWorkload(Workload):
+    """Eq. (2) with its linear maps inside the call: un-projected inputs [B,N,dm], maps [dm,H*d].
+    `shared_x`: queries, keys and values are one and the same input (self-attention)."""
+    dm: int = 0
+    shared_x: bool = True
+
+    def flops(self) -> int:
+        """Appendix B's steps, 2 FLOPs per multiply-add: the contraction of the un-projected keys and values
+        (4 N k dm per batch), W^Q on the N queries (2 N dm Hd), W^K and W^V on the k contracted rows
+        (4 k dm Hd), then the per-head work of the plain forward without its own down-projection."""
+        N, d, k, dm, Hd = self.N, self.d, self.k, self.dm, self.H * self.d
+        per_batch = 4 * N * k * dm + 2 * N * dm * Hd + 4 * k * dm * Hd
+        return per_batch * self.B + super().flops() - 4 * N * k * d * self.B * self.H
+
+    def compulsory_bytes(self) -> int:
+        """The inputs read once (one X when shared), O written once, E, F, the three maps and W read once."""
+        s = self.elem_bytes
+        x = self.B * self.N * self.dm * s * (1 if self.shared_x else 3)
+        return x + self.tokens * self.d * s + 2 * self.k * self.N * s + 3 * self.dm * self.H * self.d * s + self.m * self.d * s
+
+
 C1 = Workload("c1_perf_fp32_n256", PERFORMER, "fp32", 1, 2, 256, 32, 32, 64, BASE_SEED + 1000)
 C2 = Workload("c2_rnn_bf16_n4096", RNN, "bf16", 8, 12, 4096, 64, 256, 0, BASE_SEED + 2000)
 C3 = Workload("c3_perf_bf16_n16384", PERFORMER, "bf16", 4, 16, 16384, 64, 256, 256, BASE_SEED + 3000)
@@ -68,9 +90,13 @@ def c5(k: int, m: int) -> Workload:
 
 C5_GRID = [(k, m) for k in (64, 128, 256, 512) for m in (64, 128, 256)]
 
-BY_NAME = {w.name: w for w in (C1, C2, C3, C4)}
+# c3's shape with the linear maps inside the call: d_m = H d = 1024, self-attention
+F1 = FusedWorkload("f1_fused_perf_bf16_n16384_dm1024", PERFORMER, "bf16", 4, 16, 16384, 64, 256, 256, BASE_SEED + 6000,
+                   dm=1024, shared_x=True)
+
+BY_NAME = {w.name: w for w in (C1, C2, C3, C4, F1)}
 BY_NAME.update({c5(k, m).name: c5(k, m) for (k, m) in C5_GRID})
-ALIASES = {"c1": C1, "c2": C2, "c3": C3, "c4": C4}
+ALIASES = {"c1": C1, "c2": C2, "c3": C3, "c4": C4, "f1": F1}
 
 
 def get(name: str) -> Workload:

@@ -240,10 +240,12 @@ int key_side_dispatch(const Problem& pr, const float* kpvp, const void* W, float
 // (bf16 only); tc2 (which needs tc3) does the same for stage 2.  `timer` (may be NULL) gets an
 // event before and after each stage.  `keep_status`: the status words are left as they are (a
 // later head group of one host-buffer call; they only ever gain bits).
-template <typename T>
-int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
-                 const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc2,
-                 bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status, int* launches) {
+// `stage1(kpvp, status, launches)` fills the (zeroed) K', V' accumulators: the down-projection of
+// already projected heads, or the contraction and the linear maps of un-projected inputs.
+template <typename T, typename Stage1>
+int run_pipeline_with(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* W, void* out,
+                      cudaStream_t st, bool tc2, bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status,
+                      int* launches, Stage1&& stage1) {
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
   float* a32 = (float*)(ws + L.a32);
@@ -256,15 +258,8 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   cudaError_t e = cudaMemsetAsync(ws + clear_from, 0, L.kpvp_end - clear_from, st);
   if (e != cudaSuccess) return cuda_fail(e);
   if (timer) timer->mark(0, st);
-  int rc;
-  if (tc1) {
-    rc = launch_k1(*tc, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err);
-    if (rc) { g_last_cuda_error = cuda_err; return rc; }
-    ++*launches;
-  } else {
-    rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
-    if (rc) return rc;
-  }
+  int rc = stage1(kpvp, status, launches);
+  if (rc) return rc;
   if (timer) timer->mark(1, st);
   if (tc2) {
     float* part = L.total > L.part ? (float*)(ws + L.part) : nullptr;
@@ -291,6 +286,23 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   return FLURKA_OK;
+}
+
+template <typename T>
+int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
+                 const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc2,
+                 bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status, int* launches) {
+  auto stage1 = [&](float* kpvp, int* status, int* n) -> int {
+    if (tc1) {
+      int cuda_err = 0;
+      int rc = launch_k1(*tc, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err);
+      if (rc) { g_last_cuda_error = cuda_err; return rc; }
+      ++*n;
+      return FLURKA_OK;
+    }
+    return launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, n);
+  };
+  return run_pipeline_with<T>(pr, L, ws, Q, W, out, st, tc2, tc3, tc, timer, keep_status, launches, stage1);
 }
 
 int validate_pointers(const Problem& pr, const void* Q, const void* K, const void* V, const void* E,
@@ -571,6 +583,152 @@ const char* flurka_strerror(int code) {
 }
 
 int flurka_version(void) { return FLURKA_VERSION; }
+
+}  // extern "C"
+
+namespace {
+
+// Scratch of the entry point with un-projected inputs, after the inner problem's own layout:
+//   kt    fp32 E Xk[b], F Xv[b]: tensor path [2][B][dm/64][k][64] (64-wide column blocks), else [2][B][k][dm]
+//   a3    bf16 [2B][k][3 dm]: three-term split of kt (tensor path only)
+//   qp    Xq W^Q as [B,N,H,d] in the I/O type
+struct FusedLayout {
+  Layout L;
+  size_t kt, kt_bytes, a3, qp, total;
+};
+
+FusedLayout make_fused_layout(const Problem& pr, int dm) {
+  FusedLayout f;
+  f.L = make_layout(pr);
+  size_t off = f.L.total;
+  f.kt_bytes = (size_t)2 * pr.B * pr.k * dm * 4;
+  f.kt = off; off = align256(off + f.kt_bytes);
+  f.a3 = off; off = align256(off + (pr.fp32 ? 0 : (size_t)2 * pr.B * pr.k * 3 * dm * 2));
+  f.qp = off; off = align256(off + pr.qkv_elems() * pr.esize());
+  f.total = off;
+  return f;
+}
+
+bool fused_tensor_ok(const Problem& pr, int dm) { return tensor_path_ok(pr) && dm % 64 == 0 && dm >= 64; }
+
+template <typename T>
+int simt_map(const void* A, const void* Bm, void* C, bool a_f32, bool c_f32, int M, int K, int ncols, int Z,
+             size_t a_stride, size_t b_stride, int head_d, int z0, cudaStream_t st, int* launches) {
+  dim3 grid((ncols + 31) / 32, (M + 31) / 32, Z);
+  if (a_f32)
+    simt_linear_map<float, T, float><<<grid, 256, 0, st>>>((const float*)A, (const T*)Bm, (float*)C, M, K, ncols,
+                                                           a_stride, b_stride, head_d, z0);
+  else if (c_f32)
+    simt_linear_map<T, T, float><<<grid, 256, 0, st>>>((const T*)A, (const T*)Bm, (float*)C, M, K, ncols, a_stride,
+                                                       b_stride, head_d, z0);
+  else
+    simt_linear_map<T, T, T><<<grid, 256, 0, st>>>((const T*)A, (const T*)Bm, (T*)C, M, K, ncols, a_stride, b_stride,
+                                                   head_d, z0);
+  ++*launches;
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? FLURKA_OK : cuda_fail(e);
+}
+
+template <typename T>
+int fused_pipeline(const Problem& pr, int dm, const FusedLayout& FL, char* ws, const void* Xq, const void* Xk,
+                   const void* Xv, const void* E, const void* F, const void* Wq, const void* Wk, const void* Wv,
+                   const void* W, void* out, cudaStream_t st, bool tensor, TensorContext* tc, StageTimer* timer,
+                   int* launches) {
+  float* kt = (float*)(ws + FL.kt);
+  void* qp = ws + FL.qp;
+  auto stage1 = [&](float* kpvp, int* status, int* n) -> int {
+    int cuda_err = 0, rc;
+    cudaError_t e = cudaMemsetAsync(kt, 0, FL.kt_bytes, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (tensor) {
+      // Q = Xq W^Q first (the long one), then the contraction of the un-projected keys and values as
+      // dm/64 pseudo-heads of width 64, then W^K, W^V on the k contracted rows
+      rc = launch_k0_query_map(*tc, Xq, Wq, qp, pr.B, pr.N, pr.H, dm, pr.d, status, st, &cuda_err);
+      if (rc) { g_last_cuda_error = cuda_err; return rc; }
+      rc = launch_k1(*tc, Xk, Xv, E, F, kt, pr.B * (dm / 64), dm / 64, pr.N, 64, pr.k, status, st, &cuda_err);
+      if (rc) { g_last_cuda_error = cuda_err; return rc; }
+      rc = launch_k0_key_value_maps(*tc, kt, (__nv_bfloat16*)(ws + FL.a3), Wk, Wv, kpvp, pr.B, pr.H, dm, pr.d, pr.k,
+                                    status, st, &cuda_err);
+      if (rc) { g_last_cuda_error = cuda_err; return rc; }
+      *n += 4;
+      return FLURKA_OK;
+    }
+    const size_t xb = (size_t)pr.N * dm, ktb = (size_t)pr.k * dm;
+    // kt[t][b] = (E | F) X[b];  K', V' = kt W^K, kt W^V (head-split);  Q = Xq W^Q
+    if ((rc = simt_map<T>(E, Xk, kt, false, true, pr.k, pr.N, dm, pr.B, 0, xb, 0, 0, st, n))) return rc;
+    if ((rc = simt_map<T>(F, Xv, kt + (size_t)pr.B * ktb, false, true, pr.k, pr.N, dm, pr.B, 0, xb, 0, 0, st, n))) return rc;
+    if ((rc = simt_map<T>(kt, Wk, kpvp, true, true, pr.k, dm, pr.H * pr.d, pr.B, ktb, 0, pr.d, 0, st, n))) return rc;
+    if ((rc = simt_map<T>(kt + (size_t)pr.B * ktb, Wv, kpvp, true, true, pr.k, dm, pr.H * pr.d, pr.B, ktb, 0, pr.d, pr.B,
+                          st, n))) return rc;
+    return simt_map<T>(Xq, Wq, qp, false, sizeof(T) == 4, pr.B * pr.N, dm, pr.H * pr.d, 1, 0, 0, 0, 0, st, n);
+  };
+  return run_pipeline_with<T>(pr, FL.L, ws, qp, W, out, st, tensor, tensor, tc, timer, /*keep_status=*/false, launches,
+                              stage1);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t flurka_fused_workspace_bytes(int variant, int B, int H, int N, int dm, int d, int k, int m) {
+  Problem pr;
+  if (parse_problem(variant | FLURKA_LAYOUT_BNHD, B, H, N, d, k, m, &pr) || dm <= 0) return 0;
+  return make_fused_layout(pr, dm).total;
+}
+
+int flurka_forward_fused(const void* Xq, const void* Xk, const void* Xv, const void* E, const void* F,
+                         const void* Wq, const void* Wk, const void* Wv, const void* W, int variant, int B, int H,
+                         int N, int dm, int d, int k, int m, void* out, void* stream) {
+  Problem pr;
+  if (variant & FLURKA_LAYOUT_BNHD) return FLURKA_ERR_VARIANT;        // the layout is fixed: out is [B,N,H,d]
+  int rc = parse_problem(variant | FLURKA_LAYOUT_BNHD, B, H, N, d, k, m, &pr);
+  if (rc) return rc;
+  if (dm <= 0 || dm > 16384) return FLURKA_ERR_SHAPE;
+  if (!Xq || !Xk || !Xv || !E || !F || !Wq || !Wk || !Wv || !out) return FLURKA_ERR_NULL;
+  if (pr.kernel == FLURKA_PERFORMER && !W) return FLURKA_ERR_NULL;
+  const void* ptrs[10] = {Xq, Xk, Xv, E, F, Wq, Wk, Wv, W, out};
+  for (const void* ptr : ptrs)
+    if (ptr && ((uintptr_t)ptr & 15)) return FLURKA_ERR_ALIGN;
+  const size_t xb = (size_t)B * N * dm * pr.esize(), ob = pr.qkv_elems() * pr.esize(),
+               eb = pr.ef_elems() * pr.esize(), mb = (size_t)dm * H * d * pr.esize(), wb = pr.w_elems() * pr.esize();
+  if (overlaps(out, ob, Xq, xb) || overlaps(out, ob, Xk, xb) || overlaps(out, ob, Xv, xb) || overlaps(out, ob, E, eb) ||
+      overlaps(out, ob, F, eb) || overlaps(out, ob, Wq, mb) || overlaps(out, ob, Wk, mb) || overlaps(out, ob, Wv, mb) ||
+      (W && wb && overlaps(out, ob, W, wb)))
+    return FLURKA_ERR_OVERLAP;
+  int path = g_path;
+  const bool tensor_ok = fused_tensor_ok(pr, dm);
+  if (path >= FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
+  if (path == FLURKA_PATH_AUTO) path = tensor_ok ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
+  if (path != FLURKA_PATH_TENSOR && path != FLURKA_PATH_SIMT) return FLURKA_ERR_VARIANT;   // no bisecting paths here
+  rc = check_device();
+  if (rc) return rc;
+  DeviceState& ds = dev_state();
+  const FusedLayout FL = make_fused_layout(pr, dm);
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = nullptr;
+  rc = get_workspace(ds, FL.total, st, &ws);
+  if (rc) return rc;
+  int launches = 0;
+  ds.timer.on = g_stage_timing;
+  StageTimer* timer = g_stage_timing ? &ds.timer : nullptr;
+  if (timer) {
+    rc = timer->create();
+    if (rc != cudaSuccess) return cuda_fail((cudaError_t)rc);
+  }
+  if (pr.fp32)
+    rc = fused_pipeline<float>(pr, dm, FL, ws, Xq, Xk, Xv, E, F, Wq, Wk, Wv, W, out, st, false, &ds.tc, timer, &launches);
+  else
+    rc = fused_pipeline<__nv_bfloat16>(pr, dm, FL, ws, Xq, Xk, Xv, E, F, Wq, Wk, Wv, W, out, st,
+                                       path == FLURKA_PATH_TENSOR, &ds.tc, timer, &launches);
+  if (rc) return rc;
+  ds.timer.have = g_stage_timing;
+  ds.last_path = path;
+  ds.last_launches = launches;
+  ds.have_last = true;
+  ds.last_problem = pr;
+  ds.last_ws = ws;
+  return FLURKA_OK;
+}
 
 // A loop of nothing but exponentials: eight independent ex2.approx chains per thread, every SM full.
 namespace {

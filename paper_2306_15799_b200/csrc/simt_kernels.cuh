@@ -304,4 +304,56 @@ simt_query_side(const T* __restrict__ Q, const T* __restrict__ W, const float* _
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The linear maps of Eq. (2) and the contraction of un-projected inputs on CUDA cores: a plain
+// batched C = A B with fp32 accumulation.  A: [Z][M][K] (batch stride a_stride, 0 = shared),
+// B: [Z][K][ncols] (b_stride likewise), both row-major.  grid = (ceil(ncols/32), ceil(M/32), Z),
+// block = 256 (a 32 x 32 tile of C, four rows per thread).
+// head_d == 0: C is [Z][M][ncols] row-major.  head_d > 0: C is the K', V' workspace, fp32
+// [(z0 + z) * ncols/head_d + col/head_d][M][head_d]: column block h of the product is head h's.
+// ---------------------------------------------------------------------------------------------
+template <typename TA, typename TB, typename TC>
+__global__ void __launch_bounds__(256)
+simt_linear_map(const TA* __restrict__ A, const TB* __restrict__ Bm, TC* __restrict__ C, int M, int K, int ncols,
+                size_t a_stride, size_t b_stride, int head_d, int z0) {
+  __shared__ float sa[32][33];
+  __shared__ float sb[32][33];
+  const int z = blockIdx.z;
+  const TA* Az = A + (size_t)z * a_stride;
+  const TB* Bz = Bm + (size_t)z * b_stride;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;      // ty: 0..7
+  const int row0 = blockIdx.y * 32, col0 = blockIdx.x * 32;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int k0 = 0; k0 < K; k0 += 32) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int ar = row0 + ty + 8 * r, ak = k0 + tx;
+      sa[ty + 8 * r][tx] = (ar < M && ak < K) ? to_f32(Az[(size_t)ar * K + ak]) : 0.f;
+      const int bk = k0 + ty + 8 * r, bc = col0 + tx;
+      sb[ty + 8 * r][tx] = (bk < K && bc < ncols) ? to_f32(Bz[(size_t)bk * ncols + bc]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int kk = 0; kk < 32; ++kk) {
+      const float b = sb[kk][tx];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[r] = fmaf(sa[ty + 8 * r][kk], b, acc[r]);
+    }
+    __syncthreads();
+  }
+  const int col = col0 + tx;
+  if (col >= ncols) return;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int row = row0 + ty + 8 * r;
+    if (row >= M) continue;
+    if (head_d > 0) {
+      const size_t head = (size_t)(z0 + z) * (ncols / head_d) + col / head_d;
+      store_out(C + (head * M + row) * head_d + col % head_d, acc[r]);
+    } else {
+      store_out(C + ((size_t)z * M + row) * ncols + col, acc[r]);
+    }
+  }
+}
+
 }  // namespace flurka

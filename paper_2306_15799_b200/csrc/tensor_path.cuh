@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <string.h>
 
+#include "k0_linear_maps.cuh"
 #include "k1_down_project.cuh"
 #include "k2_key_side.cuh"
 #include "k3_query_side.cuh"
@@ -87,6 +88,7 @@ inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int ran
 
 struct TensorMaps {
   CachedMap E, F, K, V, kpvp, Q, W, W2, aT, O;
+  CachedMap A3, Wk, Wv, Xq, Wq, Qp, kpvp2;      // the linear maps of the entry point with un-projected inputs
 };
 
 // Per-device context of the tensor-core kernels: the cached tensor maps (their pointers are device
@@ -95,6 +97,7 @@ struct TensorContext {
   TensorMaps maps;
   int sms = 0;
   bool k1_attr = false;
+  bool k0_attr = false;
   int sm_total() {
     if (!sms) {
       int dev = 0;
@@ -164,6 +167,93 @@ inline int launch_k1(TensorContext& tc, const void* K, const void* V, const void
   }
   const int grid = 2 * p.k_halves * p.col_groups * p.nsplit;
   k1_down_project<<<grid, kK1Threads, kK1SmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map, tm.kpvp.map, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
+
+// Forward declaration (defined below).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_after_predecessor(void (*fn)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
+                                            Args... args);
+
+inline int k0_set_attr(TensorContext& tc, int* cuda_err) {
+  if (!tc.k0_attr) {
+    cudaError_t e = cudaFuncSetAttribute(k0_linear_map, cudaFuncAttributeMaxDynamicSharedMemorySize, kK0SmemBytes);
+    if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+    tc.k0_attr = true;
+  }
+  return 0;
+}
+
+// ---- the linear maps on the k contracted rows: K', V' (fp32, [2][B*H][k][d], already zeroed) from
+//      kt = stage 1's output for the un-projected inputs ([2][B][dm/64][k][64] fp32)
+inline int launch_k0_key_value_maps(TensorContext& tc, const float* kt, __nv_bfloat16* a3, const void* Wk,
+                                    const void* Wv, float* kpvp, int B, int H, int dm, int d, int k, int* status,
+                                    cudaStream_t st, int* cuda_err) {
+  TensorMaps& tm = tc.maps;
+  {
+    const long long total = (long long)2 * B * k * (dm >> 2);
+    int grid = (int)((total + 255) / 256);
+    if (grid > tc.sm_total() * 8) grid = tc.sm_total() * 8;
+    cudaError_t e = launch_after_predecessor(k0_split_rows, grid, 256, 0, st, kt, a3, 2 * B, k, dm);
+    if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  }
+  const unsigned long long dA[3] = {(unsigned long long)3 * dm, (unsigned long long)k, (unsigned long long)2 * B};
+  const unsigned bA[3] = {64, 128, 1};
+  const unsigned long long dB[2] = {(unsigned long long)H * d, (unsigned long long)dm};
+  const unsigned bB[2] = {64, 64};
+  const unsigned long long dO[3] = {(unsigned long long)d, (unsigned long long)k, (unsigned long long)2 * B * H};
+  const unsigned bO[3] = {32, 32, 1};
+  if (!encode_map(&tm.A3, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, a3, dA, bA) ||
+      !encode_map(&tm.Wk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, Wk, dB, bB) ||
+      !encode_map(&tm.Wv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, Wv, dB, bB) ||
+      !encode_map(&tm.kpvp2, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 3, kpvp, dO, bO)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  K0Params p;
+  p.mode = 0; p.M = k; p.chunks = 3 * dm / 64; p.b_chunks = dm / 64; p.ncols = H * d; p.d = d; p.H = H;
+  p.Z = 2 * B; p.zb_shift = B;
+  p.row_blocks = (k + 255) / 256;
+  p.col_groups = (H * d + 255) / 256;
+  const int units = p.row_blocks * p.col_groups * p.Z;
+  p.nsplit = k1_choose_nsplit(tc.sm_count(), units, p.chunks);
+  p.status = status;
+  int rc = k0_set_attr(tc, cuda_err);
+  if (rc) return rc;
+  cudaError_t e = launch_after_predecessor(k0_linear_map, units * p.nsplit, kK0Threads, kK0SmemBytes, st, tm.A3.map,
+                                           tm.Wk.map, tm.Wv.map, tm.kpvp2.map, p);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  return 0;
+}
+
+// ---- the query map: Qp [B*N][H*d] bf16 = Xq [B*N][dm] Wq [dm][H*d]
+inline int launch_k0_query_map(TensorContext& tc, const void* Xq, const void* Wq, void* Qp, int B, int N, int H, int dm,
+                               int d, int* status, cudaStream_t st, int* cuda_err) {
+  TensorMaps& tm = tc.maps;
+  const unsigned long long dA[3] = {(unsigned long long)dm, (unsigned long long)B * N, 1ull};
+  const unsigned bA[3] = {64, 128, 1};
+  const unsigned long long dB[2] = {(unsigned long long)H * d, (unsigned long long)dm};
+  const unsigned bB[2] = {64, 64};
+  const unsigned long long dO[2] = {(unsigned long long)H * d, (unsigned long long)B * N};
+  const unsigned bO[2] = {64, 32};
+  if (!encode_map(&tm.Xq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Xq, dA, bA) ||
+      !encode_map(&tm.Wq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, Wq, dB, bB) ||
+      !encode_map(&tm.Qp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, Qp, dO, bO)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  K0Params p;
+  p.mode = 1; p.M = B * N; p.chunks = dm / 64; p.b_chunks = dm / 64; p.ncols = H * d; p.d = d; p.H = H;
+  p.Z = 1; p.zb_shift = 1; p.nsplit = 1;
+  p.row_blocks = (p.M + 255) / 256;
+  p.col_groups = (H * d + 255) / 256;
+  p.status = status;
+  int rc = k0_set_attr(tc, cuda_err);
+  if (rc) return rc;
+  k0_linear_map<<<p.row_blocks * p.col_groups, kK0Threads, kK0SmemBytes, st>>>(tm.Xq.map, tm.Wq.map, tm.Wq.map,
+                                                                               tm.Qp.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;

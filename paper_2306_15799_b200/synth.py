@@ -14,7 +14,7 @@ from __future__ import annotations
 
 import torch
 
-from .configs import PERFORMER, Workload
+from .configs import PERFORMER, FusedWorkload, Workload
 
 
 def _io_dtype(io: str) -> torch.dtype:
@@ -57,4 +57,30 @@ def make_inputs(w: Workload) -> dict:
         out["W"] = block_orthogonal_features(w.m, w.d, gen).to(dt)
     else:
         out["W"] = None
+    return out
+
+
+def make_fused_inputs(w: FusedWorkload) -> dict:
+    """CPU tensors for the entry point with un-projected inputs, drawn in the order Xq, Xk, Xv (one X when
+    `w.shared_x`), Wq, Wk, Wv, E, F, W:  X ~ N(0,1) [B,N,dm];  Wq, Wk, Wv ~ N(0, 1/dm) * d^(-1/4) [dm,H*d], so
+    that X W has the distribution make_inputs gives Q, K and V;  E, F, W as in make_inputs."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(w.seed)
+    dt = _io_dtype(w.io)
+
+    def draw(shape, s):
+        x = torch.randn(*shape, generator=gen, dtype=torch.float64)
+        return x.mul_(s).to(dt)
+
+    out = {}
+    if w.shared_x:
+        out["Xq"] = out["Xk"] = out["Xv"] = draw((w.B, w.N, w.dm), 1.0)
+    else:
+        for name in ("Xq", "Xk", "Xv"):
+            out[name] = draw((w.B, w.N, w.dm), 1.0)
+    for name in ("Wq", "Wk", "Wv"):
+        out[name] = draw((w.dm, w.H * w.d), float(w.dm) ** -0.5 * float(w.d) ** -0.25)
+    for name in ("E", "F"):
+        out[name] = draw((w.k, w.N), float(w.k) ** -0.5)
+    out["W"] = block_orthogonal_features(w.m, w.d, gen).to(dt) if w.variant == PERFORMER else None
     return out
