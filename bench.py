@@ -138,6 +138,14 @@ def job_tokens_per_s(w, world, ms_per_step):
     return w.tokens * world / (ms_per_step * 1e-3)
 
 
+def is_fused(w):
+    return isinstance(w, configs.FusedWorkload)
+
+
+def host_inputs(w):
+    return synth.make_fused_inputs(w) if is_fused(w) else synth.make_inputs(w)
+
+
 def oracle_sample(w, inputs, heads):
     """Times the fp64 oracle (as it stands) on `heads` heads of the workload. Returns seconds."""
     import oracle
@@ -147,7 +155,12 @@ def oracle_sample(w, inputs, heads):
     t0 = time.perf_counter()
     for i in range(heads):
         b, h = divmod(i % (w.B * w.H), w.H)
-        oracle.head(f64(inputs["Q"][b, h]), f64(inputs["K"][b, h]), f64(inputs["V"][b, h]), E, F, W, w.variant)
+        if is_fused(w):
+            cols = slice(h * w.d, (h + 1) * w.d)
+            oracle.fused_head(f64(inputs["Xq"][b]), f64(inputs["Xk"][b]), f64(inputs["Xv"][b]), E, F,
+                              f64(inputs["Wq"][:, cols]), f64(inputs["Wk"][:, cols]), f64(inputs["Wv"][:, cols]), W, w.variant)
+        else:
+            oracle.head(f64(inputs["Q"][b, h]), f64(inputs["K"][b, h]), f64(inputs["V"][b, h]), E, F, W, w.variant)
     return time.perf_counter() - t0
 
 
@@ -159,7 +172,7 @@ def run_reference(args, w):
     import oracle
     oracle.build()
     small = configs.shrink(w, B=1, H=1)          # one head per step; E, F, W keep their full size
-    inputs = synth.make_inputs(small)
+    inputs = host_inputs(small)
     for _ in range(args.warmup):
         oracle_sample(small, inputs, 1)
     t = 0.0
@@ -188,15 +201,20 @@ def measure(w, args, binding, rank, world, local, with_e2e=True):
 
     # every rank draws its own batch (weak scaling over B*H); same recipe, rank-offset seed
     wr = rank_workload(w, rank)
-    host = synth.make_inputs(wr)
+    host = host_inputs(wr)
+    fused = is_fused(w)
     laid_out = dict(host)
-    if args.layout == "bnhd":
+    if args.layout == "bnhd" and not fused:
         for n in ("Q", "K", "V"):
             laid_out[n] = host[n].transpose(1, 2).contiguous()
-    pinned = {n: (t.pin_memory() if t is not None else None) for n, t in laid_out.items()}
+    # one X serves as queries, keys and values when the workload says so: pinned, copied and counted once
+    names = [n for n in laid_out if not (fused and w.shared_x and n in ("Xk", "Xv"))]
+    pinned = {n: (laid_out[n].pin_memory() if laid_out[n] is not None else None) for n in names}
     dev = {n: (t.cuda(non_blocking=True) if t is not None else None) for n, t in pinned.items()}
-    out = torch.empty_like(dev["Q"])
-    in_bytes = sum(t.numel() * t.element_size() for t in dev.values() if t is not None)
+    if fused and w.shared_x:
+        dev["Xk"] = dev["Xv"] = dev["Xq"]
+    out = torch.empty((w.B, w.N, w.H, w.d), dtype=dev["E"].dtype, device="cuda") if fused else torch.empty_like(dev["Q"])
+    in_bytes = sum(t.numel() * t.element_size() for n, t in dev.items() if t is not None and n in names)
     flush = None
     if in_bytes < 2 * L2_BYTES:
         flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
@@ -204,8 +222,12 @@ def measure(w, args, binding, rank, world, local, with_e2e=True):
     torch.cuda.synchronize()
 
     def step():
-        binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant,
-                               out=out, stream=stream, layout=args.layout)
+        if fused:
+            binding.flurka_forward_fused(dev["Xq"], dev["Xk"], dev["Xv"], dev["E"], dev["F"], dev["Wq"], dev["Wk"],
+                                         dev["Wv"], dev["W"], w.variant, w.H, out=out, stream=stream)
+        else:
+            binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant,
+                                   out=out, stream=stream, layout=args.layout)
 
     def barrier():
         if world > 1:
@@ -262,15 +284,29 @@ def measure(w, args, binding, rank, world, local, with_e2e=True):
     # ---- end to end: host buffers in, host buffer out, through the host entry point
     res["e2e_ms"] = None
     if with_e2e:
-        host_out = torch.empty_like(pinned["Q"]).pin_memory()
+        host_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
         e2e_steps = max(1, min(args.steps, 5))
-        binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
-                                    w.variant, out=host_out, stream=stream, layout=args.layout)
+
+        def e2e_step():
+            if fused:
+                # the entry point with un-projected inputs takes device buffers: the copies are made here,
+                # on the launch stream, from and to pinned host memory
+                with torch.cuda.stream(stream):
+                    for n in names:
+                        if pinned[n] is not None:
+                            dev[n].copy_(pinned[n], non_blocking=True)
+                    step()
+                    host_out.copy_(out, non_blocking=True)
+                stream.synchronize()
+            else:
+                binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
+                                            w.variant, out=host_out, stream=stream, layout=args.layout)
+
+        e2e_step()
         barrier()
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
-            binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"],
-                                        w.variant, out=host_out, stream=stream, layout=args.layout)
+            e2e_step()
         torch.cuda.synchronize()
         res["e2e_ms"] = 1e3 * (time.perf_counter() - t0) / e2e_steps
     res["status"] = binding.flurka_last_status()
@@ -290,7 +326,15 @@ def stage_work(w):
             2 * BH * k * d * 4 + m * d * s + BH * p * (d * 2 + 4),
             2 * BH * N * d * s + m * d * s + BH * p * (d * 2 + 4)]
     exps = [0, k * p * BH, N * p * BH]
-    return ["down_projection", "key_side", "query_side"], flops, byts, exps
+    names = ["down_projection", "key_side", "query_side"]
+    if is_fused(w):
+        # stage 0 = contraction of the un-projected inputs and the three linear maps; its bytes: X, E, F, the
+        # maps, K' and V'; the query side then reads Xq W^Q from the workspace
+        dm, Hd = w.dm, w.H * w.d
+        names[0] = "contraction_and_linear_maps"
+        flops[0] = (4 * N * k * dm + 2 * N * dm * Hd + 4 * k * dm * Hd) * w.B
+        byts[0] = w.B * N * dm * s * (1 if w.shared_x else 3) + 2 * k * N * s + 3 * dm * Hd * s + 2 * BH * k * d * 4
+    return names, flops, byts, exps
 
 
 def rooflines(w, res, peaks, steps, world, exp_rate):
@@ -405,7 +449,7 @@ def main():
             "data": "synthetic",
             "config": {"workload": w.name, "variant": "performer" if w.variant == configs.PERFORMER else "rnn",
                        "B": w.B, "H": w.H, "N": w.N, "d": w.d, "k": w.k, "m": w.m, "io": w.io, "path": res["path"],
-                       "layout": args.layout,
+                       "layout": "bnhd" if is_fused(w) else args.layout, **({"dm": w.dm, "shared_x": w.shared_x} if is_fused(w) else {}),
                        "parallelism": "replicated batches over B*H, no collective" if world > 1 else "single GPU",
                        "l2": "inputs (%.0f MB) exceed L2" % (res["in_bytes"] / 1e6) if not res["flushed"]
                              else "L2 flushed between steps (252 MiB write)"},
