@@ -16,6 +16,8 @@
  *
  * Layout.  All tensors are dense, row-major, contiguous:
  *     Q, K, V, out : [B, H, N, d]      E, F : [k, N]      W : [m, d]
+ * (E, F: [H, k, N] with FLURKA_EF_PER_HEAD or-ed into `variant` -- Theorem 1 states the method with
+ * one projection pair E_i, F_i per head; they are still shared over the batch)
  * and share one element type per call: bfloat16 (default) or float32 (FLURKA_IO_FP32 or-ed into
  * `variant`).  Accumulation is fp32 in both cases.  With FLURKA_LAYOUT_BNHD or-ed into `variant`,
  * Q, K, V and out are [B, N, H, d] instead: the heads of one position side by side, which is how a
@@ -50,6 +52,7 @@ typedef enum {
 #define FLURKA_IO_BF16 0x000 /* default element type of Q, K, V, E, F, W, out */
 #define FLURKA_IO_FP32 0x100 /* or-ed into `variant`: all of them are float32 */
 #define FLURKA_LAYOUT_BNHD 0x200 /* or-ed into `variant`: Q, K, V, out are [B,N,H,d], not [B,H,N,d] */
+#define FLURKA_EF_PER_HEAD 0x400 /* or-ed into `variant`: E, F are [H,k,N], a pair E_i, F_i per head (Theorem 1) */
 
 typedef enum {
   FLURKA_OK = 0,
@@ -78,7 +81,7 @@ typedef enum {
  * flurka_forward -- the whole forward pass of Eq. (2) on DEVICE buffers, asynchronous on `stream`.
  *
  *   Q, K, V   device, [B,H,N,d]          E, F   device, [k,N]          W   device, [m,d] (NULL for RNN)
- *   variant   flurka_kernel_t | FLURKA_IO_BF16 / FLURKA_IO_FP32 [| FLURKA_LAYOUT_BNHD]
+ *   variant   flurka_kernel_t | FLURKA_IO_BF16 / FLURKA_IO_FP32 [| FLURKA_LAYOUT_BNHD] [| FLURKA_EF_PER_HEAD]
  *   out       device, [B,H,N,d], same element type
  *   stream    a cudaStream_t passed as void*; NULL is the default stream
  *

@@ -102,12 +102,13 @@ def version() -> int:
 
 
 LAYOUT_BNHD = 0x200   # or-ed into the variant word: Q, K, V, out are [B,N,H,d]
+EF_PER_HEAD = 0x400   # or-ed into the variant word: E, F are [H,k,N], one pair per head
 
 
-def _variant_word(variant: int, dtype: torch.dtype, layout: str = "bhnd") -> int:
+def _variant_word(variant: int, dtype: torch.dtype, layout: str = "bhnd", ef_per_head: bool = False) -> int:
     if layout not in ("bhnd", "bnhd"):
         raise ValueError("flurka: layout must be 'bhnd' or 'bnhd'")
-    word = variant | (LAYOUT_BNHD if layout == "bnhd" else 0)
+    word = variant | (LAYOUT_BNHD if layout == "bnhd" else 0) | (EF_PER_HEAD if ef_per_head else 0)
     if dtype == torch.bfloat16:
         return word | IO_BF16
     if dtype == torch.float32:
@@ -129,9 +130,9 @@ def _check(Q, K, V, E, F, W, variant, out, device_type, layout="bhnd"):
         B, N, H, d = Q.shape
     else:
         B, H, N, d = Q.shape
-    if E.dim() != 2 or E.shape[1] != N or F.shape != E.shape:
-        raise ValueError("flurka: E, F must be [k,N]")
-    k = E.shape[0]
+    if F.shape != E.shape or E.shape[-1] != N or not (E.dim() == 2 or (E.dim() == 3 and E.shape[0] == H)):
+        raise ValueError("flurka: E, F must be [k,N], or [H,k,N] with one pair per head")
+    k = E.shape[-2]
     m = 0
     if variant == PERFORMER:
         if W is None or W.dim() != 2 or W.shape[1] != d or W.dtype != Q.dtype or not W.is_contiguous() \
@@ -155,7 +156,7 @@ def flurka_forward(Q, K, V, E, F, W, variant, out=None, stream=None, layout="bhn
     B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cuda", layout)
     rc = load().flurka_forward(
         Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
-        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, layout),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, layout, E.dim() == 3),
         B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
     if rc:
         raise FlurkaError(rc, "flurka_forward")
@@ -169,7 +170,7 @@ def flurka_forward_host(Q, K, V, E, F, W, variant, out=None, stream=None, layout
     B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cpu", layout)
     rc = load().flurka_forward_host(
         Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
-        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, layout),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, layout, E.dim() == 3),
         B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
     if rc:
         raise FlurkaError(rc, "flurka_forward_host")
@@ -294,7 +295,7 @@ def flurka_forward_static_scratch(Q, K, V, E, F, W, variant, out, stream=None):
     B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, out, "cuda")
     rc = load().flurka_forward_static_scratch(
         Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
-        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype),
+        W.data_ptr() if W is not None else None, _variant_word(variant, Q.dtype, "bhnd", E.dim() == 3),
         B, H, N, d, k, m, out.data_ptr(), _stream_ptr(stream))
     if rc:
         raise FlurkaError(rc, "flurka_forward_static_scratch")

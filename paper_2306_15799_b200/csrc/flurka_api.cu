@@ -18,13 +18,15 @@ struct Problem {
   int kernel;      // FLURKA_PERFORMER / FLURKA_RNN
   bool fp32;       // element type of the I/O tensors
   bool bnhd;       // Q, K, V, out are [B,N,H,d] (heads merged into the row) instead of [B,H,N,d]
+  bool ef_per_head;  // E, F are [H,k,N]: one pair per head, shared over the batch
   int B, H, N, d, k, m;
   int seq_major_heads() const { return bnhd ? H : 0; }   // what head_view() takes
+  int ef_heads() const { return ef_per_head ? H : 0; }
   int BH() const { return B * H; }
   int p() const { return kernel == FLURKA_PERFORMER ? m : d; }   // feature dimension
   size_t esize() const { return fp32 ? 4 : 2; }
   size_t qkv_elems() const { return (size_t)B * H * N * d; }
-  size_t ef_elems() const { return (size_t)k * N; }
+  size_t ef_elems() const { return (size_t)k * N * (ef_per_head ? H : 1); }
   size_t w_elems() const { return kernel == FLURKA_PERFORMER ? (size_t)m * d : 0; }
 };
 
@@ -113,7 +115,7 @@ int parse_problem(int variant, int B, int H, int N, int d, int k, int m, Problem
   const int io = variant & 0x100;
   const int layout = variant & 0x200;
   if (kernel != FLURKA_PERFORMER && kernel != FLURKA_RNN) return FLURKA_ERR_VARIANT;
-  if (variant & ~0x3ff) return FLURKA_ERR_VARIANT;
+  if (variant & ~0x7ff) return FLURKA_ERR_VARIANT;
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || k <= 0) return FLURKA_ERR_SHAPE;
   if (d > 128 || k > 4096) return FLURKA_ERR_SHAPE;
   if (kernel == FLURKA_PERFORMER && m <= 0) return FLURKA_ERR_SHAPE;
@@ -121,6 +123,7 @@ int parse_problem(int variant, int B, int H, int N, int d, int k, int m, Problem
   pr->kernel = kernel;
   pr->fp32 = io == FLURKA_IO_FP32;
   pr->bnhd = layout == FLURKA_LAYOUT_BNHD;
+  pr->ef_per_head = (variant & FLURKA_EF_PER_HEAD) != 0;
   pr->B = B; pr->H = H; pr->N = N; pr->d = d; pr->k = k;
   pr->m = kernel == FLURKA_PERFORMER ? m : 0;
   return FLURKA_OK;
@@ -192,7 +195,8 @@ int launch_simt_down_project(const Problem& pr, const void* K, const void* V, co
   nsplit = (pr.N + chunk - 1) / chunk;
   dim3 grid(jt, pr.BH(), 2 * nsplit);
   simt_down_project<T><<<grid, 256, 0, st>>>((const T*)K, (const T*)V, (const T*)E, (const T*)F, kpvp,
-                                            pr.BH(), pr.N, pr.d, pr.k, nsplit, chunk, pr.seq_major_heads());
+                                            pr.BH(), pr.N, pr.d, pr.k, nsplit, chunk, pr.seq_major_heads(),
+                                            pr.ef_heads());
   ++*launches;
   return FLURKA_OK;
 }
@@ -295,7 +299,8 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
   auto stage1 = [&](float* kpvp, int* status, int* n) -> int {
     if (tc1) {
       int cuda_err = 0;
-      int rc = launch_k1(*tc, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err);
+      int rc = launch_k1(*tc, K, V, E, F, kpvp, pr.BH(), pr.seq_major_heads(), pr.N, pr.d, pr.k, status, st, &cuda_err,
+                         pr.ef_heads());
       if (rc) { g_last_cuda_error = cuda_err; return rc; }
       ++*n;
       return FLURKA_OK;
@@ -426,8 +431,10 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
   // The heads are independent, so the call works through them in up to eight groups: while the
   // inputs of one group travel to the device, the output of the group before travels back on a second
   // stream (the link is full duplex), and the compute of a group hides under the copies.
-  // (units that are contiguous in memory: heads for [B,H,N,d], batches for [B,N,H,d])
-  const int heads = pr.bnhd ? pr.B : pr.BH();
+  // (units that are contiguous in memory: heads for [B,H,N,d], batches for [B,N,H,d]; whole batches
+  // also when every head has its own E, F, so that a group's heads keep their numbers)
+  const bool by_batch = pr.bnhd || pr.ef_per_head;
+  const int heads = by_batch ? pr.B : pr.BH();
   int groups = (int)std::min<size_t>(8, qn >> 20);           // at least 1 MiB of Q per group
   groups = std::max(1, std::min(groups, heads));
   if (groups > 1 && !ds.out_stream) {
@@ -443,10 +450,10 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
   for (int gi = 0; gi < groups; ++gi) {
     const int cnt = (int)((long long)heads * (gi + 1) / groups) - (int)((long long)heads * gi / groups);
     Problem sub = pr;
-    if (pr.bnhd) sub.B = cnt; else { sub.B = 1; sub.H = cnt; }
+    if (by_batch) sub.B = cnt; else { sub.B = 1; sub.H = cnt; }
     reserve = std::max(reserve, make_layout(sub).total);
   }
-  const size_t head_bytes = (size_t)N * d * pr.esize() * (pr.bnhd ? H : 1);
+  const size_t head_bytes = (size_t)N * d * pr.esize() * (by_batch ? H : 1);
   rc = FLURKA_OK;
   for (int gi = 0; gi < groups && rc == FLURKA_OK; ++gi) {
     const int h0 = (int)((long long)heads * gi / groups), h1 = (int)((long long)heads * (gi + 1) / groups);
@@ -457,8 +464,8 @@ int flurka_forward_host(const void* Q, const void* K, const void* V, const void*
       rc = cuda_fail(e);
       break;
     }
-    rc = forward_device(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, pr.bnhd ? h1 - h0 : 1,
-                        pr.bnhd ? H : h1 - h0, N, d, k, m, dO + off, stream, /*keep_status=*/gi > 0, reserve);
+    rc = forward_device(dQ + off, dK + off, dV + off, dE, dF, wn ? dW : nullptr, variant, by_batch ? h1 - h0 : 1,
+                        by_batch ? H : h1 - h0, N, d, k, m, dO + off, stream, /*keep_status=*/gi > 0, reserve);
     if (rc) break;
     if (groups == 1) {
       if ((e = cudaMemcpyAsync(out, dO, qn, cudaMemcpyDeviceToHost, st)) != cudaSuccess) rc = cuda_fail(e);
@@ -680,7 +687,8 @@ int flurka_forward_fused(const void* Xq, const void* Xk, const void* Xv, const v
                          const void* Wq, const void* Wk, const void* Wv, const void* W, int variant, int B, int H,
                          int N, int dm, int d, int k, int m, void* out, void* stream) {
   Problem pr;
-  if (variant & FLURKA_LAYOUT_BNHD) return FLURKA_ERR_VARIANT;        // the layout is fixed: out is [B,N,H,d]
+  // the layout is fixed (out is [B,N,H,d]); the contraction is shared by all heads, so E, F cannot be per head
+  if (variant & (FLURKA_LAYOUT_BNHD | FLURKA_EF_PER_HEAD)) return FLURKA_ERR_VARIANT;
   int rc = parse_problem(variant | FLURKA_LAYOUT_BNHD, B, H, N, d, k, m, &pr);
   if (rc) return rc;
   if (dm <= 0 || dm > 16384) return FLURKA_ERR_SHAPE;

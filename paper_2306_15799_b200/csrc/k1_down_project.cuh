@@ -2,8 +2,8 @@
 // a contraction over the sequence axis, split across CTAs along that axis.
 //
 // One CTA owns: one of the two projections (t), up to 256 rows of the projection matrix (two
-// 128-row MMA tiles), 256 output columns = 256/d consecutive heads, and a contiguous range of
-// 64-wide sequence chunks.  Per chunk TMA brings a [rows x 64] slab of E (K-major, the sequence is
+// 128-row MMA tiles), 256 output columns = 256/d consecutive heads (one head when every head has its
+// own E_i, F_i, as Theorem 1 writes them), and a contiguous range of 64-wide sequence chunks.  Per chunk TMA brings a [rows x 64] slab of E (K-major, the sequence is
 // contiguous) and, per 64 columns, a [64 x 64] slab of K or V (MN-major: the head dimension is
 // contiguous, the contracted sequence index is the slow one), both 128-byte swizzled.  A single
 // thread issues tcgen05.mma (M=128, N=ncols, K=16) into fp32 TMEM accumulators; when the range is
@@ -18,8 +18,10 @@ namespace flurka {
 struct K1Params {
   int N, d, k, BH;
   int H;           // > 0: K, V are [B,N,H,d] (the tensor map has rows of H*d elements); 0: [B,H,N,d]
+  int ef_heads;    // > 0: E, F are [ef_heads][k][N], one pair per head (Theorem 1's E_i, F_i); a CTA then owns ONE head
+  int group_cols;  // output columns per CTA: 256 (= 256/d heads sharing an E tile), or d with per-head E, F
   int nsplit;      // CTAs along the sequence
-  int col_groups;  // ceil(BH * d / 256)
+  int col_groups;  // ceil(BH * d / group_cols)
   int k_halves;    // ceil(k / 256)
   int* status;
 };
@@ -55,7 +57,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
   const int rows = min(256, p.k - kh * 256);
   const int mt = (rows + 127) >> 7;                         // MMA M-tiles (1 or 2)
   const int total_cols = p.BH * p.d;
-  const int ncols = min(256, total_cols - cg * 256);        // multiple of 64
+  const int ncols = min(p.group_cols, total_cols - cg * p.group_cols);   // multiple of 64
   const int nb = ncols >> 6;                                // 64-column slabs
   const int chunks_total = (p.N + 63) >> 6;                 // a ragged last chunk is zero-filled by TMA
   const int c_begin = (int)(((long long)s * chunks_total) / p.nsplit);
@@ -106,9 +108,11 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
         const uint32_t b_dst = a_dst + 32768;
         const int n0 = (c_begin + it) << 6;
         mbar_arrive_expect_tx(bar_full + 8 * st, tx_bytes);
-        for (int m = 0; m < mt; ++m) tma_load_2d(a_dst + m * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + m * 128);
+        // with per-head E, F this CTA's head is cg (its group is one head wide); E_i is shared over the batch
+        const int ez = p.ef_heads > 0 ? cg % p.ef_heads : 0;
+        for (int m = 0; m < mt; ++m) tma_load_3d(a_dst + m * 16384, tmP, bar_full + 8 * st, n0, kh * 256 + m * 128, ez);
         for (int b = 0; b < nb; ++b) {
-          const int slab = cg * 4 + b;                       // global 64-column slab index
+          const int slab = cg * (p.group_cols >> 6) + b;     // global 64-column slab index
           const int head = slab / dblocks, dc = slab % dblocks;
           if (p.H > 0) tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, (head % p.H) * p.d + dc * 64, n0, head / p.H);
           else tma_load_3d(b_dst + b * 8192, tmX, bar_full + 8 * st, dc * 64, n0, head);
@@ -171,7 +175,7 @@ k1_down_project(const __grid_constant__ CUtensorMap tmE, const __grid_constant__
           if (lane == 0) {
             if (row0 < p.k) {
               for (int cc = 0; cc < ncc; ++cc) {
-                const int col = cg * 256 + cc * 32;
+                const int col = cg * p.group_cols + cc * 32;
                 const int head = col / p.d, c0 = col % p.d;
                 tma_reduce_add_3d(&tmOut, stage_buf + cc * 4096, c0, row0, t * p.BH + head);
               }

@@ -47,13 +47,13 @@ __device__ __forceinline__ void store_out(__nv_bfloat16* p, float v) { *p = __fl
 // Stage 1.  grid = (ceil(k/32), B*H, 2*nsplit); block = 256.
 // blockIdx.z = t*nsplit + s: t = 0 projects K with E, t = 1 projects V with F; split s covers the
 // sequence range [s*chunk, min(N,(s+1)*chunk)).  Partial sums are added into KpVp (zeroed before).
-// KpVp layout: [2][B*H][k][d] fp32.
+// KpVp layout: [2][B*H][k][d] fp32.  E, F: [k][N] shared by all heads, or [H][k][N] (ef_heads = H).
 // ---------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
 simt_down_project(const T* __restrict__ Kin, const T* __restrict__ Vin, const T* __restrict__ E,
                   const T* __restrict__ F, float* __restrict__ KpVp, int BH, int N, int d, int k,
-                  int nsplit, int chunk, int seq_major_heads) {
+                  int nsplit, int chunk, int seq_major_heads, int ef_heads) {
   constexpr int TJ = 32, TN = 32;
   __shared__ float Ps[TJ][TN + 1];
   __shared__ float Xs[TN][128];
@@ -62,7 +62,8 @@ simt_down_project(const T* __restrict__ Kin, const T* __restrict__ Vin, const T*
   const int s = blockIdx.z % nsplit;
   const int bh = blockIdx.y;
   const int j0 = blockIdx.x * TJ;
-  const T* __restrict__ P = t ? F : E;
+  // ef_heads > 0: E and F are [ef_heads][k][N], one pair per head (head = bh % ef_heads)
+  const T* __restrict__ P = (t ? F : E) + (ef_heads > 0 ? (size_t)(bh % ef_heads) * k * N : 0);
   const HeadView hv = head_view(bh, seq_major_heads, N, d);
   const T* __restrict__ X = (t ? Vin : Kin) + hv.base;
   float* __restrict__ out = KpVp + ((size_t)t * BH + bh) * (size_t)k * d;

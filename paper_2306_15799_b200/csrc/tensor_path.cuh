@@ -135,19 +135,22 @@ inline int k1_choose_nsplit(int sms, int units, int chunks) {
 
 // ---- stage 1: K' = E K, V' = F V into kpvp (already zeroed) ----------------------------------
 // H > 0: K, V are [B,N,H,d] (H heads merged into the row); H == 0: [B,H,N,d]
+// ef_heads > 0: E, F are [ef_heads][k][N] (one pair per head; head index = bh % ef_heads)
 inline int launch_k1(TensorContext& tc, const void* K, const void* V, const void* E, const void* F, float* kpvp,
-                     int BH, int H, int N, int d, int k, int* status, cudaStream_t st, int* cuda_err) {
+                     int BH, int H, int N, int d, int k, int* status, cudaStream_t st, int* cuda_err,
+                     int ef_heads = 0) {
   TensorMaps& tm = tc.maps;
-  const unsigned long long dE[2] = {(unsigned long long)N, (unsigned long long)k};
-  const unsigned bE[2] = {64, 128};
+  const unsigned long long dE[3] = {(unsigned long long)N, (unsigned long long)k,
+                                    (unsigned long long)(ef_heads > 0 ? ef_heads : 1)};
+  const unsigned bE[3] = {64, 128, 1};
   // [B,N,H,d] is a 3-D tensor too: rows of H*d elements, head h at columns h*d .. h*d+d-1
   const unsigned long long dX[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
                                     (unsigned long long)(H > 0 ? BH / H : BH)};
   const unsigned bX[3] = {64, 64, 1};
   const unsigned long long dO[3] = {(unsigned long long)d, (unsigned long long)k, (unsigned long long)2 * BH};
   const unsigned bO[3] = {32, 32, 1};
-  if (!encode_map(&tm.E, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, E, dE, bE) ||
-      !encode_map(&tm.F, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, F, dE, bE) ||
+  if (!encode_map(&tm.E, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, E, dE, bE) ||
+      !encode_map(&tm.F, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, F, dE, bE) ||
       !encode_map(&tm.K, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, K, dX, bX) ||
       !encode_map(&tm.V, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, V, dX, bX) ||
       !encode_map(&tm.kpvp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 3, kpvp, dO, bO)) {
@@ -156,7 +159,9 @@ inline int launch_k1(TensorContext& tc, const void* K, const void* V, const void
   }
   K1Params p;
   p.N = N; p.d = d; p.k = k; p.BH = BH; p.H = H;
-  p.col_groups = (BH * d + 255) / 256;
+  p.ef_heads = ef_heads;
+  p.group_cols = ef_heads > 0 ? d : 256;
+  p.col_groups = (BH * d + p.group_cols - 1) / p.group_cols;
   p.k_halves = (k + 255) / 256;
   p.nsplit = k1_choose_nsplit(tc.sm_count(), 2 * p.col_groups * p.k_halves, (N + 63) / 64);
   p.status = status;

@@ -53,7 +53,7 @@ def test_argument_checks_need_no_device(lib):
 
     assert call(Q=None) == -1 and call(out=None) == -1 and call(W=None) == -1
     assert call(W=None, variant=1) in (-7, 0)          # RNN needs no W; only the device is missing
-    assert call(variant=7) == -2 and call(variant=0x400) == -2
+    assert call(variant=7) == -2 and call(variant=0x800) == -2
     assert call(variant=0x200) in (-7, 0)              # [B,N,H,d] layout flag is valid
     assert call(N=0) == -3 and call(d=129) == -3 and call(k=0) == -3 and call(m=0) == -3 and call(k=5000) == -3
     assert call(B=70000) == -3

@@ -6,6 +6,7 @@ import torch
 from paper_2306_15799_b200 import binding, build, configs, synth
 from paper_2306_15799_b200.configs import PERFORMER, RNN, Workload
 
+import oracle
 import parity_util as pu
 
 pytestmark = pytest.mark.gpu
@@ -323,3 +324,59 @@ def test_heads_merged_into_the_row_host_entry():
     for b in range(w.B):
         for h in range(w.H):
             pu.assert_close(got[b, h], pu.oracle_head(inputs, w, b, h), "bf16", "host, head (%d,%d)" % (b, h))
+
+
+# ----------------------------------------------------------------------------- one E_i, F_i per head
+def _per_head_inputs(w):
+    """The workload's inputs with E, F redrawn as [H,k,N]: one projection pair per head (Theorem 1)."""
+    x = synth.make_inputs(w)
+    gen = torch.Generator().manual_seed(w.seed + 17)
+    for name in ("E", "F"):
+        x[name] = (torch.randn(w.H, w.k, w.N, generator=gen, dtype=torch.float64) * float(w.k) ** -0.5).to(x["Q"].dtype)
+    return x
+
+
+def _check_per_head(w, x, out):
+    f64 = lambda t: t.double().numpy()
+    W = f64(x["W"]) if x["W"] is not None else None
+    got = out.cpu().double().numpy()
+    for b in range(w.B):
+        for h in range(w.H):
+            ref = oracle.head(f64(x["Q"][b, h]), f64(x["K"][b, h]), f64(x["V"][b, h]), f64(x["E"][h]), f64(x["F"][h]),
+                              W, w.variant)
+            pu.assert_close(got[b, h], ref, w.io, "%s per-head E, F, head (%d,%d)" % (w.name, b, h))
+
+
+PER_HEAD_CASES = [
+    (_wl("ph_simt_perf_fp32", PERFORMER, "fp32", 2, 3, 200, 24, 20, 40, 81), binding.PATH_SIMT),
+    (_wl("ph_simt_rnn_bf16", RNN, "bf16", 1, 2, 264, 64, 40, 0, 82), binding.PATH_SIMT),
+    (_wl("ph_tensor_perf_d64", PERFORMER, "bf16", 2, 3, 1024, 64, 128, 128, 83), binding.PATH_TENSOR),
+    (_wl("ph_tensor_perf_d128_k512", PERFORMER, "bf16", 1, 2, 768, 128, 512, 256, 84), binding.PATH_TENSOR),
+    (_wl("ph_tensor_rnn", RNN, "bf16", 2, 2, 1000, 64, 64, 0, 85), binding.PATH_TENSOR),
+]
+
+
+@pytest.mark.parametrize("w,path", PER_HEAD_CASES, ids=lambda v: v.name if hasattr(v, "name") else str(v))
+def test_per_head_projections(w, path):
+    import oracle  # noqa: F401
+    x = _per_head_inputs(w)
+    out = pu.run_gpu(w, x, path)
+    assert binding.flurka_last_path() == path
+    _check_per_head(w, x, out)
+
+
+def test_per_head_projections_seq_major_and_host_entry():
+    """[B,N,H,d] tensors with one E_i, F_i per head, and the host entry point, whose head groups must be
+    whole batches so that every head keeps its own pair."""
+    w = _wl("ph_host", PERFORMER, "bf16", 3, 4, 2048, 64, 128, 128, 86)
+    x = _per_head_inputs(w)
+    dev = pu.to_device(x)
+    t = lambda a: a.transpose(1, 2).contiguous()
+    out = binding.flurka_forward(t(dev["Q"]), t(dev["K"]), t(dev["V"]), dev["E"], dev["F"], dev["W"], w.variant, layout="bnhd")
+    torch.cuda.synchronize()
+    assert binding.flurka_last_status() == 0
+    _check_per_head(w, x, out.transpose(1, 2))
+    pinned = {n: (a.pin_memory() if a is not None else None) for n, a in x.items()}
+    host_out = binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"], w.variant)
+    assert binding.flurka_last_status() == 0
+    _check_per_head(w, x, host_out)
