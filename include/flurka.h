@@ -141,6 +141,31 @@ int flurka_forward_fused(const void* Xq, const void* Xk, const void* Xv, const v
                          int N, int dm, int d, int k, int m, void* out, void* stream);
 size_t flurka_fused_workspace_bytes(int variant, int B, int H, int N, int dm, int d, int k, int m);
 
+/*
+ * A forward pass sharded over the SEQUENCE (several GPUs, each holding a slice of the positions; the
+ * paper's own runs spread a model over four GPUs, Section 4).  K' = E K and V' = F V (Eq. (2)) are sums
+ * over positions, so a shard computes its part from its slice of K, V and the matching COLUMNS of E, F,
+ * the parts are added over the shards, and everything after is local to a shard's queries:
+ *
+ *   flurka_forward_partial   K, V: device [B,H,n,d] (or [B,n,H,d]), the shard's n positions; E, F: device
+ *                            [k,n], the matching columns as a dense matrix.  Leaves this shard's part of
+ *                            K', V' in the workspace (fp32, [2][B*H][k][d]).
+ *   flurka_partial_sums      Where that block is (device pointer, bytes).  The CALLER adds it over the
+ *                            shards in place -- an all-reduce (sum) of that many bytes, e.g. NCCL on the
+ *                            same stream -- which is the only exchange between the GPUs.
+ *   flurka_forward_finish    Q: device, the shard's queries (n may differ from the first call's), W, out:
+ *                            the key side and the query side on the summed K', V'.
+ *
+ * Variant word, shape limits, alignment, streams and errors as for flurka_forward; the three calls use
+ * the current device's workspace, so nothing else may run on it in between.  flurka_forward_finish
+ * returns FLURKA_ERR_WORKSPACE when no matching flurka_forward_partial came before it.
+ */
+int flurka_forward_partial(const void* K, const void* V, const void* E, const void* F, int variant, int B, int H,
+                           int N, int d, int k, int m, void* stream);
+int flurka_partial_sums(void** dev_ptr, size_t* bytes);
+int flurka_forward_finish(const void* Q, const void* W, int variant, int B, int H, int N, int d, int k, int m,
+                          void* out, void* stream);
+
 /* Bytes of device scratch flurka_forward needs for this problem (0 on invalid arguments). Holds the
  * fp32 projections K', V' (Eq. (2)'s E K and F V), the key-side feature summaries and a status word. */
 size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m);

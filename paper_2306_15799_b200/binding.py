@@ -22,6 +22,7 @@ EXPORTS = [
     "flurka_last_status", "flurka_last_cuda_error", "flurka_set_stage_timing", "flurka_last_stage_ms",
     "flurka_strerror", "flurka_version", "flurka_forward_static_scratch", "flurka_static_scratch_need",
     "flurka_measure_ex2_rate", "flurka_forward_fused", "flurka_fused_workspace_bytes",
+    "flurka_forward_partial", "flurka_partial_sums", "flurka_forward_finish",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -87,6 +88,12 @@ def load() -> ctypes.CDLL:
     lib.flurka_forward_fused.argtypes = [vp] * 9 + [ci] * 8 + [vp, vp]
     lib.flurka_fused_workspace_bytes.restype = sz
     lib.flurka_fused_workspace_bytes.argtypes = [ci] * 8
+    lib.flurka_forward_partial.restype = ci
+    lib.flurka_forward_partial.argtypes = [vp] * 4 + [ci] * 7 + [vp]
+    lib.flurka_forward_finish.restype = ci
+    lib.flurka_forward_finish.argtypes = [vp, vp] + [ci] * 7 + [vp, vp]
+    lib.flurka_partial_sums.restype = ci
+    lib.flurka_partial_sums.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(sz)]
     lib.flurka_measure_ex2_rate.restype = ci
     lib.flurka_measure_ex2_rate.argtypes = [ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -205,6 +212,67 @@ def flurka_forward_fused(Xq, Xk, Xv, E, F, Wq, Wk, Wv, W, variant, H, out=None, 
         B, H, N, dm, d, k, m, out.data_ptr(), _stream_ptr(stream))
     if rc:
         raise FlurkaError(rc, "flurka_forward_fused")
+    return out
+
+
+class _DeviceBlock:
+    """A block of library-owned device memory, presented through the CUDA array interface."""
+
+    def __init__(self, ptr: int, n_floats: int):
+        self.__cuda_array_interface__ = {"shape": (n_floats,), "typestr": "<f4", "data": (ptr, False), "version": 3,
+                                         "strides": None}
+
+
+def flurka_forward_partial(K, V, E, F, variant, m=0, stream=None, layout="bhnd"):
+    """First half of a sequence-sharded forward: this shard's part of K' = E K, V' = F V.
+    K, V: the shard's positions [B,H,n,d]; E, F: the matching columns [k,n] (dense)."""
+    if layout == "bnhd":
+        B, N, H, d = K.shape
+    else:
+        B, H, N, d = K.shape
+    for name, t in (("K", K), ("V", V), ("E", E), ("F", F)):
+        if t.device.type != "cuda" or not t.is_contiguous() or t.dtype != K.dtype:
+            raise ValueError("flurka: %s must be a contiguous CUDA tensor of K's dtype" % name)
+    if V.shape != K.shape or F.shape != E.shape or E.shape[-1] != N:
+        raise ValueError("flurka: K, V must be alike and E, F [k,n] with n the slice length")
+    rc = load().flurka_forward_partial(K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(),
+                                       _variant_word(variant, K.dtype, layout, E.dim() == 3), B, H, N, d, E.shape[-2], m,
+                                       _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_forward_partial")
+
+
+def flurka_partial_sums():
+    """The fp32 block [2][B*H][k][d] the last flurka_forward_partial left on this device, as a flat CUDA
+    tensor that aliases the library's workspace (add it over the shards in place)."""
+    ptr, n = ctypes.c_void_p(), ctypes.c_size_t()
+    rc = load().flurka_partial_sums(ctypes.byref(ptr), ctypes.byref(n))
+    if rc:
+        raise FlurkaError(rc, "flurka_partial_sums")
+    return torch.as_tensor(_DeviceBlock(ptr.value, n.value // 4), device="cuda")
+
+
+def flurka_forward_finish(Q, W, variant, k, out=None, stream=None, layout="bhnd"):
+    """Second half: key side and query side for this shard's queries on the summed K', V'."""
+    if out is None:
+        out = torch.empty_like(Q)
+    if layout == "bnhd":
+        B, N, H, d = Q.shape
+    else:
+        B, H, N, d = Q.shape
+    if Q.device.type != "cuda" or not Q.is_contiguous() or out.shape != Q.shape or out.dtype != Q.dtype \
+            or not out.is_contiguous():
+        raise ValueError("flurka: Q and out must be contiguous CUDA tensors of one shape and dtype")
+    m = 0
+    if variant == PERFORMER:
+        if W is None or W.dim() != 2 or W.shape[1] != d or W.dtype != Q.dtype or not W.is_contiguous():
+            raise ValueError("flurka: W must be a contiguous [m,d] tensor like Q")
+        m = W.shape[0]
+    rc = load().flurka_forward_finish(Q.data_ptr(), W.data_ptr() if W is not None else None,
+                                      _variant_word(variant, Q.dtype, layout), B, H, N, d, k, m, out.data_ptr(),
+                                      _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_forward_finish")
     return out
 
 

@@ -75,6 +75,7 @@ struct DeviceState {
   int last_launches = 0;
   // most recent forward (for flurka_debug_copy / flurka_last_status)
   bool have_last = false;
+  bool partial_pending = false;        // the last call was the first half of a sequence-sharded forward
   Problem last_problem{};
   char* last_ws = nullptr;
   // host-buffer entry point: device staging
@@ -249,7 +250,9 @@ int key_side_dispatch(const Problem& pr, const float* kpvp, const void* W, float
 template <typename T, typename Stage1>
 int run_pipeline_with(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* W, void* out,
                       cudaStream_t st, bool tc2, bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status,
-                      int* launches, Stage1&& stage1) {
+                      int* launches, Stage1&& stage1, int phases = 3) {
+  // phases: bit 0 = clear the accumulators and run stage 1, bit 1 = run stages 2 and 3 (a sequence-sharded
+  // forward does the two halves in separate calls, with the sum over the shards in between)
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
   float* a32 = (float*)(ws + L.a32);
@@ -259,12 +262,20 @@ int run_pipeline_with(const Problem& pr, const Layout& L, char* ws, const void* 
   int cuda_err = 0;
   // one memset: the status words, the arrival counters and the K', V' accumulators the kernels add into
   const size_t clear_from = L.status + (keep_status ? 16 : 0);
-  cudaError_t e = cudaMemsetAsync(ws + clear_from, 0, L.kpvp_end - clear_from, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  if (timer) timer->mark(0, st);
-  int rc = stage1(kpvp, status, launches);
-  if (rc) return rc;
-  if (timer) timer->mark(1, st);
+  cudaError_t e = cudaSuccess;
+  int rc = FLURKA_OK;
+  if (phases & 1) {
+    e = cudaMemsetAsync(ws + clear_from, 0, L.kpvp_end - clear_from, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (timer) timer->mark(0, st);
+    rc = stage1(kpvp, status, launches);
+    if (rc) return rc;
+    if (timer) timer->mark(1, st);
+  }
+  if (!(phases & 2)) {
+    e = cudaGetLastError();
+    return e == cudaSuccess ? FLURKA_OK : cuda_fail(e);
+  }
   if (tc2) {
     float* part = L.total > L.part ? (float*)(ws + L.part) : nullptr;
     rc = launch_k2(*tc, performer, kpvp, W, weight, aT16, part, status + 4, pr.BH(), pr.d, pr.k, pr.p(), status, st,
@@ -295,7 +306,7 @@ int run_pipeline_with(const Problem& pr, const Layout& L, char* ws, const void* 
 template <typename T>
 int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, const void* K, const void* V,
                  const void* E, const void* F, const void* W, void* out, cudaStream_t st, bool tc1, bool tc2,
-                 bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status, int* launches) {
+                 bool tc3, TensorContext* tc, StageTimer* timer, bool keep_status, int* launches, int phases = 3) {
   auto stage1 = [&](float* kpvp, int* status, int* n) -> int {
     if (tc1) {
       int cuda_err = 0;
@@ -307,7 +318,7 @@ int run_pipeline(const Problem& pr, const Layout& L, char* ws, const void* Q, co
     }
     return launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, n);
   };
-  return run_pipeline_with<T>(pr, L, ws, Q, W, out, st, tc2, tc3, tc, timer, keep_status, launches, stage1);
+  return run_pipeline_with<T>(pr, L, ws, Q, W, out, st, tc2, tc3, tc, timer, keep_status, launches, stage1, phases);
 }
 
 int validate_pointers(const Problem& pr, const void* Q, const void* K, const void* V, const void* E,
@@ -329,11 +340,24 @@ int validate_pointers(const Problem& pr, const void* Q, const void* K, const voi
 // for, so that a caller that runs several problems in a row gets one block that fits them all.
 int forward_device(const void* Q, const void* K, const void* V, const void* E, const void* F, const void* W,
                    int variant, int B, int H, int N, int d, int k, int m, void* out, void* stream,
-                   bool keep_status, size_t reserve) {
+                   bool keep_status, size_t reserve, int phases = 3) {
   Problem pr;
   int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
   if (rc) return rc;
-  rc = validate_pointers(pr, Q, K, V, E, F, W, out);
+  if (phases == 3) {
+    rc = validate_pointers(pr, Q, K, V, E, F, W, out);
+  } else if (phases == 1) {
+    // first half of a sequence-sharded forward: keys, values and projections only
+    if (!K || !V || !E || !F) return FLURKA_ERR_NULL;
+    for (const void* ptr : {K, V, E, F})
+      if ((uintptr_t)ptr & 15) return FLURKA_ERR_ALIGN;
+  } else {
+    // second half: queries, the random features, the output
+    if (!Q || !out || (pr.kernel == FLURKA_PERFORMER && !W)) return FLURKA_ERR_NULL;
+    for (const void* ptr : {Q, W, (const void*)out})
+      if (ptr && ((uintptr_t)ptr & 15)) return FLURKA_ERR_ALIGN;
+    if (overlaps(out, pr.qkv_elems() * pr.esize(), Q, pr.qkv_elems() * pr.esize())) return FLURKA_ERR_OVERLAP;
+  }
   if (rc) return rc;
   int path = g_path;
   const bool tensor_ok = tensor_path_ok(pr);
@@ -345,27 +369,38 @@ int forward_device(const void* Q, const void* K, const void* V, const void* E, c
   const Layout L = make_layout(pr);
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = nullptr;
-  rc = get_workspace(ds, std::max(L.total, reserve), st, &ws);
-  if (rc) return rc;
+  if (phases == 2) {
+    // the second half works on what the first half (and the caller's sum over the shards) left in the
+    // workspace: same device, same head count and sizes (the slice length may differ)
+    const Problem& lp = ds.last_problem;
+    if (!ds.have_last || !ds.partial_pending || lp.BH() != pr.BH() || lp.d != pr.d || lp.k != pr.k || lp.m != pr.m ||
+        lp.kernel != pr.kernel || lp.fp32 != pr.fp32)
+      return FLURKA_ERR_WORKSPACE;
+    ws = ds.last_ws;
+  } else {
+    rc = get_workspace(ds, std::max(L.total, reserve), st, &ws);
+    if (rc) return rc;
+  }
   int launches = 0;
-  ds.timer.on = g_stage_timing;
-  StageTimer* timer = g_stage_timing ? &ds.timer : nullptr;
+  ds.timer.on = g_stage_timing && phases == 3;
+  StageTimer* timer = ds.timer.on ? &ds.timer : nullptr;
   if (timer) {
     rc = timer->create();
     if (rc != cudaSuccess) return cuda_fail((cudaError_t)rc);
   }
   if (pr.fp32) {
     rc = run_pipeline<float>(pr, L, ws, Q, K, V, E, F, W, out, st, false, false, false, &ds.tc, timer, keep_status,
-                             &launches);
+                             &launches, phases);
   } else {
     const bool tc1 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE1;
     const bool tc2 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE23;
     const bool tc3 = path == FLURKA_PATH_TENSOR || path == FLURKA_PATH_TENSOR_STAGE3 || tc2;
     rc = run_pipeline<__nv_bfloat16>(pr, L, ws, Q, K, V, E, F, W, out, st, tc1, tc2, tc3, &ds.tc, timer,
-                                     keep_status, &launches);
+                                     keep_status, &launches, phases);
   }
   if (rc) return rc;
-  ds.timer.have = g_stage_timing;
+  ds.partial_pending = phases != 3;       // K', V' of a sharded forward stay in the workspace
+  ds.timer.have = ds.timer.on;
   ds.last_path = path;
   ds.last_launches = launches;
   ds.have_last = true;
@@ -382,6 +417,27 @@ int flurka_forward(const void* Q, const void* K, const void* V, const void* E, c
                    const void* W, int variant, int B, int H, int N, int d, int k, int m, void* out,
                    void* stream) {
   return forward_device(Q, K, V, E, F, W, variant, B, H, N, d, k, m, out, stream, /*keep_status=*/false, 0);
+}
+
+int flurka_forward_partial(const void* K, const void* V, const void* E, const void* F, int variant, int B, int H,
+                           int N, int d, int k, int m, void* stream) {
+  return forward_device(nullptr, K, V, E, F, nullptr, variant, B, H, N, d, k, m, nullptr, stream, false, 0, /*phases=*/1);
+}
+
+int flurka_forward_finish(const void* Q, const void* W, int variant, int B, int H, int N, int d, int k, int m,
+                          void* out, void* stream) {
+  return forward_device(Q, nullptr, nullptr, nullptr, nullptr, W, variant, B, H, N, d, k, m, out, stream, false, 0,
+                        /*phases=*/2);
+}
+
+int flurka_partial_sums(void** dev_ptr, size_t* bytes) {
+  if (!dev_ptr || !bytes) return FLURKA_ERR_NULL;
+  DeviceState& ds = dev_state();
+  if (!ds.have_last || !ds.partial_pending) return FLURKA_ERR_WORKSPACE;
+  const Layout L = make_layout(ds.last_problem);
+  *dev_ptr = ds.last_ws + L.kpvp;
+  *bytes = L.kpvp_end - L.kpvp;
+  return FLURKA_OK;
 }
 
 int flurka_forward_host(const void* Q, const void* K, const void* V, const void* E, const void* F,
@@ -730,6 +786,7 @@ int flurka_forward_fused(const void* Xq, const void* Xk, const void* Xv, const v
                                        path == FLURKA_PATH_TENSOR, &ds.tc, timer, &launches);
   if (rc) return rc;
   ds.timer.have = g_stage_timing;
+  ds.partial_pending = false;
   ds.last_path = path;
   ds.last_launches = launches;
   ds.have_last = true;

@@ -88,3 +88,62 @@ def test_reference_arm_runs_on_rank_zero_only(monkeypatch):
     line = json.loads(buf.getvalue())
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["gpu_launches"] == 0
+
+
+def _shard_worker(rank, world, port, q):
+    """One rank of a sequence-sharded forward on CPU: the library's part is played by the fp64 oracle, the
+    exchange is the real one (all-reduce of the K', V' block over gloo)."""
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    import numpy as np
+    import oracle
+    from paper_2306_15799_b200 import configs, sharded, synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w = configs.shrink(configs.C3, B=1, H=2, N=200, k=16, m=32)
+        x = {n: (t.double().numpy() if t is not None else None) for n, t in synth.make_inputs(w).items()}
+        b, e = sharded.shard_bounds(w.N, world, rank)
+        # this rank's part of K' = E K, V' = F V for every head: its positions, the matching columns
+        block = torch.from_numpy(np.stack([np.stack([x[p][:, b:e] @ x[t][0, h, b:e] for h in range(w.H)])
+                                           for p, t in (("E", "K"), ("F", "V"))]))
+        dist.all_reduce(block, op=dist.ReduceOp.SUM)
+        Kp, Vp = block[0].numpy(), block[1].numpy()
+        # the summed K', V' go through the oracle's own projection step unchanged: k rows padded to the
+        # slice length, projected with [I_k | 0]
+        n = e - b
+        pad = lambda M: np.concatenate([M, np.zeros((n - w.k, w.d))])
+        sel = np.concatenate([np.eye(w.k), np.zeros((w.k, n - w.k))], axis=1)
+        out = np.stack([oracle.head(x["Q"][0, h, b:e], pad(Kp[h]), pad(Vp[h]), sel, sel, x["W"], w.variant)
+                        for h in range(w.H)])
+        q.put((rank, (b, e), out))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sequence_sharding_two_ranks_gloo():
+    """Shard bounds tile the sequence, and the per-rank parts of K', V' summed over the ranks give every
+    rank's rows of the whole-sequence result (Eq. (2)'s contraction is a sum over positions)."""
+    import numpy as np
+    import oracle
+    from paper_2306_15799_b200 import configs, sharded, synth
+    for N, world in ((200, 2), (1000, 3), (17, 4), (8, 3)):
+        bs = [sharded.shard_bounds(N, world, r) for r in range(world)]
+        assert bs[0][0] == 0 and bs[-1][1] == N and all(a[1] == b[0] for a, b in zip(bs, bs[1:]))
+        assert all((e - b) % 8 == 0 for b, e in bs[:-1])
+    world, port = 2, 29613
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_shard_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted((q.get(timeout=180) for _ in range(world)), key=lambda t: t[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = configs.shrink(configs.C3, B=1, H=2, N=200, k=16, m=32)
+    x = {n: (t.double().numpy() if t is not None else None) for n, t in synth.make_inputs(w).items()}
+    full = np.stack([oracle.head(x["Q"][0, h], x["K"][0, h], x["V"][0, h], x["E"], x["F"], x["W"], w.variant)
+                     for h in range(w.H)])
+    for rank, (b, e), out in res:
+        assert np.abs(out - full[:, b:e]).max() < 1e-9
