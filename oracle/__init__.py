@@ -80,6 +80,9 @@ class OracleLib:
         if hasattr(lib, "flurka_oracle_fused_head"):
             lib.flurka_oracle_fused_head.restype = ci
             lib.flurka_oracle_fused_head.argtypes = [_DP] * 9 + [ci] * 7 + [_LP, ctypes.c_long] + [_DP] * 4
+        if hasattr(lib, "flurka_oracle_head_backward"):
+            lib.flurka_oracle_head_backward.restype = ci
+            lib.flurka_oracle_head_backward.argtypes = [_DP] * 7 + [ci] * 5 + [_DP] * 5
         self._lib = lib
 
     def threads(self) -> int:
@@ -160,6 +163,20 @@ class OracleLib:
             raise ValueError("flurka_oracle_fused_head failed: %d" % rc)
         return (out, {"Kp": Kp, "Vp": Vp, "Q": Qh}) if intermediates else out
 
+    def head_backward(self, Q, K, V, E, F, W, dO, variant):
+        """Gradients of sum(O * dO) for one head: returns dict(dQ, dK, dV [N,d], dE, dF [k,N])."""
+        Q, K, V, E, F, W, N, d, k, m = self._head_args(Q, K, V, E, F, W, variant)
+        dO = _f64(dO)
+        assert dO.shape == (N, d), "dO must be [N, d]"
+        g = {"dQ": np.empty((N, d)), "dK": np.empty((N, d)), "dV": np.empty((N, d)),
+             "dE": np.empty((k, N)), "dF": np.empty((k, N))}
+        rc = self._lib.flurka_oracle_head_backward(
+            _ptr(Q), _ptr(K), _ptr(V), _ptr(E), _ptr(F), _ptr(W), _ptr(dO), variant, N, d, k, m,
+            _ptr(g["dQ"]), _ptr(g["dK"]), _ptr(g["dV"]), _ptr(g["dE"]), _ptr(g["dF"]))
+        if rc:
+            raise ValueError("flurka_oracle_head_backward failed: %d" % rc)
+        return g
+
     def features(self, X, W, variant, *, stabilise=False, scope_global=False):
         """phi applied to the rows of X [rows,d]. Returns [rows,m] (PERFORMER) or [rows,d] (RNN)."""
         X, W = _f64(X), _f64(W)
@@ -210,6 +227,10 @@ def head_quadratic(*a, **kw):
 
 def fused_head(*a, **kw):
     return default().fused_head(*a, **kw)
+
+
+def head_backward(*a, **kw):
+    return default().head_backward(*a, **kw)
 
 
 def features(*a, **kw):

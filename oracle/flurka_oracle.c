@@ -355,6 +355,143 @@ int flurka_oracle_fused_head(const double *Xq, const double *Xk, const double *X
   return 0;
 }
 
+/* Derivative of the feature map (Section 2.1) with respect to its argument, contracted with dPhi:
+ *   PERFORMER  Phi_i = exp(w_i.x - |x|^2/2 - s)/sqrt(m):  dPhi_i/dx = Phi_i (w_i - x)   (s is a constant
+ *              that cancels in the output, so it carries no gradient)
+ *   RNN        Phi_c = elu(x_c) + 1:                       dPhi_c/dx_c = 1 for x_c > 0, exp(x_c) otherwise
+ * X, dX: rows x d; Phi, dPhi: rows x p.  dX is overwritten. */
+static void feature_map_backward(const double *X, int rows, int d, const double *W, int m, int variant,
+                                 const double *Phi, const double *dPhi, double *dX) {
+#pragma omp parallel for schedule(static)
+  for (int r = 0; r < rows; ++r) {
+    const double *x = X + (size_t)r * d;
+    double *dx = dX + (size_t)r * d;
+    if (variant == FLURKA_ORACLE_RNN) {
+      for (int c = 0; c < d; ++c)
+        dx[c] = dPhi[(size_t)r * d + c] * (x[c] > 0.0 ? 1.0 : exp(x[c]));
+      continue;
+    }
+    for (int c = 0; c < d; ++c) dx[c] = 0.0;
+    for (int i = 0; i < m; ++i) {
+      const double g = dPhi[(size_t)r * m + i] * Phi[(size_t)r * m + i];
+      const double *w = W + (size_t)i * d;
+      for (int c = 0; c < d; ++c) dx[c] += g * (w[c] - x[c]);
+    }
+  }
+}
+
+/*
+ * Backward pass of one head (the paper trains these models, Sections 1 and 4; it prints no backward
+ * formulas, so this is the chain rule applied to steps 1 to 4 of flurka_oracle_head, in reverse):
+ * given dO (N x d), the gradients of  sum(O * dO)  with respect to Q, K, V (N x d) and E, F (k x N).
+ *   4'. O_n = num_n / den_n:   dnum_n = dO_n / den_n,   dden_n = -(O_n . dO_n) / den_n
+ *       num_n = Phi_q[n] KV, den_n = Phi_q[n] . z:
+ *       dPhi_q[n,i] = KV_i . dnum_n + z_i dden_n,  dKV_i += Phi_q[n,i] dnum_n,  dz_i += Phi_q[n,i] dden_n
+ *   3'. KV = Phi_k^T V', z = Phi_k^T 1:  dPhi_k[j,i] = dKV_i . V'_j + dz_i,  dV'_j = sum_i Phi_k[j,i] dKV_i
+ *   2'. through the feature maps (feature_map_backward): dQ, dK'
+ *   1'. K' = E K, V' = F V:  dK = E^T dK',  dE = dK' K^T,  dV = F^T dV',  dF = dV' V^T
+ * Any of the five outputs may be NULL.
+ */
+int flurka_oracle_head_backward(const double *Q, const double *K, const double *V, const double *E,
+                                const double *F, const double *W, const double *dO, int variant, int N,
+                                int d, int k, int m, double *dQ, double *dK, double *dV, double *dE,
+                                double *dF) {
+  int rc = check_args(Q, K, V, E, F, W, variant, N, d, k, m, dO);
+  if (rc) return rc;
+  const int p = (variant == FLURKA_ORACLE_PERFORMER) ? m : d;
+  double *Kp = (double *)malloc((size_t)k * d * sizeof(double));
+  double *Vp = (double *)malloc((size_t)k * d * sizeof(double));
+  double *Phik = (double *)malloc((size_t)k * p * sizeof(double));
+  double *Phiq = (double *)malloc((size_t)N * p * sizeof(double));
+  double *KV = (double *)calloc((size_t)p * d, sizeof(double));
+  double *z = (double *)calloc((size_t)p, sizeof(double));
+  double *dPhiq = (double *)malloc((size_t)N * p * sizeof(double));
+  double *dPhik = (double *)malloc((size_t)k * p * sizeof(double));
+  double *dKV = (double *)calloc((size_t)p * d, sizeof(double));
+  double *dz = (double *)calloc((size_t)p, sizeof(double));
+  double *dKp = (double *)malloc((size_t)k * d * sizeof(double));
+  double *dVp = (double *)calloc((size_t)k * d, sizeof(double));
+  double *dQl = (double *)malloc((size_t)N * d * sizeof(double));
+  if (!Kp || !Vp || !Phik || !Phiq || !KV || !z || !dPhiq || !dPhik || !dKV || !dz || !dKp || !dVp || !dQl) {
+    free(Kp); free(Vp); free(Phik); free(Phiq); free(KV); free(z); free(dPhiq); free(dPhik); free(dKV);
+    free(dz); free(dKp); free(dVp); free(dQl);
+    return -7;
+  }
+  /* forward, steps 1 to 3 */
+  down_project(E, K, N, d, k, Kp);
+  down_project(F, V, N, d, k, Vp);
+  feature_map(Kp, k, d, W, m, variant, 1, /*one scalar per head*/ 1, Phik);
+  feature_map(Q, N, d, W, m, variant, 1, /*one scalar per row*/ 0, Phiq);
+  for (int j = 0; j < k; ++j)
+    for (int i = 0; i < p; ++i) {
+      const double f = Phik[(size_t)j * p + i];
+      z[i] += f;
+      for (int c = 0; c < d; ++c) KV[(size_t)i * d + c] += f * Vp[(size_t)j * d + c];
+    }
+  /* step 4 forward and 4' backward, row by row (the sums into dKV, dz are taken serially) */
+  for (int n = 0; n < N; ++n) {
+    const double *fq = Phiq + (size_t)n * p;
+    const double *go = dO + (size_t)n * d;
+    double den = 0.0, odo = 0.0;
+    for (int i = 0; i < p; ++i) den += fq[i] * z[i];
+    for (int c = 0; c < d; ++c) {
+      double num = 0.0;
+      for (int i = 0; i < p; ++i) num += fq[i] * KV[(size_t)i * d + c];
+      odo += (num / den) * go[c];
+    }
+    const double dden = -odo / den;
+    for (int i = 0; i < p; ++i) {
+      double acc = z[i] * dden;
+      for (int c = 0; c < d; ++c) {
+        const double dnum = go[c] / den;
+        acc += KV[(size_t)i * d + c] * dnum;
+        dKV[(size_t)i * d + c] += fq[i] * dnum;
+      }
+      dPhiq[(size_t)n * p + i] = acc;
+      dz[i] += fq[i] * dden;
+    }
+  }
+  /* 3' */
+  for (int j = 0; j < k; ++j)
+    for (int i = 0; i < p; ++i) {
+      double acc = dz[i];
+      for (int c = 0; c < d; ++c) {
+        acc += dKV[(size_t)i * d + c] * Vp[(size_t)j * d + c];
+        dVp[(size_t)j * d + c] += Phik[(size_t)j * p + i] * dKV[(size_t)i * d + c];
+      }
+      dPhik[(size_t)j * p + i] = acc;
+    }
+  /* 2' */
+  feature_map_backward(Q, N, d, W, m, variant, Phiq, dPhiq, dQl);
+  feature_map_backward(Kp, k, d, W, m, variant, Phik, dPhik, dKp);
+  if (dQ) memcpy(dQ, dQl, (size_t)N * d * sizeof(double));
+  /* 1' */
+#pragma omp parallel for schedule(static)
+  for (int n = 0; n < N; ++n) {
+    for (int c = 0; c < d; ++c) {
+      double gk = 0.0, gv = 0.0;
+      for (int j = 0; j < k; ++j) {
+        gk += E[(size_t)j * N + n] * dKp[(size_t)j * d + c];
+        gv += F[(size_t)j * N + n] * dVp[(size_t)j * d + c];
+      }
+      if (dK) dK[(size_t)n * d + c] = gk;
+      if (dV) dV[(size_t)n * d + c] = gv;
+    }
+    for (int j = 0; j < k; ++j) {
+      double ge = 0.0, gf = 0.0;
+      for (int c = 0; c < d; ++c) {
+        ge += dKp[(size_t)j * d + c] * K[(size_t)n * d + c];
+        gf += dVp[(size_t)j * d + c] * V[(size_t)n * d + c];
+      }
+      if (dE) dE[(size_t)j * N + n] = ge;
+      if (dF) dF[(size_t)j * N + n] = gf;
+    }
+  }
+  free(Kp); free(Vp); free(Phik); free(Phiq); free(KV); free(z); free(dPhiq); free(dPhik); free(dKV);
+  free(dz); free(dKp); free(dVp); free(dQl);
+  return 0;
+}
+
 /*
  * The feature map on its own (Section 2.1): X is rows x d, Phi is rows x p with
  * p = m (PERFORMER, phi(x) = m^{-1/2} [psi_1(x) .. psi_m(x)]) or p = d (RNN).

@@ -323,6 +323,53 @@ def pin_fused_special_cases(orc):
         assert _rel(lin, sep) < 1e-11
 
 
+def pin_backward_matches_finite_differences(orc):
+    """The backward pass is the derivative of the (pinned) forward pass: for a random dO, the directional
+    derivative of sum(O * dO) along random directions in Q, K, V, E, F equals <gradient, direction>."""
+    for variant in (PERFORMER, RNN):
+        for seed in (31, 32):
+            Q, K, V, E, F, W = _tiny(seed, N=14, d=5, k=4, m=9)
+            Wv = W if variant == PERFORMER else None
+            r = _rng(seed + 100)
+            dO = r.normal(size=Q.shape)
+            g = orc.head_backward(Q, K, V, E, F, Wv, dO, variant)
+            x = {"Q": Q, "K": K, "V": V, "E": E, "F": F}
+            loss = lambda y: float((orc.head(y["Q"], y["K"], y["V"], y["E"], y["F"], Wv, variant) * dO).sum())
+            for name in ("Q", "K", "V", "E", "F"):
+                u = r.normal(size=x[name].shape)
+                h = 1e-5
+                plus, minus = dict(x), dict(x)
+                plus[name] = x[name] + h * u
+                minus[name] = x[name] - h * u
+                fd = (loss(plus) - loss(minus)) / (2 * h)
+                an = float((g["d" + name] * u).sum())
+                assert abs(fd - an) <= 2e-6 * max(1.0, abs(fd)), ("backward vs finite differences", variant, name, fd, an)
+
+
+def pin_backward_special_cases(orc):
+    """One projected key: O_n = F V for every row, so nothing flows to Q, K, E, and dV = F^T (sum_n dO_n),
+    dF = (sum_n dO_n) V^T.  The gradients are linear in dO.  V = const * 1 with F 1 = 1 gives O = const:
+    the gradients with respect to Q, K, E vanish again."""
+    for variant in (PERFORMER, RNN):
+        Q, K, V, E, F, W = _tiny(41, N=12, d=4, k=1, m=6)
+        Wv = W if variant == PERFORMER else None
+        dO = _rng(42).normal(size=Q.shape)
+        g = orc.head_backward(Q, K, V, E, F, Wv, dO, variant)
+        s = dO.sum(axis=0)
+        assert max(np.abs(g["dQ"]).max(), np.abs(g["dK"]).max(), np.abs(g["dE"]).max()) < 1e-12
+        assert np.allclose(g["dV"], np.outer(F[0], s), atol=1e-12) and np.allclose(g["dF"], (V @ s)[None, :], atol=1e-12)
+        Q, K, V, E, F, W = _tiny(43, N=16, d=4, k=5, m=8)
+        Wv = W if variant == PERFORMER else None
+        d1, d2 = _rng(44).normal(size=Q.shape), _rng(45).normal(size=Q.shape)
+        ga, gb = orc.head_backward(Q, K, V, E, F, Wv, d1, variant), orc.head_backward(Q, K, V, E, F, Wv, d2, variant)
+        gc = orc.head_backward(Q, K, V, E, F, Wv, 2.0 * d1 - 0.5 * d2, variant)
+        for name in gc:
+            assert _rel(gc[name], 2.0 * ga[name] - 0.5 * gb[name]) < 1e-11
+        Fm = np.abs(F) / np.abs(F).sum(axis=1, keepdims=True)          # rows sum to one
+        gconst = orc.head_backward(Q, K, np.full_like(V, 0.7), E, Fm, Wv, d1, variant)
+        assert max(np.abs(gconst["dQ"]).max(), np.abs(gconst["dK"]).max(), np.abs(gconst["dE"]).max()) < 1e-10
+
+
 ALL_PINS = [
     pin_quadratic_equals_associative,
     pin_identity_projection,
@@ -338,6 +385,8 @@ ALL_PINS = [
     pin_forward_layout,
     pin_fused_maps_commute_with_the_contraction,
     pin_fused_special_cases,
+    pin_backward_matches_finite_differences,
+    pin_backward_special_cases,
 ]
 
 
@@ -372,6 +421,12 @@ MUTANTS = {
     "fused_query_map_is_key_map": ("linear_map(Xs, (int)n_rows, dm, Wq, d, Qs);", "linear_map(Xs, (int)n_rows, dm, Wk, d, Qs);"),
     "linear_map_transposed": ("y[c] += x * w[c];", "y[c] += x * Wm[(size_t)c * dm + e];"),
     "fused_queries_contracted_too": ("double *Xs = gather_rows(Xq, dm, rows, nq);", "double *Xs = gather_rows(Xk, dm, rows, nq);"),
+    "backward_denominator_sign": ("const double dden = -odo / den;", "const double dden = odo / den;"),
+    "backward_feature_shift_dropped": ("dx[c] += g * (w[c] - x[c]);", "dx[c] += g * w[c];"),
+    "backward_elu_slope": ("(x[c] > 0.0 ? 1.0 : exp(x[c]))", "(x[c] > 0.0 ? 1.0 : exp(x[c]) - 1.0)"),
+    "backward_normaliser_gradient_dropped": ("double acc = dz[i];", "double acc = 0.0;"),
+    "backward_dE_uses_values": ("ge += dKp[(size_t)j * d + c] * K[(size_t)n * d + c];", "ge += dKp[(size_t)j * d + c] * V[(size_t)n * d + c];"),
+    "backward_dK_through_F": ("gk += E[(size_t)j * N + n] * dKp[(size_t)j * d + c];", "gk += F[(size_t)j * N + n] * dKp[(size_t)j * d + c];"),
     "head_stride_wrong": ("const size_t head = (size_t)N * d;", "const size_t head = (size_t)N * d / 2 * 2 - d;"),
 }
 
