@@ -166,6 +166,22 @@ int flurka_partial_sums(void** dev_ptr, size_t* bytes);
 int flurka_forward_finish(const void* Q, const void* W, int variant, int B, int H, int N, int d, int k, int m,
                           void* out, void* stream);
 
+/*
+ * flurka_backward -- the gradients of flurka_forward's output (the method is one for training, Sections 1
+ * and 4; the paper prints no backward formulas, these follow from Eq. (2) and Appendix D by the chain rule):
+ * given dO = d loss / d out, writes d loss / d Q, K, V (shapes of Q, K, V) and d loss / d E, F (shape of E,
+ * F: summed over every batch and head that shares the pair).  W is not learned and gets no gradient.
+ * All buffers are DEVICE buffers of the call's element type; variant word, layouts, limits, alignment,
+ * stream and workspace rules as for flurka_forward (flurka_backward_workspace_bytes says how much scratch).
+ * The forward's key-side summaries are recomputed inside the call, so nothing has to be kept from the
+ * forward pass.  Runs on CUDA cores with fp32 arithmetic for every shape; no output may overlap an input
+ * or another output.
+ */
+int flurka_backward(const void* Q, const void* K, const void* V, const void* E, const void* F, const void* W,
+                    const void* dO, int variant, int B, int H, int N, int d, int k, int m, void* dQ, void* dK,
+                    void* dV, void* dE, void* dF, void* stream);
+size_t flurka_backward_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m);
+
 /* Bytes of device scratch flurka_forward needs for this problem (0 on invalid arguments). Holds the
  * fp32 projections K', V' (Eq. (2)'s E K and F V), the key-side feature summaries and a status word. */
 size_t flurka_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m);

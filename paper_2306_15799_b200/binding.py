@@ -23,6 +23,7 @@ EXPORTS = [
     "flurka_strerror", "flurka_version", "flurka_forward_static_scratch", "flurka_static_scratch_need",
     "flurka_measure_ex2_rate", "flurka_forward_fused", "flurka_fused_workspace_bytes",
     "flurka_forward_partial", "flurka_partial_sums", "flurka_forward_finish",
+    "flurka_backward", "flurka_backward_workspace_bytes",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -94,6 +95,10 @@ def load() -> ctypes.CDLL:
     lib.flurka_forward_finish.argtypes = [vp, vp] + [ci] * 7 + [vp, vp]
     lib.flurka_partial_sums.restype = ci
     lib.flurka_partial_sums.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(sz)]
+    lib.flurka_backward.restype = ci
+    lib.flurka_backward.argtypes = [vp] * 7 + [ci] * 7 + [vp] * 6
+    lib.flurka_backward_workspace_bytes.restype = sz
+    lib.flurka_backward_workspace_bytes.argtypes = [ci] * 7
     lib.flurka_measure_ex2_rate.restype = ci
     lib.flurka_measure_ex2_rate.argtypes = [ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -274,6 +279,24 @@ def flurka_forward_finish(Q, W, variant, k, out=None, stream=None, layout="bhnd"
     if rc:
         raise FlurkaError(rc, "flurka_forward_finish")
     return out
+
+
+def flurka_backward(Q, K, V, E, F, W, dO, variant, stream=None, layout="bhnd"):
+    """Gradients of the forward's output with respect to Q, K, V, E, F, given dO (device tensors).
+    Returns (dQ, dK, dV, dE, dF), shaped and typed like the inputs."""
+    B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, dO, "cuda", layout)
+    grads = [torch.empty_like(t) for t in (Q, K, V, E, F)]
+    rc = load().flurka_backward(
+        Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(), W.data_ptr() if W is not None else None,
+        dO.data_ptr(), _variant_word(variant, Q.dtype, layout, E.dim() == 3), B, H, N, d, k, m,
+        *[g.data_ptr() for g in grads], _stream_ptr(stream))
+    if rc:
+        raise FlurkaError(rc, "flurka_backward")
+    return tuple(grads)
+
+
+def flurka_backward_workspace_bytes(variant, io_dtype, B, H, N, d, k, m) -> int:
+    return int(load().flurka_backward_workspace_bytes(_variant_word(variant, io_dtype), B, H, N, d, k, m))
 
 
 def flurka_fused_workspace_bytes(variant, io_dtype, B, H, N, dm, d, k, m) -> int:

@@ -7,6 +7,7 @@
 #include <algorithm>
 #include <stdint.h>
 
+#include "simt_backward.cuh"
 #include "simt_kernels.cuh"
 #include "tensor_path.cuh"
 
@@ -788,6 +789,143 @@ int flurka_forward_fused(const void* Xq, const void* Xk, const void* Xv, const v
   ds.timer.have = g_stage_timing;
   ds.partial_pending = false;
   ds.last_path = path;
+  ds.last_launches = launches;
+  ds.have_last = true;
+  ds.last_problem = pr;
+  ds.last_ws = ws;
+  return FLURKA_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+// Scratch of the backward pass, after the forward layout: da [BH][p][d], db [BH][p] (adjacent: one
+// memset), then dK', dV' [2][BH][k][d]; all fp32.
+struct BackwardLayout {
+  Layout L;
+  size_t da, dab_bytes, db, dkpvp, total;
+};
+
+BackwardLayout make_backward_layout(const Problem& pr) {
+  BackwardLayout b;
+  b.L = make_layout(pr, /*with_split_scratch=*/false);
+  size_t off = b.L.total;
+  const size_t da_bytes = (size_t)pr.BH() * pr.p() * pr.d * 4;
+  b.da = off;
+  b.db = off + da_bytes;
+  b.dab_bytes = da_bytes + (size_t)pr.BH() * pr.p() * 4;
+  off = align256(off + b.dab_bytes);
+  b.dkpvp = off; off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
+  b.total = off;
+  return b;
+}
+
+template <typename T, bool P>
+int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, const void* Q, const void* K,
+                      const void* V, const void* E, const void* F, const void* W, const void* dO, void* dQ, void* dK,
+                      void* dV, void* dE, void* dF, cudaStream_t st, int* launches) {
+  const Layout& L = BL.L;
+  float* kpvp = (float*)(ws + L.kpvp);
+  float* weight = (float*)(ws + L.weight);
+  float* a32 = (float*)(ws + L.a32);
+  float* da = (float*)(ws + BL.da);
+  float* db = (float*)(ws + BL.db);
+  float* dkpvp = (float*)(ws + BL.dkpvp);
+  const int smh = pr.seq_major_heads(), efh = pr.ef_heads();
+  cudaError_t e = cudaMemsetAsync(ws + L.status, 0, L.kpvp_end - L.status, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemsetAsync(da, 0, BL.dab_bytes, st)) != cudaSuccess) return cuda_fail(e);
+  // the forward's stages 1 and 2 again: K', V', a_i, b_i (or z_i)
+  int rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
+  if (rc) return rc;
+  rc = launch_simt_key_side<T, P>(pr, kpvp, W, weight, a32, nullptr, st, launches);
+  if (rc) return rc;
+  {
+    auto fn = simt_bwd_query_side<T, P>;
+    const size_t smem = ((size_t)2 * 32 * (pr.d + 1) + 32 * 33 + 32 * pr.d) * 4;
+    if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+      return cuda_fail(e);
+    dim3 grid((pr.N + 31) / 32, pr.BH());
+    fn<<<grid, 256, smem, st>>>((const T*)Q, (const T*)W, (const T*)dO, weight, a32, (T*)dQ, da, db, pr.N, pr.d,
+                                pr.p(), smh);
+    ++*launches;
+  }
+  {
+    auto fn = simt_bwd_key_side<T, P>;
+    const size_t smem = (size_t)3 * 32 * (pr.d + 1) * 4;
+    if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+      return cuda_fail(e);
+    dim3 grid((pr.k + 7) / 8, pr.BH());
+    fn<<<grid, 256, smem, st>>>(kpvp, (const T*)W, weight, a32, da, db, dkpvp, pr.BH(), pr.d, pr.k, pr.p());
+    ++*launches;
+  }
+  {
+    dim3 grid((pr.N + 31) / 32, pr.BH(), 2);
+    simt_bwd_inputs<T><<<grid, 256, 0, st>>>((const T*)E, (const T*)F, dkpvp, (T*)dK, (T*)dV, pr.BH(), pr.N, pr.d,
+                                             pr.k, smh, efh);
+    ++*launches;
+    dim3 grid2((pr.N + 31) / 32, (pr.k + 31) / 32, 2 * (efh > 0 ? efh : 1));
+    simt_bwd_projections<T><<<grid2, 256, 0, st>>>((const T*)K, (const T*)V, dkpvp, (T*)dE, (T*)dF, pr.BH(), pr.N,
+                                                   pr.d, pr.k, smh, efh);
+    ++*launches;
+  }
+  e = cudaGetLastError();
+  return e == cudaSuccess ? FLURKA_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t flurka_backward_workspace_bytes(int variant, int B, int H, int N, int d, int k, int m) {
+  Problem pr;
+  if (parse_problem(variant, B, H, N, d, k, m, &pr)) return 0;
+  return make_backward_layout(pr).total;
+}
+
+int flurka_backward(const void* Q, const void* K, const void* V, const void* E, const void* F, const void* W,
+                    const void* dO, int variant, int B, int H, int N, int d, int k, int m, void* dQ, void* dK,
+                    void* dV, void* dE, void* dF, void* stream) {
+  Problem pr;
+  int rc = parse_problem(variant, B, H, N, d, k, m, &pr);
+  if (rc) return rc;
+  if (!Q || !K || !V || !E || !F || !dO || !dQ || !dK || !dV || !dE || !dF) return FLURKA_ERR_NULL;
+  if (pr.kernel == FLURKA_PERFORMER && !W) return FLURKA_ERR_NULL;
+  const void* ins[7] = {Q, K, V, E, F, W, dO};
+  void* outs[5] = {dQ, dK, dV, dE, dF};
+  const size_t qb = pr.qkv_elems() * pr.esize(), eb = pr.ef_elems() * pr.esize(), wb = pr.w_elems() * pr.esize();
+  const size_t in_bytes[7] = {qb, qb, qb, eb, eb, wb, qb}, out_bytes[5] = {qb, qb, qb, eb, eb};
+  for (const void* ptr : ins)
+    if (ptr && ((uintptr_t)ptr & 15)) return FLURKA_ERR_ALIGN;
+  for (int o = 0; o < 5; ++o) {
+    if ((uintptr_t)outs[o] & 15) return FLURKA_ERR_ALIGN;
+    for (int i = 0; i < 7; ++i)
+      if (ins[i] && in_bytes[i] && overlaps(outs[o], out_bytes[o], ins[i], in_bytes[i])) return FLURKA_ERR_OVERLAP;
+    for (int o2 = 0; o2 < o; ++o2)
+      if (overlaps(outs[o], out_bytes[o], outs[o2], out_bytes[o2])) return FLURKA_ERR_OVERLAP;
+  }
+  rc = check_device();
+  if (rc) return rc;
+  DeviceState& ds = dev_state();
+  const BackwardLayout BL = make_backward_layout(pr);
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = nullptr;
+  rc = get_workspace(ds, BL.total, st, &ws);
+  if (rc) return rc;
+  int launches = 0;
+  const bool perf = pr.kernel == FLURKA_PERFORMER;
+  if (pr.fp32)
+    rc = perf ? backward_pipeline<float, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches)
+              : backward_pipeline<float, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches);
+  else
+    rc = perf ? backward_pipeline<__nv_bfloat16, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches)
+              : backward_pipeline<__nv_bfloat16, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st,
+                                                        &launches);
+  if (rc) return rc;
+  ds.partial_pending = false;
+  ds.timer.have = false;
+  ds.last_path = FLURKA_PATH_SIMT;
   ds.last_launches = launches;
   ds.have_last = true;
   ds.last_problem = pr;

@@ -1,0 +1,118 @@
+"""flurka_backward against the fp64 oracle's backward pass (itself pinned by finite differences of the
+forward oracle), element-wise through relative Frobenius norms per gradient."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2306_15799_b200 import binding, build, synth
+from paper_2306_15799_b200.configs import PERFORMER, RNN, Workload
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+# fp32 I/O: every step is fp32 with sums of up to N (or k, m) terms and one cancelling difference
+# (a_i.dO_n - O_n.dO_n), so gradients carry about 1e-5 relative error; bf16 I/O adds the rounding of the
+# stored gradients (2^-9 each): the gates are 1e-3 and 1e-2 of the gradient's Frobenius norm.
+TOL = {"fp32": 1e-3, "bf16": 1e-2}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    binding.load()
+
+
+def _oracle_grads(w, x, dO, per_head):
+    f64 = lambda t: t.double().numpy()
+    W = f64(x["W"]) if x["W"] is not None else None
+    g = {n: np.zeros(tuple(x[n[1:]].shape)) for n in ("dQ", "dK", "dV", "dE", "dF")}
+    for b in range(w.B):
+        for h in range(w.H):
+            E, F = (f64(x["E"][h]), f64(x["F"][h])) if per_head else (f64(x["E"]), f64(x["F"]))
+            r = oracle.head_backward(f64(x["Q"][b, h]), f64(x["K"][b, h]), f64(x["V"][b, h]), E, F, W, f64(dO[b, h]), w.variant)
+            for n in ("dQ", "dK", "dV"):
+                g[n][b, h] = r[n]
+            for n in ("dE", "dF"):
+                if per_head:
+                    g[n][h] += r[n]
+                else:
+                    g[n] += r[n]
+    return g
+
+
+def _check(w, layout="bhnd", per_head=False):
+    x = synth.make_inputs(w)
+    gen = torch.Generator().manual_seed(w.seed + 5)
+    if per_head:
+        for name in ("E", "F"):
+            x[name] = (torch.randn(w.H, w.k, w.N, generator=gen, dtype=torch.float64) * float(w.k) ** -0.5).to(x["Q"].dtype)
+    dO = torch.randn(w.B, w.H, w.N, w.d, generator=gen, dtype=torch.float64).to(x["Q"].dtype)
+    dev = pu.to_device(x)
+    t = (lambda a: a.transpose(1, 2).contiguous()) if layout == "bnhd" else (lambda a: a)
+    got = binding.flurka_backward(t(dev["Q"]), t(dev["K"]), t(dev["V"]), dev["E"], dev["F"], dev["W"], t(dO.cuda()),
+                                  w.variant, layout=layout)
+    torch.cuda.synchronize()
+    assert binding.flurka_last_status() == 0
+    ref = _oracle_grads(w, x, dO, per_head)
+    for name, tensor in zip(("dQ", "dK", "dV", "dE", "dF"), got):
+        arr = tensor.transpose(1, 2) if (layout == "bnhd" and tensor.dim() == 4) else tensor
+        arr = arr.cpu().double().numpy()
+        assert np.isfinite(arr).all(), name
+        rel = np.linalg.norm(arr - ref[name]) / max(np.linalg.norm(ref[name]), 1e-300)
+        assert rel <= TOL[w.io], "%s %s: rel-Fro %.3e > %.0e" % (w.name, name, rel, TOL[w.io])
+
+
+CASES = [
+    Workload("bwd_perf_fp32", PERFORMER, "fp32", 2, 2, 100, 24, 12, 40, 301),
+    Workload("bwd_rnn_fp32", RNN, "fp32", 1, 3, 77, 20, 9, 0, 302),
+    Workload("bwd_perf_bf16_d64", PERFORMER, "bf16", 1, 2, 300, 64, 40, 96, 303),
+    Workload("bwd_rnn_bf16_d128", RNN, "bf16", 1, 2, 160, 128, 33, 0, 304),
+    Workload("bwd_perf_fp32_ragged", PERFORMER, "fp32", 1, 1, 45, 33, 5, 37, 305),
+]
+
+
+@pytest.mark.parametrize("w", CASES, ids=lambda w: w.name)
+def test_backward_matches_oracle(w):
+    _check(w)
+
+
+def test_backward_seq_major_layout_and_per_head_projections():
+    _check(Workload("bwd_bnhd", PERFORMER, "fp32", 2, 3, 64, 16, 8, 24, 306), layout="bnhd")
+    _check(Workload("bwd_per_head", RNN, "fp32", 2, 2, 64, 16, 8, 0, 307), per_head=True)
+    _check(Workload("bwd_per_head_perf", PERFORMER, "fp32", 2, 2, 72, 16, 8, 24, 308), per_head=True)
+
+
+def test_backward_is_the_derivative_of_the_forward():
+    """Directional derivative of sum(out * dO) through flurka_forward (fp32) against <gradient, direction>."""
+    w = Workload("bwd_fd", PERFORMER, "fp32", 1, 1, 64, 16, 8, 24, 309)
+    x = pu.to_device(synth.make_inputs(w))
+    gen = torch.Generator().manual_seed(7)
+    dO = torch.randn(1, 1, 64, 16, generator=gen).cuda()
+    u = torch.randn(1, 1, 64, 16, generator=gen).cuda()
+    dQ = binding.flurka_backward(x["Q"], x["K"], x["V"], x["E"], x["F"], x["W"], dO, w.variant)[0]
+    h = 1e-2
+    f = lambda q: float((binding.flurka_forward(q.contiguous(), x["K"], x["V"], x["E"], x["F"], x["W"], w.variant).double()
+                         * dO.double()).sum())
+    fd = (f(x["Q"] + h * u) - f(x["Q"] - h * u)) / (2 * h)
+    an = float((dQ.double() * u.double()).sum())
+    assert abs(fd - an) <= 2e-2 * max(abs(fd), 1e-3), (fd, an)
+
+
+def test_backward_argument_errors():
+    w = Workload("bwd_args", RNN, "fp32", 1, 1, 32, 8, 4, 0, 310)
+    x = pu.to_device(synth.make_inputs(w))
+    lib = binding.load()
+    g = [torch.empty_like(x[n]) for n in ("Q", "K", "V", "E", "F")]
+    ptr = lambda t: t.data_ptr()
+    base = [ptr(x["Q"]), ptr(x["K"]), ptr(x["V"]), ptr(x["E"]), ptr(x["F"]), None, ptr(g[0])]
+    dims = [RNN | 0x100, 1, 1, 32, 8, 4, 0]
+    outs = [ptr(t) for t in g]
+    assert lib.flurka_backward(*base, *dims, *outs, None) == -8                 # dO is also dQ
+    dO = torch.zeros_like(x["Q"])
+    base[6] = ptr(dO)
+    assert lib.flurka_backward(*base, *dims, outs[0], outs[0], *outs[2:], None) == -8
+    assert lib.flurka_backward(*base, *dims, None, *outs[1:], None) == -1
+    assert lib.flurka_backward(*base, *dims, *outs, None) == 0
+    assert binding.flurka_backward_workspace_bytes(RNN, torch.float32, 1, 1, 32, 8, 4, 0) > 0
