@@ -392,20 +392,35 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
   if (tid == 0) grid_launch_dependents();   // only the write-out (and the merge) is left
   // ---- a_i = accumulator / z_i, stored transposed ([d][p], fp16) for stage 3
   if (nsplit == 1) {
+    // through shared memory (the staging buffer is free by now): every row owner drops its feature's d
+    // values into a [d][128] fp16 tile, then all threads copy the tile out 16 bytes at a time, so a^T
+    // leaves in whole 128- or 256-byte runs
     if (warp < 4 && ok) {
-      // whole warps are either inside or outside the p features (p is a multiple of 64); the TMEM
-      // loads are warp-wide either way, only the stores are predicated
       const uint32_t tb = tmem + ((uint32_t)(warp * 32) << 16) + kK2OCol;
       const float inv = 1.f / zsum;
-      __half* dst = prm.aT16 + (size_t)head * d * p + feat;
+      const uint32_t col_addr = sm_stage + (uint32_t)(warp * 32 + lane) * 2u;
       for (int c = 0; c < d; c += 32) {
         uint32_t r[32];
         tmem_ld32(tb + c, r);
         tmem_wait_ld(r);
-        if (feat < p) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) dst[(size_t)(c + e) * p] = __float2half_rn(__uint_as_float(r[e]) * inv);
+        for (int e = 0; e < 32; ++e) {
+          const unsigned short h = __half_as_ushort(__float2half_rn(__uint_as_float(r[e]) * inv));
+          asm volatile("st.shared.u16 [%0], %1;" ::"r"(col_addr + (uint32_t)(c + e) * 256u), "h"(h) : "memory");
         }
+      }
+    }
+    __syncthreads();
+    if (ok) {
+      const int live = min(128, p - i0);                    // a multiple of 64
+      const int cpr = live >> 3;                            // 16-byte pieces per row
+      __half* dst = prm.aT16 + (size_t)head * d * p + i0;
+      for (int idx = tid; idx < d * cpr; idx += kK2Threads) {
+        const int c = idx / cpr, ch = idx % cpr;
+        uint32_t v0, v1, v2, v3;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(sm_stage + (uint32_t)c * 256u + (uint32_t)ch * 16u));
+        *reinterpret_cast<uint4*>(dst + (size_t)c * p + ch * 8) = make_uint4(v0, v1, v2, v3);
       }
     }
   } else {
