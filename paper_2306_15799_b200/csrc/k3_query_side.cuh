@@ -465,40 +465,47 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           }
           mx = fmaxf(fmax3(mx, mx1, mx2), mx3);
           const float shift = mx * kLog2e;
-          // pass 2: p = 2^(S log2e - shift), fp16 pairs back into columns [c/2, c/2+16)
+          // pass 2: p = 2^(S log2e - shift), fp16 pairs back into the buffer at half the width.  Scale and
+          // shift and the row sums run two-wide; three pairs in eight take their exponential as a cubic on
+          // the FMA pipe, the others on the special-function unit, which is the busiest unit of this kernel
+          // (an all-MUFU loop of two warps per scheduler takes 8.9 cycles per warp-wide ex2; this mix 7.1).
+          const uint64_t l2 = pack2(kLog2e, kLog2e), ms2 = pack2(-shift, -shift);
+          uint64_t den2 = pack2(0.f, 0.f);
+          auto exp_block = [&](const uint32_t (&r)[32], uint32_t (&h)[16]) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              uint64_t x2 = fma2(pack2u(r[2 * e], r[2 * e + 1]), l2, ms2);
+              float e0, e1;
+              if ((e & 7) == 1 || (e & 7) == 4 || (e & 7) == 6) {
+                float x0, x1;
+                unpack2(x2, x0, x1);
+                // far below what fp16 can hold the result is 0 either way; the cubic needs its exponent in range
+                exp2_cubic2(pack2(fmaxf(x0, -60.f), fmaxf(x1, -60.f)), e0, e1);
+              } else {
+                float x0, x1;
+                unpack2(x2, x0, x1);
+                e0 = ex2_approx(x0);
+                e1 = ex2_approx(x1);
+              }
+              den2 = add2(den2, pack2(e0, e1));
+              const __half2 hh = __floats2half2_rn(e0, e1);
+              h[e] = *reinterpret_cast<const uint32_t*>(&hh);
+            }
+          };
           for (int c = 0; c < p; c += 64) {
             uint32_t h[16];
             tmem_wait_ld(ra);
             tmem_ld32(tb + c + 32, rb);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float x0 = fmaf(__uint_as_float(ra[2 * e]), kLog2e, -shift);
-              const float x1 = fmaf(__uint_as_float(ra[2 * e + 1]), kLog2e, -shift);
-              const float e0 = ex2_approx(x0);
-              const float e1 = ex2_approx(x1);
-              denom += e0;
-              denom1 += e1;
-              const __half2 hh = __floats2half2_rn(e0, e1);
-              h[e] = *reinterpret_cast<const uint32_t*>(&hh);
-            }
+            exp_block(ra, h);
             const uint32_t pc = pcol(c >> 6);
             tmem_st16(tb + pc, h);
             tmem_wait_ld(rb);
             if (c + 64 < p) tmem_ld32(tb + c + 64, ra);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float x0 = fmaf(__uint_as_float(rb[2 * e]), kLog2e, -shift);
-              const float x1 = fmaf(__uint_as_float(rb[2 * e + 1]), kLog2e, -shift);
-              const float e0 = ex2_approx(x0);
-              const float e1 = ex2_approx(x1);
-              denom += e0;
-              denom1 += e1;
-              const __half2 hh = __floats2half2_rn(e0, e1);
-              h[e] = *reinterpret_cast<const uint32_t*>(&hh);
-            }
+            exp_block(rb, h);
             tmem_st16(tb + pc + 16, h);
             if ((c >> 6) >= q_first && c + 64 < p) hand_over(buf, c >> 6);
           }
+          unpack2(den2, denom, denom1);
         } else {
           // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
           // (no wait for the buffer: this thread has itself read out the tile that used it before, and

@@ -60,11 +60,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One try: the thread may be suspended until the phase completes or about 4 us have passed (the
+// suspend-time hint; without it waiting threads come back to poll far more often, and their polling
+// costs the working warps of a power-limited kernel 1 to 2 % of their clock).
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 4000;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -84,7 +87,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 1023u) == 0) {
+    if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
         atomicOr(status, 1);
@@ -206,6 +209,59 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------ packed fp32 pairs
+// sm_100 has two-wide fp32 FMA / ADD on 64-bit register pairs; a pair of adjacent registers (as
+// tcgen05.ld delivers them) packs and unpacks without a move.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t a, uint32_t b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ void unpack2u(uint64_t v, uint32_t& a, uint32_t& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
+// 2^x for a pair of x in [-100, 1] on the FMA pipe instead of the special-function unit: n = round(x)
+// (by adding 1.5 * 2^23, which leaves n in the low mantissa bits), f = x - n in [-1/2, 1/2], a cubic in
+// f (relative error below 8e-5, well under the rounding of the fp16 result), n added to the exponent
+// field as an integer.
+__device__ __forceinline__ void exp2_cubic2(uint64_t x2, float& e0, float& e1) {
+  const uint64_t magic = pack2(12582912.f, 12582912.f);
+  const uint64_t t2 = add2(x2, magic);
+  const uint64_t f2 = sub2(x2, sub2(t2, magic));
+  uint64_t p2 = fma2(pack2(0.05520551f, 0.05520551f), f2, pack2(0.24261397f, 0.24261397f));
+  p2 = fma2(p2, f2, pack2(0.69325477f, 0.69325477f));
+  p2 = fma2(p2, f2, pack2(0.99992770f, 0.99992770f));
+  uint32_t ta, tb, pa, pb;
+  unpack2u(t2, ta, tb);
+  unpack2u(p2, pa, pb);
+  e0 = __uint_as_float(pa + (ta << 23));
+  e1 = __uint_as_float(pb + (tb << 23));
+}
 
 // ------------------------------------------------------------------------------ MMA
 // D[tmem] (+)= A[smem] * B[smem]; one thread issues.

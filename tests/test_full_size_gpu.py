@@ -85,3 +85,36 @@ def test_c5_sweep_points(k, m):
 
 def test_c5_one_point_full_batch():
     _check_full(configs.c5(512, 256), heads=[(0, 0), (7, 11)], n_rows=256)
+
+
+def test_fused_full_size():
+    """The entry point with un-projected inputs at its benchmark size (c3's shape, d_m = 1024): two sampled
+    heads, 256 sampled rows each, with the full-size K', V' after the linear maps."""
+    import oracle
+    w = configs.F1
+    x = synth.make_fused_inputs(w)
+    dev = {n: (t.cuda() if t is not None else None) for n, t in x.items() if n not in ("Xk", "Xv")}
+    out = binding.flurka_forward_fused(dev["Xq"], dev["Xq"], dev["Xq"], dev["E"], dev["F"], dev["Wq"], dev["Wk"],
+                                       dev["Wv"], dev["W"], w.variant, w.H)
+    torch.cuda.synchronize()
+    assert binding.flurka_last_status() == 0
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    assert bool(torch.isfinite(out.float()).all())
+    Kp = binding.flurka_debug_copy(0, (w.B, w.H, w.k, w.d))
+    Vp = binding.flurka_debug_copy(1, (w.B, w.H, w.k, w.d))
+    torch.cuda.synchronize()
+    f64 = lambda t: t.double().numpy()
+    rng = np.random.default_rng(61)
+    for (b, h) in [(0, 0), (3, 11)]:
+        rows = np.sort(rng.choice(w.N, size=256, replace=False))
+        rows[0], rows[-1] = 0, w.N - 1
+        cols = slice(h * w.d, (h + 1) * w.d)
+        X = f64(x["Xq"][b])
+        ref, mid = oracle.fused_head(X, X, X, f64(x["E"]), f64(x["F"]), f64(x["Wq"][:, cols]), f64(x["Wk"][:, cols]),
+                                     f64(x["Wv"][:, cols]), f64(x["W"]), w.variant, rows=rows, intermediates=True)
+        for mine, theirs, nm in ((Kp[b, h], mid["Kp"], "K'"), (Vp[b, h], mid["Vp"], "V'")):
+            err = np.abs(mine.cpu().double().numpy() - theirs).max()
+            assert err < 3e-5 * max(1.0, np.abs(theirs).max()), "%s %s head (%d,%d): %.3e" % (w.name, nm, b, h, err)
+        got = out[b, :, h, :].cpu()[torch.from_numpy(rows)].double().numpy()
+        rel, mx = pu.assert_close(got, ref, w.io, "%s head (%d,%d)" % (w.name, b, h))
+        print("%s head (%d,%d): rel-Fro %.3e, max-abs %.3e" % (w.name, b, h, rel, mx))
