@@ -70,6 +70,11 @@ TENSOR_CASES = [
     _fw("fused_rnn", RNN, "bf16", 2, 2, 1024, 192, 64, 128, 0, 64),
     _fw("fused_perf_ragged_n", PERFORMER, "bf16", 1, 3, 1000, 192, 64, 64, 64, 65, shared_x=False),
     _fw("fused_perf_k512", PERFORMER, "bf16", 1, 6, 640, 384, 64, 512, 128, 66),
+    # smallest sizes of every dimension of the map kernels: one 64-wide chunk of d_m, one head of 64 columns,
+    # 64 projected rows (half an MMA tile), a batch whose B*N is not a multiple of the 256-row block
+    _fw("fused_perf_dm64_one_head", PERFORMER, "bf16", 3, 1, 200, 64, 64, 64, 64, 74),
+    _fw("fused_rnn_d128_k64", RNN, "bf16", 1, 1, 136, 128, 128, 64, 0, 75),
+    _fw("fused_perf_wide_dm", PERFORMER, "bf16", 1, 2, 256, 1024, 64, 128, 192, 76, shared_x=False),
 ]
 
 
