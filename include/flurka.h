@@ -198,6 +198,11 @@ int flurka_set_path(int path);
  * the default), so that small problems still exercise several tiles per CTA. Returns the old limit. */
 int flurka_set_cta_limit(int max_ctas);
 
+/* Tuning / test knob: whether the tensor-core down-projection (Eq. (2)'s E K, F V) may run as pairs of
+ * CTAs that share the K / V tiles (the default, used when k % 256 == 0, B*H*d % 256 == 0 and E, F are
+ * shared by the heads) or always as single CTAs.  Returns the old setting. */
+int flurka_set_stage1_pairs(int on);
+
 /* The path the most recent successful flurka_forward took (never FLURKA_PATH_AUTO). */
 int flurka_last_path(void);
 

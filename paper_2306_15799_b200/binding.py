@@ -23,7 +23,7 @@ EXPORTS = [
     "flurka_strerror", "flurka_version", "flurka_forward_static_scratch", "flurka_static_scratch_need",
     "flurka_measure_ex2_rate", "flurka_forward_fused", "flurka_fused_workspace_bytes",
     "flurka_forward_partial", "flurka_partial_sums", "flurka_forward_finish",
-    "flurka_backward", "flurka_backward_workspace_bytes",
+    "flurka_backward", "flurka_backward_workspace_bytes", "flurka_set_stage1_pairs",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -99,6 +99,8 @@ def load() -> ctypes.CDLL:
     lib.flurka_backward.argtypes = [vp] * 7 + [ci] * 7 + [vp] * 6
     lib.flurka_backward_workspace_bytes.restype = sz
     lib.flurka_backward_workspace_bytes.argtypes = [ci] * 7
+    lib.flurka_set_stage1_pairs.restype = ci
+    lib.flurka_set_stage1_pairs.argtypes = [ci]
     lib.flurka_measure_ex2_rate.restype = ci
     lib.flurka_measure_ex2_rate.argtypes = [ctypes.POINTER(ctypes.c_double)]
     _lib = lib
@@ -324,6 +326,10 @@ def flurka_set_workspace(buf) -> None:
 
 def flurka_set_path(path: int) -> int:
     return int(load().flurka_set_path(path))
+
+
+def flurka_set_stage1_pairs(on: bool) -> bool:
+    return bool(load().flurka_set_stage1_pairs(1 if on else 0))
 
 
 def flurka_set_cta_limit(max_ctas: int) -> int:

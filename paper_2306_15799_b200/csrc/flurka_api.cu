@@ -571,6 +571,12 @@ int flurka_set_cta_limit(int max_ctas) {
   return prev;
 }
 
+int flurka_set_stage1_pairs(int on) {
+  const int prev = stage1_pairs();
+  stage1_pairs() = on != 0;
+  return prev;
+}
+
 int flurka_last_path(void) { return dev_state().last_path; }
 int flurka_last_launches(void) { return dev_state().last_launches; }
 

@@ -8,6 +8,7 @@
 
 #include "k0_linear_maps.cuh"
 #include "k1_down_project.cuh"
+#include "k1_down_project_pair.cuh"
 #include "k2_key_side.cuh"
 #include "k3_query_side.cuh"
 
@@ -97,6 +98,7 @@ struct TensorContext {
   TensorMaps maps;
   int sms = 0;
   bool k1_attr = false;
+  bool k1p_attr = false;
   bool k0_attr = false;
   int sm_total() {
     if (!sms) {
@@ -110,6 +112,12 @@ struct TensorContext {
   // SMs the persistent kernels may use (the test knob caps it)
   int sm_count();
 };
+
+// whether stage 1 may run as pairs of CTAs (tcgen05.mma.cta_group::2) where the shape allows
+inline int& stage1_pairs() {
+  static int on = 1;
+  return on;
+}
 
 // 0 = use every SM; otherwise the persistent kernels are launched with at most this many CTAs
 inline int& cta_limit() {
@@ -156,6 +164,26 @@ inline int launch_k1(TensorContext& tc, const void* K, const void* V, const void
       !encode_map(&tm.kpvp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 3, kpvp, dO, bO)) {
     *cuda_err = (int)cudaErrorInvalidValue;
     return -6;
+  }
+  if (stage1_pairs() && ef_heads == 0 && k % 256 == 0 && (BH * d) % 256 == 0) {
+    // two CTAs per output tile: 256 projection rows x 512 columns per pair
+    K1PairParams pp;
+    pp.N = N; pp.d = d; pp.k = k; pp.BH = BH; pp.H = H;
+    pp.col_groups = (BH * d + 511) / 512;
+    pp.k_halves = k / 256;
+    pp.nsplit = k1_choose_nsplit(tc.sm_count() / 2, 2 * pp.col_groups * pp.k_halves, (N + 63) / 64);
+    pp.status = status;
+    if (!tc.k1p_attr) {
+      cudaError_t e = cudaFuncSetAttribute(k1_down_project_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kK1PSmemBytes);
+      if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+      tc.k1p_attr = true;
+    }
+    const int pairs = 2 * pp.k_halves * pp.col_groups * pp.nsplit;
+    k1_down_project_pair<<<2 * pairs, kK1PThreads, kK1PSmemBytes, st>>>(tm.E.map, tm.F.map, tm.K.map, tm.V.map,
+                                                                        tm.kpvp.map, pp);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+    return 0;
   }
   K1Params p;
   p.N = N; p.d = d; p.k = k; p.BH = BH; p.H = H;

@@ -380,3 +380,31 @@ def test_per_head_projections_seq_major_and_host_entry():
     host_out = binding.flurka_forward_host(pinned["Q"], pinned["K"], pinned["V"], pinned["E"], pinned["F"], pinned["W"], w.variant)
     assert binding.flurka_last_status() == 0
     _check_per_head(w, x, host_out)
+
+
+# ----------------------------------------------------------------------------- stage 1 as CTA pairs
+@pytest.mark.parametrize("shape", [(1, 4, 1024, 64, 256), (2, 2, 1536, 128, 512), (1, 12, 1000, 64, 256), (3, 4, 640, 64, 512)],
+                         ids=lambda s: "B%d_H%d_N%d_d%d_k%d" % s)
+def test_stage1_pairs_and_single_ctas_match_oracle(shape):
+    """The down-projection as pairs of CTAs (two-CTA MMAs; k a multiple of 256 and B*H*d a multiple of 256)
+    and as single CTAs: K' = E K and V' = F V of every head against the oracle, both ways, with the ragged
+    last chunk, one and two 256-column halves per pair, and both halves of k = 512."""
+    B, H, N, d, k = shape
+    w = _wl("stage1_pairs", PERFORMER, "bf16", B, H, N, d, k, 64, 97 + N)
+    x = synth.make_inputs(w)
+    f64 = lambda t: t.double().numpy()
+    for on in (True, False):
+        prev = binding.flurka_set_stage1_pairs(on)
+        try:
+            out = pu.run_gpu(w, x, binding.PATH_TENSOR)
+            Kp = binding.flurka_debug_copy(0, (w.B, w.H, w.k, w.d)).cpu().double().numpy()
+            Vp = binding.flurka_debug_copy(1, (w.B, w.H, w.k, w.d)).cpu().double().numpy()
+            torch.cuda.synchronize()
+        finally:
+            binding.flurka_set_stage1_pairs(prev)
+        for b in range(B):
+            for h in range(H):
+                for got, want in ((Kp[b, h], f64(x["E"]) @ f64(x["K"][b, h])), (Vp[b, h], f64(x["F"]) @ f64(x["V"][b, h]))):
+                    assert np.abs(got - want).max() <= 3e-5 * max(1.0, np.abs(want).max())
+        got = out.cpu().double().numpy()
+        pu.assert_close(got[B - 1, H - 1], pu.oracle_head(x, w, B - 1, H - 1), "bf16", "stage 1 %s" % ("pairs" if on else "single"))
