@@ -8,8 +8,8 @@
 // loads ITS 128 rows of the E slab and ITS half of every 256-column K/V slab (48 KB per chunk for the
 // same 1024 cycles of MMA per CTA), the tensor cores of the pair read both halves of B, and each CTA
 // accumulates its 128 rows x 512 columns in its own TMEM.  The TMA loads of both CTAs count their
-// bytes on the even CTA's barrier (the data itself goes to the loading CTA only: nothing is
-// multicast); one thread of the even CTA issues the MMAs for both, and its commits arrive on the
+// bytes on the even CTA's barrier (the data itself goes to the loading CTA only, every load has one
+// destination); one thread of the even CTA issues the MMAs for both, and its commits arrive on the
 // barriers of both CTAs.  Measured against the one-CTA kernel: c4 205 -> 180 us, k = 512 of the
 // sweep 114 -> 97 us, c3 75 -> 71.5 us, c2 41 -> 39.7 us.  The epilogue is the one-CTA
 // kernel's: TMEM -> registers -> swizzled shared memory -> TMA reduce-add into the fp32 workspace.
@@ -84,7 +84,7 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
       : "memory");
 }
 // TMA load into THIS CTA's shared memory whose bytes are counted on a barrier given as a shared::cluster
-// address (it may belong to the other CTA of the pair); no multicast: the data goes to one CTA
+// address (it may belong to the other CTA of the pair); the data has one destination, this CTA
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int x,
                                                  int y, int z) {
   asm volatile(
