@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 
 #include "tc_common.cuh"
+#include "k1_down_project_pair.cuh"
 
 namespace flurka {
 
@@ -272,6 +273,174 @@ __global__ void k0_split_rows(const float* __restrict__ src, __nv_bfloat16* __re
     }
   }
   tc::grid_launch_dependents();
+}
+
+// ---------------------------------------------------------------------------------------------
+// Mode 1 (Q = Xq W^Q, bf16 store) as pairs of CTAs, the way k1_down_project_pair runs stage 1: a
+// cluster of two owns 256 rows x 512 columns, each CTA loads its 128 rows of A and its 128-column
+// half of each 256-column slab of the weights (48 KB per chunk instead of 64), both CTAs' TMA bytes
+// are counted on the even CTA's barrier, one thread of the even CTA issues tcgen05.mma.cta_group::2
+// (M = 256 over the pair, N = 256, K = 16), and each CTA stores its own 128 x 512 accumulator.
+// Needs ncols (= H d) a multiple of 256; the host uses the one-CTA kernel otherwise.
+// ---------------------------------------------------------------------------------------------
+constexpr int kK0PStages = 4;
+constexpr int kK0PStageBytes = 49152;
+constexpr int kK0PSmemBytes = kK0PStages * kK0PStageBytes + 1024 + 256;
+
+namespace tc {
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster_addr, int x,
+                                                 int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+}  // namespace tc
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kK0Threads, 1)
+k0_query_map_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmOut, const K0Params p) {
+  using namespace tc;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + kK0PStages * kK0PStageBytes;
+  const uint32_t bar_full = bar_base;                 // [4] even CTA's: the loads of both CTAs have landed
+  const uint32_t bar_empty = bar_base + 32;           // [4] the pair's MMAs have read the stage
+  const uint32_t bar_accum = bar_base + 96;
+  const uint32_t tmem_slot = bar_base + 112;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_shared;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  // ---- which piece of the problem (col_groups here counts 512-column groups)
+  int idx = blockIdx.x >> 1;
+  const int cg = idx % p.col_groups; idx /= p.col_groups;
+  const int rb = idx;
+  const int ncols = min(512, p.ncols - cg * 512);           // 256 or 512
+  const int nj = ncols >> 8;
+  const int nchunks = p.chunks;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < kK0PStages; ++i) {
+      mbar_init(bar_full + 8 * i, 1);
+      mbar_init(bar_empty + 8 * i, 1);
+    }
+    mbar_init(bar_accum, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, 512);
+    tmem_relinquish_pair();
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  if (threadIdx.x == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_shared = v;
+  }
+  cluster_sync_all();
+  const uint32_t tmem = tmem_base_shared;
+  grid_dependency_wait();
+
+  if (warp == 0) {
+    if (elect_one()) {
+      // ------------------------------------------------ TMA producer (each CTA feeds its own shared memory)
+      prefetch_tmap(&tmA);
+      prefetch_tmap(&tmB);
+      const uint32_t tx_bytes = (uint32_t)(16384 + nj * 16384);
+      bool ok = true;
+      int issued = 0;
+      for (int it = 0; it < nchunks && ok; ++it) {
+        const int st = it % kK0PStages;
+        if (it >= kK0PStages) ok = mbar_wait(bar_empty + 8 * st, ((it / kK0PStages) - 1) & 1, p.status, &abort_flag);
+        if (!ok) break;
+        const uint32_t a_dst = smem_base + st * kK0PStageBytes;
+        const uint32_t b_dst = a_dst + 16384;
+        const uint32_t fb = map_to_cta(bar_full + 8 * st, 0);
+        if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * st, 2 * tx_bytes);
+        tma_load_3d_pair(map_to_cta(a_dst, rank), &tmA, fb, it << 6, rb * 256 + (int)rank * 128, 0);
+        for (int j = 0; j < nj; ++j)
+          for (int b = 0; b < 2; ++b)
+            tma_load_2d_pair(map_to_cta(b_dst + (uint32_t)(j * 2 + b) * 8192u, rank), &tmB, fb,
+                             cg * 512 + j * 256 + (int)rank * 128 + b * 64, (it % p.b_chunks) << 6);
+        ++issued;
+      }
+      if (!ok && rank == 0) {
+        for (int it = max(0, issued - kK0PStages); it < issued; ++it)
+          (void)mbar_wait(bar_full + 8 * (it % kK0PStages), (it / kK0PStages) & 1, p.status, &abort_flag);
+      }
+    }
+  } else if (warp == 1) {
+    if (rank == 0 && elect_one()) {
+      // ------------------------------------------------ even CTA: MMA issuer for the pair
+      const uint32_t idesc = make_idesc(kFmtBF16, /*A K-major*/ 0, /*B MN-major*/ 1, 256, 256);
+      bool ok = true;
+      for (int it = 0; it < nchunks; ++it) {
+        const int st = it % kK0PStages;
+        ok = mbar_wait(bar_full + 8 * st, (it / kK0PStages) & 1, p.status, &abort_flag);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_base = smem_base + st * kK0PStageBytes;
+        const uint32_t b_base = a_base + 16384;
+        const uint64_t ad = make_sdesc(a_base, 16, 1024, kSwizzle128);
+        for (int j = 0; j < nj; ++j) {
+          const uint64_t bd = make_sdesc(b_base + j * 16384, 8192, 1024, kSwizzle128);
+          mma_ss_x4_pair(tmem + j * 256, ad, bd, 2, 128, idesc, it > 0 ? 1u : 0u);
+        }
+        mma_commit_pair(bar_empty + 8 * st);
+      }
+      if (ok) mma_commit_pair(bar_accum);
+    }
+  } else {
+    // ------------------------------------------------ epilogue: this CTA's 128 rows, bf16 slabs of [32 x 64], TMA stores
+    const int q = warp & 3;
+    bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
+    if (warp == 2 && lane == 0) grid_launch_dependents();
+    if (ok) {
+      tcgen05_fence_after();
+      const uint32_t stage_buf = smem_base + (warp - 2) * 32768;
+      const int row0 = rb * 256 + (int)rank * 128 + q * 32;
+      const int ncc = ncols >> 6;
+      for (int cc = 0; cc < ncc; ++cc) {
+        uint32_t ra[32], rb2[32];
+        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + cc * 64, ra);
+        tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + cc * 64 + 32, rb2);
+        tmem_wait_ld(ra);
+        tmem_wait_ld(rb2);
+        const uint32_t row_addr = stage_buf + cc * 4096 + lane * 128;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t* src = g < 4 ? ra : rb2;
+          uint32_t v[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(src[(g & 3) * 8 + 2 * e]),
+                                                            __uint_as_float(src[(g & 3) * 8 + 2 * e + 1]));
+            v[e] = *reinterpret_cast<const uint32_t*>(&o2);
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + ((g ^ (lane & 7)) << 4)),
+                       "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        if (row0 < p.M)
+          for (int cc = 0; cc < ncc; ++cc) tma_store_2d(&tmOut, stage_buf + cc * 4096, cg * 512 + cc * 64, row0);
+        bulk_commit_group();
+        bulk_wait_group0();
+      }
+      __syncwarp();
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) tmem_dealloc_pair(tmem, 512);
 }
 
 }  // namespace flurka

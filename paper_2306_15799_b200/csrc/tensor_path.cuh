@@ -100,6 +100,7 @@ struct TensorContext {
   bool k1_attr = false;
   bool k1p_attr = false;
   bool k0_attr = false;
+  bool k0p_attr = false;
   int sm_total() {
     if (!sms) {
       int dev = 0;
@@ -283,6 +284,19 @@ inline int launch_k0_query_map(TensorContext& tc, const void* Xq, const void* Wq
   p.row_blocks = (p.M + 255) / 256;
   p.col_groups = (H * d + 255) / 256;
   p.status = status;
+  if (stage1_pairs() && (H * d) % 256 == 0) {
+    // as pairs of CTAs: 256 rows x 512 columns per pair
+    p.col_groups = (H * d + 511) / 512;
+    if (!tc.k0p_attr) {
+      cudaError_t e = cudaFuncSetAttribute(k0_query_map_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kK0PSmemBytes);
+      if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+      tc.k0p_attr = true;
+    }
+    k0_query_map_pair<<<2 * p.row_blocks * p.col_groups, kK0Threads, kK0PSmemBytes, st>>>(tm.Xq.map, tm.Wq.map, tm.Qp.map, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+    return 0;
+  }
   int rc = k0_set_attr(tc, cuda_err);
   if (rc) return rc;
   k0_linear_map<<<p.row_blocks * p.col_groups, kK0Threads, kK0SmemBytes, st>>>(tm.Xq.map, tm.Wq.map, tm.Wq.map,

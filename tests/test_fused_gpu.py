@@ -75,6 +75,10 @@ TENSOR_CASES = [
     _fw("fused_perf_dm64_one_head", PERFORMER, "bf16", 3, 1, 200, 64, 64, 64, 64, 74),
     _fw("fused_rnn_d128_k64", RNN, "bf16", 1, 1, 136, 128, 128, 64, 0, 75),
     _fw("fused_perf_wide_dm", PERFORMER, "bf16", 1, 2, 256, 1024, 64, 128, 192, 76, shared_x=False),
+    # H d a multiple of 256 (the query map runs as pairs of CTAs): one 512-column group with a ragged last row
+    # block, and a 512-column group followed by a 256-column one
+    _fw("fused_perf_hd512_ragged_rows", PERFORMER, "bf16", 1, 8, 1000, 192, 64, 128, 128, 77),
+    _fw("fused_perf_hd768", PERFORMER, "bf16", 2, 12, 640, 128, 64, 256, 64, 78, shared_x=False),
 ]
 
 
@@ -91,6 +95,15 @@ def test_fused_tensor_path_with_few_ctas(limit):
         _check(_fw("fused_perf_few_ctas", PERFORMER, "bf16", 1, 2, 896, 128, 64, 128, 128, 67), binding.PATH_TENSOR)
     finally:
         binding.flurka_set_cta_limit(prev)
+
+
+def test_fused_tensor_path_without_cta_pairs():
+    """The one-CTA kernels of the query map and of stage 1 on a shape that otherwise runs as pairs."""
+    prev = binding.flurka_set_stage1_pairs(0)
+    try:
+        _check(_fw("fused_perf_hd512_single_ctas", PERFORMER, "bf16", 1, 8, 1000, 192, 64, 256, 128, 79), binding.PATH_TENSOR)
+    finally:
+        binding.flurka_set_stage1_pairs(prev)
 
 
 SIMT_CASES = [
