@@ -810,8 +810,13 @@ namespace {
 // memset), then dK', dV' [2][BH][k][d]; all fp32.
 struct BackwardLayout {
   Layout L;
-  size_t da, dab_bytes, db, dkpvp, total;
+  size_t da, dab_bytes, db, dkpvp, abf, total;
 };
+
+// the query side of the backward has a tensor-core kernel for PERFORMER with d = 64 and 128 or 256 features
+bool backward_tensor_ok(const Problem& pr) {
+  return tensor_path_ok(pr) && pr.kernel == FLURKA_PERFORMER && pr.d == 64 && (pr.m == 128 || pr.m == 256);
+}
 
 BackwardLayout make_backward_layout(const Problem& pr) {
   BackwardLayout b;
@@ -823,6 +828,8 @@ BackwardLayout make_backward_layout(const Problem& pr) {
   b.dab_bytes = da_bytes + (size_t)pr.BH() * pr.p() * 4;
   off = align256(off + b.dab_bytes);
   b.dkpvp = off; off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
+  b.abf = off;
+  if (backward_tensor_ok(pr)) off = align256(off + (size_t)2 * pr.BH() * pr.p() * pr.d * 2);   // a as two bf16 terms
   b.total = off;
   return b;
 }
@@ -830,7 +837,8 @@ BackwardLayout make_backward_layout(const Problem& pr) {
 template <typename T, bool P>
 int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, const void* Q, const void* K,
                       const void* V, const void* E, const void* F, const void* W, const void* dO, void* dQ, void* dK,
-                      void* dV, void* dE, void* dF, cudaStream_t st, int* launches) {
+                      void* dV, void* dE, void* dF, cudaStream_t st, int* launches, TensorContext* tc) {
+  // tc != NULL: stage 1 and the query side run on the tensor-core kernels (bf16 PERFORMER, d = 64)
   const Layout& L = BL.L;
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
@@ -843,11 +851,24 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
   if (e != cudaSuccess) return cuda_fail(e);
   if ((e = cudaMemsetAsync(da, 0, BL.dab_bytes, st)) != cudaSuccess) return cuda_fail(e);
   // the forward's stages 1 and 2 again: K', V', a_i, b_i (or z_i)
-  int rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
-  if (rc) return rc;
+  int rc = FLURKA_OK;
+  int cuda_err = 0;
+  if (tc) {
+    rc = launch_k1(*tc, K, V, E, F, kpvp, pr.BH(), smh, pr.N, pr.d, pr.k, (int*)(ws + L.status), st, &cuda_err, efh);
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
+    ++*launches;
+  } else {
+    rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
+    if (rc) return rc;
+  }
   rc = launch_simt_key_side<T, P>(pr, kpvp, W, weight, a32, nullptr, st, launches);
   if (rc) return rc;
-  {
+  if (tc) {
+    rc = launch_k4(*tc, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.p(),
+                   (int*)(ws + L.status), st, &cuda_err);
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
+    *launches += 2;
+  } else {
     auto fn = simt_bwd_query_side<T, P>;
     const size_t smem = ((size_t)2 * 32 * (pr.d + 1) + 32 * 33 + 32 * pr.d) * 4;
     if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
@@ -921,17 +942,23 @@ int flurka_backward(const void* Q, const void* K, const void* V, const void* E, 
   if (rc) return rc;
   int launches = 0;
   const bool perf = pr.kernel == FLURKA_PERFORMER;
+  // tensor-core kernels for stage 1 and the query side where the shape allows (and the path knob does not
+  // force the CUDA-core kernels); a forced tensor path with another shape is refused
+  const bool tensor_ok = backward_tensor_ok(pr);
+  if (g_path >= FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
+  TensorContext* tc = (tensor_ok && g_path != FLURKA_PATH_SIMT) ? &ds.tc : nullptr;
   if (pr.fp32)
-    rc = perf ? backward_pipeline<float, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches)
-              : backward_pipeline<float, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches);
+    rc = perf ? backward_pipeline<float, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, nullptr)
+              : backward_pipeline<float, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches,
+                                                nullptr);
   else
-    rc = perf ? backward_pipeline<__nv_bfloat16, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches)
+    rc = perf ? backward_pipeline<__nv_bfloat16, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, tc)
               : backward_pipeline<__nv_bfloat16, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st,
-                                                        &launches);
+                                                        &launches, nullptr);
   if (rc) return rc;
   ds.partial_pending = false;
   ds.timer.have = false;
-  ds.last_path = FLURKA_PATH_SIMT;
+  ds.last_path = tc ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
   ds.last_launches = launches;
   ds.have_last = true;
   ds.last_problem = pr;

@@ -1,0 +1,429 @@
+// Backward of the query side on tensor cores (PERFORMER, bf16, d = 64, p = 128 or 256 features).
+//
+// The forward's query side (arxiv 2306.15799, Eq. (2) with the normalised weights of Appendix D) is
+//     O_n = sum_i P_ni a_i,    P_n. = softmax_i(l_n.),    l_ni = w_i . q_n + b_i.
+// The paper trains through it but prints no backward formulas; by the chain rule, given dO,
+//     g_ni = dO_n . a_i,   delta_n = sum_i P_ni g_ni,   c_ni = P_ni (g_ni - delta_n),
+//     dq_n = sum_i c_ni w_i,   da_i = sum_n P_ni dO_n,   db_i = sum_n c_ni = a_i . da_i - sum_n P_ni delta_n.
+// Per tile of 128 query rows every product is a tcgen05 MMA with fp32 accumulators in TMEM:
+//     S = Q W^T + 1 b^T  and  G = dO a^T  (a as two bf16 terms, so g is exact to 2^-17),
+//     dQ = C W  (C = bf16 c, the A operand read from TMEM),
+//     da += P^T dO  and  (P^T delta) += P^T [delta_hi delta_mid delta_lo]  (P = bf16, written to shared memory
+//     by the row owners in the canonical 128-byte-swizzled layout, used as an MN-major A operand),
+// in two sweeps over the features, 128 at a time: the first gives each row its log-sum-exp and
+// delta_n (running maximum, sum and P-weighted sum of g), the second forms P and c.  da and P^T delta
+// stay in TMEM over all the tiles a CTA has of one head and are added to global memory (atomics) when
+// the head changes; db comes from them there.  One thread per query row (4 warps), one MMA issuer, one
+// TMA thread; the phases of a tile follow one another (block barriers), nothing here waits for another CTA.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "tc_common.cuh"
+
+namespace flurka {
+
+struct K4Params {
+  int N, p, BH, H;              // H > 0: Q, dO, dQ are [B,N,H,64]; H == 0: [BH,N,64]
+  int tiles_per_head, total_tiles;
+  const float* weight;          // [BH][p]      b_i
+  const float* a32;             // [BH][p][64]  a_i (fp32)
+  __nv_bfloat16* dQ;
+  float* da;                    // [BH][p][64]  added to
+  float* db;                    // [BH][p]      added to
+  int* status;
+};
+
+constexpr int kK4Threads = 192;
+// shared memory: W 32 KB | a_hi 32 KB | a_lo 32 KB | 2 x (Q tile 16 KB, dO tile 16 KB) | P tile 32 KB |
+// ones 4 KB | bias 8 KB | delta 4 KB | barriers
+constexpr uint32_t kK4W = 0, kK4AHi = 32768, kK4ALo = 65536, kK4In = 98304, kK4P = 163840, kK4Ones = 196608,
+                   kK4Bias = 200704, kK4Delta = 208896, kK4Bars = 212992;
+constexpr int kK4SmemBytes = 212992 + 256 + 1024;
+// TMEM columns: S 0..127 (c as bf16 pairs over 0..63), G 128..255, dQ 256..319, da 320..447 (two
+// 128-feature tiles of 64 columns), P^T delta 448..479 (two tiles of 16 columns)
+constexpr uint32_t kK4ColG = 128, kK4ColDQ = 256, kK4ColDA = 320, kK4ColDD = 448;
+
+__device__ __forceinline__ uint32_t k4_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %2, %1;" : "=r"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ float k4_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// a [BH][p][64] fp32 -> two bf16 terms, [BH][2][p][64]
+__global__ void k4_split_a(const float* __restrict__ a32, __nv_bfloat16* __restrict__ abf, int BH, int p) {
+  const long long per_head = (long long)p * 64;
+  const long long total = (long long)BH * per_head;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long h = i / per_head, r = i % per_head;
+    const float x = a32[i];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    abf[(h * 2) * per_head + r] = hi;
+    abf[(h * 2 + 1) * per_head + r] = __float2bfloat16_rn(x - __bfloat162float(hi));
+  }
+}
+
+__global__ void __launch_bounds__(kK4Threads, 1)
+k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
+                  const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
+                  const K4Params prm) {
+  using namespace tc;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + kK4Bars;
+  const uint32_t bar_w = bars, bar_head = bars + 8, bar_in = bars + 16 /* [2] */, bar_mma = bars + 32,
+                 bar_mma2 = bars + 40, tmem_slot = bars + 48;
+  __shared__ int abort_flag;
+  __shared__ uint32_t tmem_base_shared;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int p = prm.p, nh = p >> 7;
+  const bool owner = warp >= 2;
+  const int q4 = warp & 3, row = q4 * 32 + lane;
+  const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+
+  const int t_begin = (int)(((long long)blockIdx.x * prm.total_tiles) / gridDim.x);
+  const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.total_tiles) / gridDim.x);
+  const int ntiles = t_end - t_begin;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(bar_w, 1);
+    mbar_init(bar_head, 1);
+    mbar_init(bar_in, 1);
+    mbar_init(bar_in + 8, 1);
+    mbar_init(bar_mma, 1);
+    mbar_init(bar_mma2, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  if (warp == 2) {
+    // the all-ones A operand of the bias step: [128 x 16] bf16, no swizzle, columns 0..2 are 1
+    // (element (r, c) at (r/8)*256 + (c/8)*128 + (r%8)*16 + (c%8)*2 bytes)
+    __nv_bfloat16* ones = reinterpret_cast<__nv_bfloat16*>(base_ptr + kK4Ones);
+    for (int e = lane; e < 128 * 16; e += 32) {
+      const int r = e >> 4, c = e & 15;
+      ones[(r >> 3) * 128 + (c >> 3) * 64 + (r & 7) * 8 + (c & 7)] = __float2bfloat16_rn(c < 3 ? 1.f : 0.f);
+    }
+  }
+  if (warp == 3) {
+    // the delta operand [16 x 128] (K-major, no swizzle): rows 0..2 are rewritten per tile, the rest stays zero
+    uint32_t* dz = reinterpret_cast<uint32_t*>(base_ptr + kK4Delta);
+    for (int e = lane; e < 1024; e += 32) dz[e] = 0u;
+  }
+  fence_proxy_async_smem();
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  if (tid == 0) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(tmem_slot));
+    tmem_base_shared = v;
+  }
+  __syncthreads();
+  const uint32_t tmem = tmem_base_shared;
+
+  auto load_tile = [&](int i) {
+    const int tile = t_begin + i;
+    const int head = tile / prm.tiles_per_head;
+    const int row0 = (tile % prm.tiles_per_head) * 128;
+    const uint32_t st = (uint32_t)(i & 1);
+    const uint32_t dst = base + kK4In + st * 32768u;
+    mbar_arrive_expect_tx(bar_in + 8 * st, 32768u);
+    if (prm.H > 0) {
+      tma_load_3d(dst, &tmQ, bar_in + 8 * st, (head % prm.H) * 64, row0, head / prm.H);
+      tma_load_3d(dst + 16384, &tmDO, bar_in + 8 * st, (head % prm.H) * 64, row0, head / prm.H);
+    } else {
+      tma_load_3d(dst, &tmQ, bar_in + 8 * st, 0, row0, head);
+      tma_load_3d(dst + 16384, &tmDO, bar_in + 8 * st, 0, row0, head);
+    }
+  };
+
+  // da, P^T delta of one head leave TMEM: thread = feature; db from the identity in the header
+  auto flush = [&](int head) {
+    if (!owner) return;
+    tcgen05_fence_after();
+    for (int hh = 0; hh < nh; ++hh) {
+      uint32_t dd[32];                       // columns 0..2 are this tile's P^T delta terms (the load is 32 wide)
+      tmem_ld32(tmem + lane_off + kK4ColDD + hh * 16, dd);
+      tmem_wait_ld(dd);
+      const int feat = hh * 128 + row;
+      const float* arow = prm.a32 + ((size_t)head * p + feat) * 64;
+      float* darow = prm.da + ((size_t)head * p + feat) * 64;
+      float dot = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < 64; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_off + kK4ColDA + hh * 64 + c, r);
+        tmem_wait_ld(r);
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 av = *reinterpret_cast<const float4*>(arow + c + e);
+          dot = fmaf(av.x, __uint_as_float(r[e]), dot);
+          dot = fmaf(av.y, __uint_as_float(r[e + 1]), dot);
+          dot = fmaf(av.z, __uint_as_float(r[e + 2]), dot);
+          dot = fmaf(av.w, __uint_as_float(r[e + 3]), dot);
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) atomicAdd(darow + c + e, __uint_as_float(r[e]));
+      }
+      const float pd = __uint_as_float(dd[0]) + __uint_as_float(dd[1]) + __uint_as_float(dd[2]);
+      atomicAdd(prm.db + (size_t)head * p + feat, dot - pd);
+    }
+    tcgen05_fence_before();
+  };
+
+  bool ok = true;
+  uint32_t ph_mma = 0, ph_mma2 = 0, ph_head = 0;
+  int head_prev = -1;
+  bool first_of_head = true;
+  const float kLog2e = 1.4426950408889634f;
+  const uint32_t idescS = make_idesc(kFmtBF16, 0, 0, 128, 128);   // S, G: both operands K-major
+  const uint32_t idescQ = make_idesc(kFmtBF16, 0, 1, 128, 64);    // dQ: A from TMEM, W as an MN-major B
+  const uint32_t idescA = make_idesc(kFmtBF16, 1, 1, 128, 64);    // da: P^T (MN-major A) x dO (MN-major B)
+  const uint32_t idescD = make_idesc(kFmtBF16, 1, 0, 128, 16);    // P^T delta: delta as a K-major B
+
+  if (ntiles > 0 && tid == 0) {
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmDO);
+    prefetch_tmap(&tmW);
+    prefetch_tmap(&tmA);
+    mbar_arrive_expect_tx(bar_w, (uint32_t)p * 128u);
+    tma_load_2d(base + kK4W, &tmW, bar_w, 0, 0);
+    load_tile(0);
+  }
+  if (ntiles > 0) {
+    const bool mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
+    ok = __syncthreads_and(mine) != 0;
+  }
+
+  for (int i = 0; i < ntiles && ok; ++i) {
+    const int tile = t_begin + i;
+    const int head = tile / prm.tiles_per_head;
+    const int row0 = (tile % prm.tiles_per_head) * 128;
+    const uint32_t st = (uint32_t)(i & 1);
+    const uint32_t sm_q = base + kK4In + st * 32768u, sm_do = sm_q + 16384u;
+
+    if (head != head_prev) {
+      // every MMA issued so far has completed (the last wait of the previous tile), so the accumulators
+      // of the old head can leave and its operands can be replaced
+      if (head_prev >= 0) flush(head_prev);
+      __syncthreads();
+      if (tid == 0) {
+        mbar_arrive_expect_tx(bar_head, 2u * (uint32_t)p * 128u);
+        tma_load_3d(base + kK4AHi, &tmA, bar_head, 0, 0, head * 2);
+        tma_load_3d(base + kK4ALo, &tmA, bar_head, 0, 0, head * 2 + 1);
+      }
+      if (warp == 1) {
+        // bias[f][c], c < 16, no swizzle: b_f - max b as three bf16 terms in columns 0..2
+        const float* wv = prm.weight + (size_t)head * p;
+        float mx = -INFINITY;
+        for (int f = lane; f < p; f += 32) mx = fmaxf(mx, wv[f]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        __nv_bfloat16* bias = reinterpret_cast<__nv_bfloat16*>(base_ptr + kK4Bias);
+        for (int f = lane; f < 256; f += 32) {
+          float b = (f < p) ? wv[f] - mx : 0.f;
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(b);  b -= __bfloat162float(h0);
+          const __nv_bfloat16 h1 = __float2bfloat16_rn(b);  b -= __bfloat162float(h1);
+          const __nv_bfloat16 h2 = __float2bfloat16_rn(b);
+          __nv_bfloat16* rowp = bias + (f >> 3) * 128 + (f & 7) * 8;
+          rowp[0] = h0; rowp[1] = h1; rowp[2] = h2;
+#pragma unroll
+          for (int c = 3; c < 8; ++c) rowp[c] = __float2bfloat16_rn(0.f);
+#pragma unroll
+          for (int c = 0; c < 8; ++c) rowp[64 + c] = __float2bfloat16_rn(0.f);
+        }
+        fence_proxy_async_smem();
+      }
+      const bool mine = mbar_wait(bar_head, ph_head, prm.status, &abort_flag);
+      ph_head ^= 1;
+      ok = __syncthreads_and(mine) != 0;
+      if (!ok) break;
+      head_prev = head;
+      first_of_head = true;
+    }
+    // the other stage held tile i-1, which is complete: fetch tile i+1 into it
+    if (tid == 0 && i + 1 < ntiles) load_tile(i + 1);
+    {
+      const bool mine = mbar_wait(bar_in + 8 * st, (uint32_t)(i >> 1) & 1u, prm.status, &abort_flag);
+      ok = __syncthreads_and(mine) != 0;
+      if (!ok) break;
+    }
+
+    auto issue_sg = [&](int h) {
+      tcgen05_fence_after();
+      const uint64_t aq = make_sdesc(sm_q, 16, 1024, kSwizzle128);
+      const uint64_t bw = make_sdesc(base + kK4W + h * 16384, 16, 1024, kSwizzle128);
+      mma_ss_x4(tmem, aq, bw, 2, 2, idescS, 0u);
+      const uint64_t a1 = make_sdesc(base + kK4Ones, 128, 256, kSwizzleNone);
+      const uint64_t b1 = make_sdesc(base + kK4Bias + h * 4096, 128, 256, kSwizzleNone);
+      mma_ss(tmem, a1, b1, idescS, 1u);
+      const uint64_t ag = make_sdesc(sm_do, 16, 1024, kSwizzle128);
+      const uint64_t bh = make_sdesc(base + kK4AHi + h * 16384, 16, 1024, kSwizzle128);
+      const uint64_t bl = make_sdesc(base + kK4ALo + h * 16384, 16, 1024, kSwizzle128);
+      mma_ss_x4(tmem + kK4ColG, ag, bh, 2, 2, idescS, 0u);
+      mma_ss_x4(tmem + kK4ColG, ag, bl, 2, 2, idescS, 1u);
+      mma_commit(bar_mma);
+    };
+
+    // ------------------------------------------------------------ sweep 1: log-sum-exp and delta of each row
+    float mx = -INFINITY, den = 0.f, num = 0.f;     // mx in the base-2 domain
+    for (int h = 0; h < nh && ok; ++h) {
+      if (tid == 32) issue_sg(h);
+      bool mine = true;
+      if (owner) {
+        mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
+        if (mine) {
+          tcgen05_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < 128; c += 32) {
+            uint32_t rs[32], rg[32];
+            tmem_ld32(tmem + lane_off + c, rs);
+            tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
+            tmem_wait_ld(rs);
+            tmem_wait_ld(rg);
+            float cm = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) cm = fmax3(cm, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]));
+            const float nm = fmaxf(mx, cm * kLog2e);
+            const float sc = k4_ex2(mx - nm);
+            den *= sc;
+            num *= sc;
+            mx = nm;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float pe = k4_ex2(fmaf(__uint_as_float(rs[e]), kLog2e, -mx));
+              den += pe;
+              num = fmaf(pe, __uint_as_float(rg[e]), num);
+            }
+          }
+          tcgen05_fence_before();
+        }
+      }
+      ph_mma ^= 1;
+      ok = __syncthreads_and(mine) != 0;          // S, G have been read out
+    }
+    if (!ok) break;
+    const float lse2 = mx + __log2f(den);
+    const float delta = num / den;
+    if (owner) {
+      // delta_n as three bf16 terms: element (c, n) of the [16 x 128] operand at (n/8)*128 + c*16 + (n%8)*2 bytes
+      __nv_bfloat16* dt = reinterpret_cast<__nv_bfloat16*>(base_ptr + kK4Delta) + (row >> 3) * 64 + (row & 7);
+      float r = delta;
+      const __nv_bfloat16 d0 = __float2bfloat16_rn(r);  r -= __bfloat162float(d0);
+      const __nv_bfloat16 d1 = __float2bfloat16_rn(r);  r -= __bfloat162float(d1);
+      const __nv_bfloat16 d2 = __float2bfloat16_rn(r);
+      dt[0] = d0; dt[8] = d1; dt[16] = d2;
+    }
+
+    // ------------------------------------------------------------ sweep 2: P, c and the three products they feed
+    for (int h = 0; h < nh && ok; ++h) {
+      if (tid == 32) issue_sg(h);
+      bool mine = true;
+      if (owner) {
+        mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
+        if (mine) {
+          tcgen05_fence_after();
+          const uint32_t prow = base + kK4P + (uint32_t)row * 128u;
+#pragma unroll 1
+          for (int c = 0; c < 128; c += 32) {
+            uint32_t rs[32], rg[32], cw[16];
+            tmem_ld32(tmem + lane_off + c, rs);
+            tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
+            tmem_wait_ld(rs);
+            tmem_wait_ld(rg);
+            const uint32_t slab = prow + (uint32_t)(c >> 6) * 16384u;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint32_t pw[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int j = 8 * g + 2 * e;
+                const float p0 = k4_ex2(fmaf(__uint_as_float(rs[j]), kLog2e, -lse2));
+                const float p1 = k4_ex2(fmaf(__uint_as_float(rs[j + 1]), kLog2e, -lse2));
+                pw[e] = k4_bf16x2(p0, p1);
+                cw[4 * g + e] = k4_bf16x2(p0 * (__uint_as_float(rg[j]) - delta), p1 * (__uint_as_float(rg[j + 1]) - delta));
+              }
+              const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + g);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + ((chunk ^ (uint32_t)(row & 7)) << 4)),
+                           "r"(pw[0]), "r"(pw[1]), "r"(pw[2]), "r"(pw[3]) : "memory");
+            }
+            tmem_st16(tmem + lane_off + (c >> 1), cw);
+          }
+          tmem_wait_st();
+          fence_proxy_async_smem();
+          tcgen05_fence_before();
+        }
+      }
+      ph_mma ^= 1;
+      ok = __syncthreads_and(mine) != 0;
+      if (!ok) break;
+      if (tid == 32) {
+        tcgen05_fence_after();
+        // dQ (+)= c W: 128 features = 8 steps of 16, A 8 columns per step, B 16 rows of W per step
+        for (int j = 0; j < 2; ++j) {
+          const uint64_t bw = make_sdesc(base + kK4W + h * 16384 + j * 8192, 8192, 1024, kSwizzle128);
+          mma_ts_x4(tmem + kK4ColDQ, tmem + j * 32, bw, 128, idescQ, (h > 0 || j > 0) ? 1u : 0u);
+        }
+        // da_h (+)= P_h^T dO and (P^T delta)_h: 128 rows = 8 steps of 16 rows (2048 B of P and of dO, 256 B of delta)
+        for (int j = 0; j < 2; ++j) {
+          const uint64_t ap = make_sdesc(base + kK4P + j * 8192, 16384, 1024, kSwizzle128);
+          const uint64_t bo = make_sdesc(sm_do + j * 8192, 8192, 1024, kSwizzle128);
+          mma_ss_x4(tmem + kK4ColDA + h * 64, ap, bo, 128, 128, idescA, (!first_of_head || j > 0) ? 1u : 0u);
+          const uint64_t bd = make_sdesc(base + kK4Delta + j * 1024, 128, 2048, kSwizzleNone);
+          mma_ss_x4(tmem + kK4ColDD + h * 16, ap, bd, 128, 16, idescD, (!first_of_head || j > 0) ? 1u : 0u);
+        }
+        mma_commit(bar_mma2);
+      }
+      // c, P and (after the last half) dQ: wait for these products before anything is overwritten or read
+      mine = mbar_wait(bar_mma2, ph_mma2, prm.status, &abort_flag);
+      ph_mma2 ^= 1;
+      ok = __syncthreads_and(mine) != 0;
+    }
+    if (!ok) break;
+    first_of_head = false;
+
+    // ------------------------------------------------------------ dQ rows
+    if (owner) {
+      tcgen05_fence_after();
+      uint32_t ra[32], rb[32];
+      tmem_ld32(tmem + lane_off + kK4ColDQ, ra);
+      tmem_ld32(tmem + lane_off + kK4ColDQ + 32, rb);
+      tmem_wait_ld(ra);
+      tmem_wait_ld(rb);
+      tcgen05_fence_before();
+      if (row0 + row < prm.N) {
+        __nv_bfloat16* orow = prm.H > 0
+            ? prm.dQ + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * 64
+            : prm.dQ + ((size_t)head * prm.N + row0 + row) * 64;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t* src = g < 4 ? ra : rb;
+          uint4 v;
+          v.x = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 0]), __uint_as_float(src[(g & 3) * 8 + 1]));
+          v.y = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 2]), __uint_as_float(src[(g & 3) * 8 + 3]));
+          v.z = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 4]), __uint_as_float(src[(g & 3) * 8 + 5]));
+          v.w = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 6]), __uint_as_float(src[(g & 3) * 8 + 7]));
+          *reinterpret_cast<uint4*>(orow + g * 8) = v;
+        }
+      }
+    }
+    __syncthreads();      // dQ has been read: the next tile may overwrite it
+  }
+  if (ok && head_prev >= 0) flush(head_prev);
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace flurka

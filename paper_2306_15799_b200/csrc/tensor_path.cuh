@@ -11,6 +11,7 @@
 #include "k1_down_project_pair.cuh"
 #include "k2_key_side.cuh"
 #include "k3_query_side.cuh"
+#include "k4_bwd_query_side.cuh"
 
 namespace flurka {
 
@@ -89,6 +90,7 @@ inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int ran
 
 struct TensorMaps {
   CachedMap E, F, K, V, kpvp, Q, W, W2, aT, O;
+  CachedMap dO, abf;                            // backward of the query side
   CachedMap A3, Wk, Wv, Xq, Wq, Qp, kpvp2;      // the linear maps of the entry point with un-projected inputs
 };
 
@@ -427,6 +429,50 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
   e = launch_after_predecessor(fn, grid, kK3Threads, L.total, st, tm.Q.map, performer ? tm.W.map : tm.Q.map,
                                tm.aT.map, d == 64 ? tm.O.map : tm.Q.map, prm);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
+
+// ---- backward of the query side (PERFORMER, d = 64, p = 128 or 256): dQ, and da, db added to ---------
+// abf: scratch for the two bf16 terms of a, [BH][2][p][64]
+inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const void* W, const float* a32,
+                     const float* weight, __nv_bfloat16* abf, void* dQ, float* da, float* db, int BH, int H, int N,
+                     int p, int* status, cudaStream_t st, int* cuda_err) {
+  TensorMaps& tm = tc.maps;
+  const int d = 64;
+  const unsigned long long dQd[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
+                                     (unsigned long long)(H > 0 ? BH / H : BH)};
+  const unsigned bQ[3] = {64, 128, 1};
+  const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
+  const unsigned bW[2] = {64, (unsigned)p};
+  const unsigned long long dA[3] = {(unsigned long long)d, (unsigned long long)p, (unsigned long long)BH * 2};
+  const unsigned bA[3] = {64, (unsigned)p, 1};
+  if (!encode_map(&tm.Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Q, dQd, bQ) ||
+      !encode_map(&tm.dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, dO, dQd, bQ) ||
+      !encode_map(&tm.W, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW) ||
+      !encode_map(&tm.abf, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, abf, dA, bA)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  {
+    const long long total = (long long)BH * p * 64;
+    int grid = (int)((total + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    k4_split_a<<<grid, 256, 0, st>>>(a32, abf, BH, p);
+  }
+  K4Params prm;
+  prm.N = N; prm.p = p; prm.BH = BH; prm.H = H;
+  prm.tiles_per_head = (N + 127) / 128;
+  prm.total_tiles = prm.tiles_per_head * BH;
+  prm.weight = weight; prm.a32 = a32;
+  prm.dQ = reinterpret_cast<__nv_bfloat16*>(dQ);
+  prm.da = da; prm.db = db; prm.status = status;
+  cudaError_t e = cudaFuncSetAttribute(k4_bwd_query_side, cudaFuncAttributeMaxDynamicSharedMemorySize, kK4SmemBytes);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  int grid = tc.sm_count();
+  if (grid > prm.total_tiles) grid = prm.total_tiles;
+  k4_bwd_query_side<<<grid, kK4Threads, kK4SmemBytes, st>>>(tm.Q.map, tm.dO.map, tm.W.map, tm.abf.map, prm);
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;

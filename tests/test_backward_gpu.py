@@ -78,6 +78,41 @@ def test_backward_matches_oracle(w):
     _check(w)
 
 
+TENSOR_CASES = [
+    # bf16 PERFORMER with d = 64 and 128 or 256 features: stage 1 and the query side on the tensor-core kernels
+    Workload("bwd_tc_m256", PERFORMER, "bf16", 1, 3, 520, 64, 64, 256, 311),
+    Workload("bwd_tc_m128", PERFORMER, "bf16", 2, 2, 384, 64, 128, 128, 312),
+    Workload("bwd_tc_m256_k256", PERFORMER, "bf16", 1, 2, 1000, 64, 256, 256, 313),
+]
+
+
+@pytest.mark.parametrize("w", TENSOR_CASES, ids=lambda w: w.name)
+def test_backward_tensor_path_matches_oracle(w):
+    _check(w)
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+
+
+@pytest.mark.parametrize("limit", [1, 2])
+def test_backward_tensor_path_with_few_ctas(limit):
+    """A CTA's tiles cross from one head to the next: its accumulators of da, db leave and start again."""
+    prev = binding.flurka_set_cta_limit(limit)
+    try:
+        _check(Workload("bwd_tc_few_ctas", PERFORMER, "bf16", 1, 3, 520, 64, 64, 256, 314))
+        _check(Workload("bwd_tc_few_ctas_bnhd", PERFORMER, "bf16", 2, 2, 264, 64, 64, 128, 315), layout="bnhd")
+        assert binding.flurka_last_path() == binding.PATH_TENSOR
+    finally:
+        binding.flurka_set_cta_limit(prev)
+
+
+def test_backward_cuda_core_path_on_a_tensor_shape():
+    prev = binding.flurka_set_path(binding.PATH_SIMT)
+    try:
+        _check(Workload("bwd_simt_on_tc_shape", PERFORMER, "bf16", 1, 2, 264, 64, 64, 128, 316))
+        assert binding.flurka_last_path() == binding.PATH_SIMT
+    finally:
+        binding.flurka_set_path(prev)
+
+
 def test_backward_seq_major_layout_and_per_head_projections():
     _check(Workload("bwd_bnhd", PERFORMER, "fp32", 2, 3, 64, 16, 8, 24, 306), layout="bnhd")
     _check(Workload("bwd_per_head", RNN, "fp32", 2, 2, 64, 16, 8, 0, 307), per_head=True)
