@@ -810,7 +810,7 @@ namespace {
 // memset), then dK', dV' [2][BH][k][d]; all fp32.
 struct BackwardLayout {
   Layout L;
-  size_t da, dab_bytes, db, dkpvp, abf, total;
+  size_t da, dab_bytes, db, dkpvp, abf, split, total;
 };
 
 // the query side of the backward has a tensor-core kernel for PERFORMER with d = 64 and 128 or 256 features
@@ -830,6 +830,8 @@ BackwardLayout make_backward_layout(const Problem& pr) {
   b.dkpvp = off; off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
   b.abf = off;
   if (backward_tensor_ok(pr)) off = align256(off + (size_t)2 * pr.BH() * pr.p() * pr.d * 2);   // a as two bf16 terms
+  b.split = off;
+  if (tensor_path_ok(pr)) off = align256(off + (size_t)2 * pr.k * 2 * pr.BH() * pr.d * 2);      // dK', dV' as two bf16 terms
   b.total = off;
   return b;
 }
@@ -837,8 +839,9 @@ BackwardLayout make_backward_layout(const Problem& pr) {
 template <typename T, bool P>
 int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, const void* Q, const void* K,
                       const void* V, const void* E, const void* F, const void* W, const void* dO, void* dQ, void* dK,
-                      void* dV, void* dE, void* dF, cudaStream_t st, int* launches, TensorContext* tc) {
-  // tc != NULL: stage 1 and the query side run on the tensor-core kernels (bf16 PERFORMER, d = 64)
+                      void* dV, void* dE, void* dF, cudaStream_t st, int* launches, TensorContext* tc, bool tcq) {
+  // tc != NULL: stage 1 and (with shared E, F) the projection gradients run on the tensor-core kernels;
+  // tcq: so does the query side (bf16 PERFORMER, d = 64, 128 or 256 features)
   const Layout& L = BL.L;
   float* kpvp = (float*)(ws + L.kpvp);
   float* weight = (float*)(ws + L.weight);
@@ -863,7 +866,7 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
   }
   rc = launch_simt_key_side<T, P>(pr, kpvp, W, weight, a32, nullptr, st, launches);
   if (rc) return rc;
-  if (tc) {
+  if (tc && tcq) {
     rc = launch_k4(*tc, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.p(),
                    (int*)(ws + L.status), st, &cuda_err);
     if (rc) { g_last_cuda_error = cuda_err; return rc; }
@@ -887,7 +890,12 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
     fn<<<grid, 256, smem, st>>>(kpvp, (const T*)W, weight, a32, da, db, dkpvp, pr.BH(), pr.d, pr.k, pr.p());
     ++*launches;
   }
-  {
+  if (tc && efh == 0) {
+    rc = launch_k5(*tc, E, F, K, V, dkpvp, (__nv_bfloat16*)(ws + BL.split), dK, dV, dE, dF, pr.BH(), smh, pr.N, pr.d, pr.k,
+                   (int*)(ws + L.status), st, &cuda_err);
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
+    *launches += 3;
+  } else {
     dim3 grid((pr.N + 31) / 32, pr.BH(), 2);
     simt_bwd_inputs<T><<<grid, 256, 0, st>>>((const T*)E, (const T*)F, dkpvp, (T*)dK, (T*)dV, pr.BH(), pr.N, pr.d,
                                              pr.k, smh, efh);
@@ -946,19 +954,20 @@ int flurka_backward(const void* Q, const void* K, const void* V, const void* E, 
   // force the CUDA-core kernels); a forced tensor path with another shape is refused
   const bool tensor_ok = backward_tensor_ok(pr);
   if (g_path >= FLURKA_PATH_TENSOR && !tensor_ok) return FLURKA_ERR_SHAPE;
-  TensorContext* tc = (tensor_ok && g_path != FLURKA_PATH_SIMT) ? &ds.tc : nullptr;
+  TensorContext* tc = (tensor_path_ok(pr) && g_path != FLURKA_PATH_SIMT) ? &ds.tc : nullptr;
+  const bool tcq = tc && tensor_ok;
   if (pr.fp32)
-    rc = perf ? backward_pipeline<float, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, nullptr)
+    rc = perf ? backward_pipeline<float, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, nullptr, false)
               : backward_pipeline<float, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches,
-                                                nullptr);
+                                                nullptr, false);
   else
-    rc = perf ? backward_pipeline<__nv_bfloat16, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, tc)
+    rc = perf ? backward_pipeline<__nv_bfloat16, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, tc, tcq)
               : backward_pipeline<__nv_bfloat16, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st,
-                                                        &launches, nullptr);
+                                                        &launches, tc, false);
   if (rc) return rc;
   ds.partial_pending = false;
   ds.timer.have = false;
-  ds.last_path = tc ? FLURKA_PATH_TENSOR : FLURKA_PATH_SIMT;
+  ds.last_path = tcq ? FLURKA_PATH_TENSOR : (tc ? FLURKA_PATH_TENSOR_STAGE1 : FLURKA_PATH_SIMT);
   ds.last_launches = launches;
   ds.have_last = true;
   ds.last_problem = pr;

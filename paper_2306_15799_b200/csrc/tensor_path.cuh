@@ -12,6 +12,7 @@
 #include "k2_key_side.cuh"
 #include "k3_query_side.cuh"
 #include "k4_bwd_query_side.cuh"
+#include "k5_bwd_projections.cuh"
 
 namespace flurka {
 
@@ -91,6 +92,7 @@ inline bool encode_map(CachedMap* cm, CUtensorMapDataType dt, int esize, int ran
 struct TensorMaps {
   CachedMap E, F, K, V, kpvp, Q, W, W2, aT, O;
   CachedMap dO, abf;                            // backward of the query side
+  CachedMap bE, bF, bK, bV, split64, split128, gK, gV, gE, gF;   // backward of the down-projection
   CachedMap A3, Wk, Wv, Xq, Wq, Qp, kpvp2;      // the linear maps of the entry point with un-projected inputs
 };
 
@@ -103,6 +105,7 @@ struct TensorContext {
   bool k1p_attr = false;
   bool k0_attr = false;
   bool k0p_attr = false;
+  bool k5_attr = false;
   int sm_total() {
     if (!sms) {
       int dev = 0;
@@ -474,6 +477,57 @@ inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const voi
   if (grid > prm.total_tiles) grid = prm.total_tiles;
   k4_bwd_query_side<<<grid, kK4Threads, kK4SmemBytes, st>>>(tm.Q.map, tm.dO.map, tm.W.map, tm.abf.map, prm);
   e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
+
+// ---- backward of the down-projection: dK, dV, dE, dF from the fp32 dK', dV' (shared E, F) -------------
+// split: scratch for the two bf16 terms of dK', dV', [2][k][2][BH][d]
+inline int launch_k5(TensorContext& tc, const void* E, const void* F, const void* K, const void* V, const float* dkpvp,
+                     __nv_bfloat16* split, void* dK, void* dV, void* dE, void* dF, int BH, int H, int N, int d, int k,
+                     int* status, cudaStream_t st, int* cuda_err) {
+  TensorMaps& tm = tc.maps;
+  const unsigned long long hd = (unsigned long long)BH * d;
+  const unsigned long long dEF[2] = {(unsigned long long)N, (unsigned long long)k};
+  const unsigned bEF[2] = {64, 64}, bGE[2] = {64, 32};
+  const unsigned long long dKV[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
+                                     (unsigned long long)(H > 0 ? BH / H : BH)};
+  const unsigned bKV[3] = {64, 256, 1}, bGK[3] = {64, 32, 1};
+  const unsigned long long dS[3] = {2 * hd, (unsigned long long)k, 2};
+  const unsigned bS64[3] = {64, 64, 1}, bS128[3] = {64, 128, 1};
+  const CUtensorMapDataType bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  if (!encode_map(&tm.bE, bf, 2, 2, E, dEF, bEF) || !encode_map(&tm.bF, bf, 2, 2, F, dEF, bEF) ||
+      !encode_map(&tm.bK, bf, 2, 3, K, dKV, bKV) || !encode_map(&tm.bV, bf, 2, 3, V, dKV, bKV) ||
+      !encode_map(&tm.split64, bf, 2, 3, split, dS, bS64) || !encode_map(&tm.split128, bf, 2, 3, split, dS, bS128) ||
+      !encode_map(&tm.gK, bf, 2, 3, dK, dKV, bGK) || !encode_map(&tm.gV, bf, 2, 3, dV, dKV, bGK) ||
+      !encode_map(&tm.gE, bf, 2, 2, dE, dEF, bGE) || !encode_map(&tm.gF, bf, 2, 2, dF, dEF, bGE)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  if (!tc.k5_attr) {
+    cudaError_t e = cudaFuncSetAttribute(k5_bwd_projections<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kK5SmemBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k5_bwd_projections<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kK5SmemBytes);
+    if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+    tc.k5_attr = true;
+  }
+  {
+    const long long total = (long long)2 * BH * k * (d / 4);
+    int grid = (int)((total + 255) / 256);
+    if (grid > 148 * 8) grid = 148 * 8;
+    k5_split_rows<<<grid, 256, 0, st>>>(dkpvp, split, BH, k, d);
+  }
+  K5Params p;
+  p.N = N; p.k = k; p.d = d; p.BH = BH; p.H = H; p.status = status;
+  p.row_blocks = (N + 255) / 256;
+  p.col_groups = (int)((hd + 255) / 256);
+  k5_bwd_projections<0><<<2 * p.row_blocks * p.col_groups, kK5Threads, kK5SmemBytes, st>>>(
+      tm.bE.map, tm.bF.map, tm.split64.map, tm.gK.map, tm.gV.map, p);
+  p.row_blocks = (k + 255) / 256;
+  p.col_groups = (N + 255) / 256;
+  k5_bwd_projections<1><<<2 * p.row_blocks * p.col_groups, kK5Threads, kK5SmemBytes, st>>>(
+      tm.bK.map, tm.bV.map, tm.split128.map, tm.gE.map, tm.gF.map, p);
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
 }

@@ -92,6 +92,16 @@ def test_backward_tensor_path_matches_oracle(w):
     assert binding.flurka_last_path() == binding.PATH_TENSOR
 
 
+def test_backward_tensor_stage1_and_projection_gradients_only():
+    """Shapes whose query side has no tensor-core backward still take stage 1 and dK, dV, dE, dF from the
+    tensor-core kernels: RNN, d = 128 (two 64-column blocks per head), 64 features, ragged N and k = 64."""
+    for w, layout in ((Workload("bwd_tc1_rnn_d128", RNN, "bf16", 1, 3, 200, 128, 64, 0, 317), "bhnd"),
+                      (Workload("bwd_tc1_perf_m64", PERFORMER, "bf16", 2, 2, 328, 64, 192, 64, 318), "bnhd"),
+                      (Workload("bwd_tc1_perf_d128", PERFORMER, "bf16", 1, 2, 520, 128, 320, 128, 319), "bhnd")):
+        _check(w, layout=layout)
+        assert binding.flurka_last_path() == binding.PATH_TENSOR_STAGE1
+
+
 @pytest.mark.parametrize("limit", [1, 2])
 def test_backward_tensor_path_with_few_ctas(limit):
     """A CTA's tiles cross from one head to the next: its accumulators of da, db leave and start again."""
