@@ -864,8 +864,16 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
     rc = launch_simt_down_project<T>(pr, K, V, E, F, kpvp, st, launches);
     if (rc) return rc;
   }
-  rc = launch_simt_key_side<T, P>(pr, kpvp, W, weight, a32, nullptr, st, launches);
-  if (rc) return rc;
+  if (tc) {
+    // the key side on its tensor-core kernel, one CTA per (head, feature tile), with a in fp32 as well
+    rc = launch_k2(*tc, P, kpvp, W, weight, (__half*)(ws + L.aT16), nullptr, nullptr, pr.BH(), pr.d, pr.k, pr.p(),
+                   (int*)(ws + L.status), st, &cuda_err, a32);
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
+    ++*launches;
+  } else {
+    rc = launch_simt_key_side<T, P>(pr, kpvp, W, weight, a32, nullptr, st, launches);
+    if (rc) return rc;
+  }
   if (tc && tcq) {
     rc = launch_k4(*tc, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.p(),
                    (int*)(ws + L.status), st, &cuda_err);

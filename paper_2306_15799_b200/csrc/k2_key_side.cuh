@@ -36,6 +36,7 @@ struct K2Params {
   const float* kpvp;        // [2][BH][k][d] fp32
   float* weight;            // [BH][p]      b_i (PERFORMER) or z_i (RNN)
   __half* aT16;             // [BH][d][p]   a^T
+  float* a32;               // [BH][p][d]   a in fp32 as well (the backward pass wants it), or NULL
   int* status;
   int nsplit;               // CTAs per (head, feature tile) along the keys (1..4; PERFORMER only)
   float* part;              // nsplit > 1: [BH * ftiles][nsplit][d + 2][128]  max, sum, accumulator columns
@@ -408,6 +409,13 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
           const unsigned short h = __half_as_ushort(__float2half_rn(__uint_as_float(r[e]) * inv));
           asm volatile("st.shared.u16 [%0], %1;" ::"r"(col_addr + (uint32_t)(c + e) * 256u), "h"(h) : "memory");
         }
+        if (prm.a32 && feat < p) {
+          float4* arow = reinterpret_cast<float4*>(prm.a32 + ((size_t)head * p + feat) * d + c);
+#pragma unroll
+          for (int e = 0; e < 32; e += 4)
+            arow[e >> 2] = make_float4(__uint_as_float(r[e]) * inv, __uint_as_float(r[e + 1]) * inv,
+                                       __uint_as_float(r[e + 2]) * inv, __uint_as_float(r[e + 3]) * inv);
+        }
       }
     }
     __syncthreads();
@@ -485,6 +493,7 @@ k2_key_side(const __grid_constant__ CUtensorMap tmW, const K2Params prm) {
           for (int q = 0; q < 4; ++q)
             if (q < nsplit) acc = fmaf(scale[q], v[q][e], acc);
           if (f < p) dst[(size_t)(c0 + e) * p] = __float2half_rn(acc * inv);
+          if (prm.a32 && f < p) prm.a32[((size_t)head * p + f) * d + c0 + e] = acc * inv;
         }
       }
       if (tid == 0) prm.counters[unit] = 0;

@@ -355,7 +355,7 @@ inline size_t k2_part_floats(bool performer, int BH, int d, int k, int p) {
 // ---- stage 2: per-feature summaries a (fp16, transposed) and weights b / z from K', V' --------
 inline int launch_k2(TensorContext& tc, bool performer, const float* kpvp, const void* W, float* weight,
                      __half* aT16, float* part, int* counters, int BH, int d, int k, int p, int* status,
-                     cudaStream_t st, int* cuda_err) {
+                     cudaStream_t st, int* cuda_err, float* a32 = nullptr) {
   TensorMaps& tm = tc.maps;
   if (performer) {
     const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
@@ -371,6 +371,7 @@ inline int launch_k2(TensorContext& tc, bool performer, const float* kpvp, const
   prm.kpvp = kpvp;
   prm.weight = weight;
   prm.aT16 = aT16;
+  prm.a32 = a32;
   prm.status = status;
   prm.nsplit = (part && counters) ? k2_nsplit(tc.sm_total(), performer, BH, k, p) : 1;
   prm.part = part;
