@@ -13,8 +13,8 @@
 // in two sweeps over the features, 128 at a time: the first gives each row its log-sum-exp and
 // delta_n (running maximum, sum and P-weighted sum of g), the second forms P and c.  da and P^T delta
 // stay in TMEM over all the tiles a CTA has of one head and are added to global memory (atomics) when
-// the head changes; db comes from them there.  One thread per query row (4 warps), one MMA issuer, one
-// TMA thread; the phases of a tile follow one another (block barriers), nothing here waits for another CTA.
+// the head changes; db comes from them there.  Two threads per query row (8 warps; each takes 64 of the 128
+// features of a step), one MMA issuer, one TMA thread; the phases of a tile follow one another (block barriers), nothing here waits for another CTA.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -34,13 +34,13 @@ struct K4Params {
   int* status;
 };
 
-constexpr int kK4Threads = 192;
+constexpr int kK4Threads = 320;
 // shared memory: W 32 KB | a_hi 32 KB | a_lo 32 KB | 2 x (Q tile 16 KB, dO tile 16 KB) | P tile 32 KB |
 // ones 4 KB | bias 8 KB | delta 4 KB | barriers
 constexpr uint32_t kK4W = 0, kK4AHi = 32768, kK4ALo = 65536, kK4In = 98304, kK4P = 163840, kK4Ones = 196608,
                    kK4Bias = 200704, kK4Delta = 208896, kK4Bars = 212992;
 constexpr int kK4SmemBytes = 212992 + 256 + 1024;
-// TMEM columns: S 0..127 (c as bf16 pairs over 0..63), G 128..255, dQ 256..319, da 320..447 (two
+// TMEM columns: S 0..127 (c as bf16 pairs over 0..31 and 64..95), G 128..255, dQ 256..319, da 320..447 (two
 // 128-feature tiles of 64 columns), P^T delta 448..479 (two tiles of 16 columns)
 constexpr uint32_t kK4ColG = 128, kK4ColDQ = 256, kK4ColDA = 320, kK4ColDD = 448;
 
@@ -81,11 +81,13 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                  bar_mma2 = bars + 40, tmem_slot = bars + 48;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
+  __shared__ float stat[2][3][128];             // sweep 1: (maximum, sum, weighted sum) of the two threads of a row
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = prm.p, nh = p >> 7;
   const bool owner = warp >= 2;
   const int q4 = warp & 3, row = q4 * 32 + lane;
+  const int fh = (warp - 2) >> 2;              // which 64 of a step's 128 features this row owner takes
   const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
 
   const int t_begin = (int)(((long long)blockIdx.x * prm.total_tiles) / gridDim.x);
@@ -150,9 +152,10 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   // da, P^T delta of one head leave TMEM: thread = feature; db from the identity in the header
   auto flush = [&](int head) {
-    if (!owner) return;
+    if (!owner || fh >= nh) return;
     tcgen05_fence_after();
-    for (int hh = 0; hh < nh; ++hh) {
+    {
+      const int hh = fh;                     // the two groups of row owners take one feature tile each
       uint32_t dd[32];                       // columns 0..2 are this tile's P^T delta terms (the load is 32 wide)
       tmem_ld32(tmem + lane_off + kK4ColDD + hh * 16, dd);
       tmem_wait_ld(dd);
@@ -279,14 +282,14 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // ------------------------------------------------------------ sweep 1: log-sum-exp and delta of each row
     float mx = -INFINITY, den = 0.f, num = 0.f;     // mx in the base-2 domain
     for (int h = 0; h < nh && ok; ++h) {
-      if (tid == 32) issue_sg(h);
+      if (warp == 1 && elect_one()) issue_sg(h);
       bool mine = true;
       if (owner) {
         mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
         if (mine) {
           tcgen05_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < 128; c += 32) {
+          for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
             uint32_t rs[32], rg[32];
             tmem_ld32(tmem + lane_off + c, rs);
             tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
@@ -314,9 +317,20 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       ok = __syncthreads_and(mine) != 0;          // S, G have been read out
     }
     if (!ok) break;
+    // the two threads of a row put their parts together (both in the same order, so they agree to the bit)
+    if (owner) { stat[fh][0][row] = mx; stat[fh][1][row] = den; stat[fh][2][row] = num; }
+    __syncthreads();
+    if (owner) {
+      const float m0 = stat[0][0][row], m1 = stat[1][0][row];
+      const float nm = fmaxf(m0, m1);
+      const float s0 = k4_ex2(m0 - nm), s1 = k4_ex2(m1 - nm);
+      mx = nm;
+      den = fmaf(stat[0][1][row], s0, stat[1][1][row] * s1);
+      num = fmaf(stat[0][2][row], s0, stat[1][2][row] * s1);
+    }
     const float lse2 = mx + __log2f(den);
     const float delta = num / den;
-    if (owner) {
+    if (owner && fh == 0) {
       // delta_n as three bf16 terms: element (c, n) of the [16 x 128] operand at (n/8)*128 + c*16 + (n%8)*2 bytes
       __nv_bfloat16* dt = reinterpret_cast<__nv_bfloat16*>(base_ptr + kK4Delta) + (row >> 3) * 64 + (row & 7);
       float r = delta;
@@ -328,7 +342,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     // ------------------------------------------------------------ sweep 2: P, c and the three products they feed
     for (int h = 0; h < nh && ok; ++h) {
-      if (tid == 32) issue_sg(h);
+      if (warp == 1 && elect_one()) issue_sg(h);
       bool mine = true;
       if (owner) {
         mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
@@ -336,7 +350,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tcgen05_fence_after();
           const uint32_t prow = base + kK4P + (uint32_t)row * 128u;
 #pragma unroll 1
-          for (int c = 0; c < 128; c += 32) {
+          for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
             uint32_t rs[32], rg[32], cw[16];
             tmem_ld32(tmem + lane_off + c, rs);
             tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
@@ -358,7 +372,8 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
               asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + ((chunk ^ (uint32_t)(row & 7)) << 4)),
                            "r"(pw[0]), "r"(pw[1]), "r"(pw[2]), "r"(pw[3]) : "memory");
             }
-            tmem_st16(tmem + lane_off + (c >> 1), cw);
+            // over this thread's own (already read) part of S: features 0..63 at columns 0..31, 64..127 at 64..95
+            tmem_st16(tmem + lane_off + fh * 64 + ((c & 63) >> 1), cw);
           }
           tmem_wait_st();
           fence_proxy_async_smem();
@@ -368,12 +383,12 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       ph_mma ^= 1;
       ok = __syncthreads_and(mine) != 0;
       if (!ok) break;
-      if (tid == 32) {
+      if (warp == 1 && elect_one()) {
         tcgen05_fence_after();
         // dQ (+)= c W: 128 features = 8 steps of 16, A 8 columns per step, B 16 rows of W per step
         for (int j = 0; j < 2; ++j) {
           const uint64_t bw = make_sdesc(base + kK4W + h * 16384 + j * 8192, 8192, 1024, kSwizzle128);
-          mma_ts_x4(tmem + kK4ColDQ, tmem + j * 32, bw, 128, idescQ, (h > 0 || j > 0) ? 1u : 0u);
+          mma_ts_x4(tmem + kK4ColDQ, tmem + j * 64, bw, 128, idescQ, (h > 0 || j > 0) ? 1u : 0u);
         }
         // da_h (+)= P_h^T dO and (P^T delta)_h: 128 rows = 8 steps of 16 rows (2048 B of P and of dO, 256 B of delta)
         for (int j = 0; j < 2; ++j) {
@@ -393,27 +408,25 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (!ok) break;
     first_of_head = false;
 
-    // ------------------------------------------------------------ dQ rows
+    // ------------------------------------------------------------ dQ rows (32 columns per thread)
     if (owner) {
       tcgen05_fence_after();
-      uint32_t ra[32], rb[32];
-      tmem_ld32(tmem + lane_off + kK4ColDQ, ra);
-      tmem_ld32(tmem + lane_off + kK4ColDQ + 32, rb);
+      uint32_t ra[32];
+      tmem_ld32(tmem + lane_off + kK4ColDQ + fh * 32, ra);
       tmem_wait_ld(ra);
-      tmem_wait_ld(rb);
       tcgen05_fence_before();
       if (row0 + row < prm.N) {
         __nv_bfloat16* orow = prm.H > 0
             ? prm.dQ + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * 64
             : prm.dQ + ((size_t)head * prm.N + row0 + row) * 64;
+        orow += fh * 32;
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const uint32_t* src = g < 4 ? ra : rb;
+        for (int g = 0; g < 4; ++g) {
           uint4 v;
-          v.x = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 0]), __uint_as_float(src[(g & 3) * 8 + 1]));
-          v.y = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 2]), __uint_as_float(src[(g & 3) * 8 + 3]));
-          v.z = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 4]), __uint_as_float(src[(g & 3) * 8 + 5]));
-          v.w = k4_bf16x2(__uint_as_float(src[(g & 3) * 8 + 6]), __uint_as_float(src[(g & 3) * 8 + 7]));
+          v.x = k4_bf16x2(__uint_as_float(ra[g * 8 + 0]), __uint_as_float(ra[g * 8 + 1]));
+          v.y = k4_bf16x2(__uint_as_float(ra[g * 8 + 2]), __uint_as_float(ra[g * 8 + 3]));
+          v.z = k4_bf16x2(__uint_as_float(ra[g * 8 + 4]), __uint_as_float(ra[g * 8 + 5]));
+          v.w = k4_bf16x2(__uint_as_float(ra[g * 8 + 6]), __uint_as_float(ra[g * 8 + 7]));
           *reinterpret_cast<uint4*>(orow + g * 8) = v;
         }
       }
