@@ -314,6 +314,72 @@ def measure(w, args, binding, rank, world, local, with_e2e=True):
     return res
 
 
+def backward_work(w):
+    """Algorithmic FLOPs and compulsory bytes of one backward pass (all heads): the forward's stage 1 and
+    key side again, the query side's four products (S, dO a^T, dQ, da), the key side's four, and the four
+    products with E, F, K, V that give dK, dV, dE, dF; bytes: Q, K, V, dO in, dQ, dK, dV out, E, F in, dE, dF out."""
+    N, d, k, m, BH, s = w.N, w.d, w.k, w.m, w.B * w.H, w.elem_bytes
+    perf = w.variant == configs.PERFORMER
+    p = m if perf else d
+    flops = BH * (12 * N * k * d + (8 * N * p * d if perf else 0) + (12 * k * p * d if perf else 0))
+    byts = 7 * BH * N * d * s + 4 * k * N * s
+    return flops, byts
+
+
+def measure_backward(w, args, binding, rank, world):
+    """Times flurka_backward on workload `w` (device-resident inputs, CUDA events on the launch stream, the
+    same warm-up and L2 rules as the forward)."""
+    wr = rank_workload(w, rank)
+    host = host_inputs(wr)
+    dev = {n: (t.cuda() if t is not None else None) for n, t in host.items()}
+    gen = torch.Generator().manual_seed(wr.seed + 17)
+    dO = torch.randn(host["Q"].shape, generator=gen, dtype=torch.float32).to(host["Q"].dtype).cuda()
+    in_bytes = sum(t.numel() * t.element_size() for t in dev.values() if t is not None) + dO.numel() * dO.element_size()
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if in_bytes < 2 * L2_BYTES else None
+    stream = torch.cuda.Stream()
+    grads = None
+
+    def step():
+        return binding.flurka_backward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], dO, w.variant,
+                                       stream=stream, out=grads)
+
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        grads = step()
+        for _ in range(max(args.warmup, 3)):
+            step()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    with torch.cuda.stream(stream):
+        for i in range(args.steps):
+            if flush is not None:
+                flush.zero_()
+            starts[i].record(stream)
+            step()
+            stops[i].record(stream)
+    torch.cuda.synchronize()
+    step_ms = [a.elapsed_time(b) for a, b in zip(starts, stops)]
+    return {"step_ms": step_ms, "total_ms": sum(step_ms), "launches": binding.flurka_last_launches() * args.steps,
+            "path": {1: "simt", 2: "tensor", 3: "tensor stage 1 and projections, cuda-core query side"}.get(binding.flurka_last_path(), "?"),
+            "status": binding.flurka_last_status(), "flushed": flush is not None}
+
+
+def backward_block(w, rb, peaks, steps, world):
+    ms = rb["total_ms"] / steps
+    flops, byts = backward_work(w)
+    t_t, t_h = flops / (peaks["bf16_tflops"] * 1e12), byts / (peaks["hbm_gbs"] * 1e9)
+    return {"value": job_tokens_per_s(w, world, ms), "unit": UNIT, "ms_per_step": ms,
+            "step_ms_min": min(rb["step_ms"]), "step_ms_median": statistics.median(rb["step_ms"]),
+            "path": rb["path"], "gpu_launches": rb["launches"], "device_status": rb["status"],
+            "path_roofline": {"flops": flops, "bytes": byts, "t_tensor_us": t_t * 1e6, "t_hbm_us": t_h * 1e6,
+                              "frac": max(t_t, t_h) / (ms * 1e-3),
+                              "peak_source": "of " + peaks["source"] + " (burst GEMM figure)"}}
+
+
 def stage_work(w):
     """Algorithmic FLOPs, bytes and exponentials of the three stages (all heads), and their names."""
     N, d, k, m, BH, s = w.N, w.d, w.k, w.m, w.B * w.H, w.elem_bytes
@@ -386,6 +452,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-also", action="store_true", help="default run: skip the second target configuration (c4)")
+    ap.add_argument("--no-backward", action="store_true", help="skip the backward-pass block under `also`")
     ap.add_argument("--heads", default="", help="B,H override: a smaller batch of the same workload (profiling)")
     ap.add_argument("--no-load", action="store_true", help="skip the sustained-load phase before timing (profiling)")
     ap.add_argument("--layout", default="bhnd", choices=["bhnd", "bnhd"],
@@ -433,6 +500,12 @@ def main():
         r4["total_ms"] = max_over_ranks([r4["total_ms"]], world, device="cuda")[0]
         also = (w4, r4)
 
+    bwd = None
+    if not args.no_backward and not is_fused(w):
+        # the backward pass of the same workload (gradients of Q, K, V, E, F), timed the same way
+        bwd = measure_backward(w, args, binding, rank, world)
+        bwd["total_ms"] = max_over_ranks([bwd["total_ms"]], world, device="cuda")[0]
+
     if rank == 0:
         peaks = measured_peaks()
         exp_rate = binding.flurka_measure_ex2_rate()          # Gexp/s of a bare ex2.approx loop on this GPU, now
@@ -475,6 +548,8 @@ def main():
                 "clocks": {"sm_mhz": r4["clocks"]["sm_mhz"], "sm_max_mhz": r4["clocks"]["sm_max_mhz"],
                            "reasons": r4["clocks"]["reasons"]},
                 "gpu_launches": r4["launches"], "roofline": rf4, "path_roofline": pr4, "device_status": r4["status"]}}
+        if bwd is not None:
+            line.setdefault("also", {})["backward_" + w.name] = backward_block(w, bwd, peaks, args.steps, world)
         if not args.no_cpu_baseline and world == 1:
             import oracle
             oracle.build()

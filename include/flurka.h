@@ -174,8 +174,14 @@ int flurka_forward_finish(const void* Q, const void* W, int variant, int B, int 
  * All buffers are DEVICE buffers of the call's element type; variant word, layouts, limits, alignment,
  * stream and workspace rules as for flurka_forward (flurka_backward_workspace_bytes says how much scratch).
  * The forward's key-side summaries are recomputed inside the call, so nothing has to be kept from the
- * forward pass.  Runs on CUDA cores with fp32 arithmetic for every shape; no output may overlap an input
- * or another output.
+ * forward pass.  No output may overlap an input or another output.
+ * Kernels: where flurka_forward's tensor-core path takes the shape (bf16, the rules below) the two
+ * down-projections, the key-side summaries and, with E, F shared by the heads, the gradients dK, dV, dE, dF
+ * (products with E, F, K, V: dK', dV' enter as two bf16 terms) run on tcgen05 kernels; for PERFORMER with
+ * d = 64 and m = 128 or 256 so does the query side (dQ and the gradients of the key-side summaries).
+ * flurka_last_path() then reports FLURKA_PATH_TENSOR (query side included) or FLURKA_PATH_TENSOR_STAGE1.
+ * Everything else, and every shape under FLURKA_PATH_SIMT, runs on CUDA cores with fp32 arithmetic;
+ * FLURKA_PATH_TENSOR forced on a shape without a tensor-core query side returns FLURKA_ERR_SHAPE.
  */
 int flurka_backward(const void* Q, const void* K, const void* V, const void* E, const void* F, const void* W,
                     const void* dO, int variant, int B, int H, int N, int d, int k, int m, void* dQ, void* dK,
@@ -203,7 +209,7 @@ int flurka_set_cta_limit(int max_ctas);
  * shared by the heads) or always as single CTAs.  Returns the old setting. */
 int flurka_set_stage1_pairs(int on);
 
-/* The path the most recent successful flurka_forward took (never FLURKA_PATH_AUTO). */
+/* The path the most recent successful flurka_forward (or flurka_backward) took (never FLURKA_PATH_AUTO). */
 int flurka_last_path(void);
 
 /* Number of kernels the most recent successful flurka_forward launched. */

@@ -283,11 +283,14 @@ def flurka_forward_finish(Q, W, variant, k, out=None, stream=None, layout="bhnd"
     return out
 
 
-def flurka_backward(Q, K, V, E, F, W, dO, variant, stream=None, layout="bhnd"):
+def flurka_backward(Q, K, V, E, F, W, dO, variant, stream=None, layout="bhnd", out=None):
     """Gradients of the forward's output with respect to Q, K, V, E, F, given dO (device tensors).
-    Returns (dQ, dK, dV, dE, dF), shaped and typed like the inputs."""
+    Returns (dQ, dK, dV, dE, dF), shaped and typed like the inputs (`out`: five such tensors to write into)."""
     B, H, N, d, k, m = _check(Q, K, V, E, F, W, variant, dO, "cuda", layout)
-    grads = [torch.empty_like(t) for t in (Q, K, V, E, F)]
+    grads = list(out) if out is not None else [torch.empty_like(t) for t in (Q, K, V, E, F)]
+    for g, t in zip(grads, (Q, K, V, E, F)):
+        if g.shape != t.shape or g.dtype != t.dtype or not g.is_cuda or not g.is_contiguous():
+            raise ValueError("flurka_backward: `out` must hold five contiguous device tensors shaped like Q, K, V, E, F")
     rc = load().flurka_backward(
         Q.data_ptr(), K.data_ptr(), V.data_ptr(), E.data_ptr(), F.data_ptr(), W.data_ptr() if W is not None else None,
         dO.data_ptr(), _variant_word(variant, Q.dtype, layout, E.dim() == 3), B, H, N, d, k, m,
