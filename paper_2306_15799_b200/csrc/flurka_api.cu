@@ -894,7 +894,7 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
     const size_t smem = (size_t)3 * 32 * (pr.d + 1) * 4;
     if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
       return cuda_fail(e);
-    dim3 grid((pr.k + 7) / 8, pr.BH());
+    dim3 grid((pr.k + 8 * kBwdKeysPerWarp - 1) / (8 * kBwdKeysPerWarp), pr.BH());
     fn<<<grid, 256, smem, st>>>(kpvp, (const T*)W, weight, a32, da, db, dkpvp, pr.BH(), pr.d, pr.k, pr.p());
     ++*launches;
   }

@@ -24,9 +24,18 @@ struct K5Params {
   int* status;
 };
 
-constexpr int kK5Stages = 3;
-constexpr int kK5StageBytes = 65536;                  // 32 KB of A + 32 KB of B
-constexpr int kK5SmemBytes = kK5Stages * kK5StageBytes + 1024 + 256;
+// kMode 0 has a short contraction (2 k / 64 chunks) and a long epilogue: 128 x 256 outputs per CTA and two
+// 48 KB stages, so that two CTAs share an SM and one's epilogue runs under the other's MMAs; kMode 1 has a
+// long contraction: 256 x 256 outputs and three 64 KB stages
+template <int kMode> struct K5Shape {
+  static constexpr int kRows = kMode == 0 ? 128 : 256;
+  static constexpr int kStages = kMode == 0 ? 2 : 3;
+  static constexpr int kABytes = kRows * 128;                       // 64 contraction elements per row
+  static constexpr int kStageBytes = kABytes + 32768;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+  static constexpr int kTmemCols = kRows * 2;
+  static constexpr int kCtasPerSm = kMode == 0 ? 2 : 1;
+};
 constexpr int kK5Threads = 192;
 
 // dK', dV' [2][BH][k][d] fp32 -> split [2][k][2][BH][d] bf16 (hi terms of all heads, then lo terms)
@@ -56,13 +65,15 @@ __global__ void k5_split_rows(const float* __restrict__ src, __nv_bfloat16* __re
 // tmS: the split matrix (kMode 0: boxes of 64 x 64; kMode 1: boxes of 64 x 128 rows);
 // tmO0/tmO1: dK, dV (boxes of 64 c x 32 n) or dE, dF (boxes of 64 n x 32 k)
 template <int kMode>
-__global__ void __launch_bounds__(kK5Threads, 1)
+__global__ void __launch_bounds__(kK5Threads, K5Shape<kMode>::kCtasPerSm)
 k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_constant__ CUtensorMap tmP1,
                    const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmO0,
                    const __grid_constant__ CUtensorMap tmO1, const K5Params p) {
   using namespace tc;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  constexpr int kK5Stages = K5Shape<kMode>::kStages, kK5StageBytes = K5Shape<kMode>::kStageBytes;
+  constexpr int kRows = K5Shape<kMode>::kRows, kABytes = K5Shape<kMode>::kABytes;
   const uint32_t bar_base = smem_base + kK5Stages * kK5StageBytes;
   const uint32_t bar_full = bar_base;                 // [3]
   const uint32_t bar_empty = bar_base + 24;           // [3]
@@ -78,7 +89,7 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
   const int z = idx;                                        // 0: keys / E, 1: values / F
   const int M = kMode == 0 ? p.N : p.k;                     // output rows
   const int NC = kMode == 0 ? p.BH * p.d : p.N;             // output columns
-  const int rows = min(256, M - rb * 256);
+  const int rows = min(kRows, M - rb * kRows);
   const int mt = (rows + 127) >> 7;
   const int ncols = kMode == 0 ? min(256, NC - cg * 256) : 256;   // kMode 1: columns past N are zero and clipped
   const int hd = p.BH * p.d;
@@ -97,7 +108,7 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 512);
+    tmem_alloc(tmem_slot, K5Shape<kMode>::kTmemCols);
     tmem_relinquish();
   }
   tcgen05_fence_before();
@@ -124,7 +135,7 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
         if (it >= kK5Stages) ok = mbar_wait(bar_empty + 8 * st, ((it / kK5Stages) - 1) & 1, p.status, &abort_flag);
         if (!ok) break;
         const uint32_t a_dst = smem_base + st * kK5StageBytes;
-        const uint32_t b_dst = a_dst + 32768;
+        const uint32_t b_dst = a_dst + kABytes;
         const uint32_t bar = bar_full + 8 * st;
         const int t = it / per_term, c = it % per_term;
         mbar_arrive_expect_tx(bar, tx_bytes);
@@ -132,12 +143,12 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
           // A: rows n of E^T as two 64-row slabs per M-tile (n contiguous: MN-major); B: 64 rows of the split matrix
           for (int m = 0; m < mt; ++m)
             for (int s = 0; s < 2; ++s)
-              tma_load_2d(a_dst + m * 16384 + s * 8192, tmP, bar, rb * 256 + m * 128 + s * 64, c << 6);
+              tma_load_2d(a_dst + m * 16384 + s * 8192, tmP, bar, rb * kRows + m * 128 + s * 64, c << 6);
           for (int b = 0; b < (ncols >> 6); ++b)
             tma_load_3d(b_dst + b * 8192, &tmS, bar, t * hd + cg * 256 + b * 64, c << 6, z);
         } else {
           // A: 128 rows of the split matrix per M-tile (K-major); B: 256 rows n of one head's K or V (K-major)
-          for (int m = 0; m < mt; ++m) tma_load_3d(a_dst + m * 16384, &tmS, bar, t * hd + (c << 6), rb * 256 + m * 128, z);
+          for (int m = 0; m < mt; ++m) tma_load_3d(a_dst + m * 16384, &tmS, bar, t * hd + (c << 6), rb * kRows + m * 128, z);
           const int col = c << 6, head = col / p.d, c0 = col % p.d;
           if (p.H > 0) tma_load_3d(b_dst, tmP, bar, (head % p.H) * p.d + c0, cg * 256, head / p.H);
           else tma_load_3d(b_dst, tmP, bar, c0, cg * 256, head);
@@ -160,7 +171,7 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
         if (!ok) break;
         tcgen05_fence_after();
         const uint32_t a_base = smem_base + st * kK5StageBytes;
-        const uint32_t b_base = a_base + 32768;
+        const uint32_t b_base = a_base + kABytes;
         for (int m = 0; m < mt; ++m) {
           if (kMode == 0) {
             // MN-major operands: 64-wide slabs 8192 B apart, 8-row (contraction) groups 1024 B apart, 16 rows per step
@@ -184,9 +195,9 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
     bool ok = mbar_wait(bar_accum, 0, p.status, &abort_flag);
     if (ok) {
       tcgen05_fence_after();
-      const uint32_t stage_buf = smem_base + (warp - 2) * 32768;   // the ring is drained
+      const uint32_t stage_buf = smem_base + (warp - 2) * 16384;   // the ring is drained; 4 slabs of 4 KB per warp
       for (int m = 0; m < mt; ++m) {
-        const int row0 = rb * 256 + m * 128 + q * 32;
+        const int row0 = rb * kRows + m * 128 + q * 32;
         const int ncc = ncols >> 6;
         for (int cc = 0; cc < ncc; ++cc) {
           uint32_t ra[32], rb2[32];
@@ -235,7 +246,7 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 512);
+  if (warp == 1) tmem_dealloc(tmem, K5Shape<kMode>::kTmemCols);
 }
 
 }  // namespace flurka

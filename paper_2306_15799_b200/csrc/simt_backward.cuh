@@ -213,41 +213,56 @@ simt_bwd_query_side(const T* __restrict__ Q, const T* __restrict__ W, const T* _
 }
 
 // ---------------------------------------------------------------------------------------------
-// Key side.  grid = (ceil(k/8), B*H); block = 256: one warp per projected key j.  Features in chunks
-// of 32 (lane = feature for the scalar parts, lane = column for the sums over features).
+// Key side.  grid = (ceil(k/32), B*H); block = 256: a warp owns four projected keys, so that every
+// chunk of W, a, da a block brings into shared memory (32 features at a time) serves 32 keys and every
+// value read from it in the inner loops serves four.  Lane = feature for the scalar parts (A_ij, g_ij),
+// lane = column for the sums over features; A and dL of a chunk go through shared memory so that the
+// column loop reads the four keys' values of a feature with one 16-byte broadcast load each.
 // Inputs: K', V' (KpVp), W, a, b (weight), da, db.  Outputs: dKpVp [2][B*H][k][d] fp32 (dK' then dV').
 // Dynamic shared memory: 3 * 32 * (d+1) floats (W, a, da chunks).
 // ---------------------------------------------------------------------------------------------
+constexpr int kBwdKeysPerWarp = 4;
 template <typename T, bool kPerformer>
 __global__ void __launch_bounds__(256)
 simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const float* __restrict__ weight,
                   const float* __restrict__ a32, const float* __restrict__ da, const float* __restrict__ db,
                   float* __restrict__ dKpVp, int BH, int d, int k, int p) {
+  constexpr int KW = kBwdKeysPerWarp;
   extern __shared__ float smem[];
   float* Ws = smem;                          // [32][d+1]
   float* As = Ws + 32 * (d + 1);             // [32][d+1]
   float* Ds = As + 32 * (d + 1);             // [32][d+1]  da chunk
-  __shared__ float ks[8][128], vs[8][128];
+  __shared__ float ks[8 * KW][128], vs[8 * KW][128];
+  __shared__ __align__(16) float sA[8][32][KW], sdL[8][32][KW];
   __shared__ float bs[32], dbs[32];
 
   const int bh = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int j = blockIdx.x * 8 + warp;
-  const bool key_live = j < k;
+  const int j0 = (blockIdx.x * 8 + warp) * KW;                 // this warp's keys j0 .. j0 + KW - 1
   const float* __restrict__ Kp = KpVp + (size_t)bh * k * d;
   const float* __restrict__ Vp = KpVp + ((size_t)BH + bh) * (size_t)k * d;
-  float half_sq = 0.f;
-  for (int c = lane; c < d; c += 32) {
-    const float x = key_live ? Kp[(size_t)j * d + c] : 0.f;
-    ks[warp][c] = x;
-    vs[warp][c] = key_live ? Vp[(size_t)j * d + c] : 0.f;
-    half_sq = fmaf(x, x, half_sq);
-  }
+  float half_sq[KW];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) half_sq += __shfl_xor_sync(0xffffffffu, half_sq, o);
-  half_sq *= 0.5f;
-  float dk[4] = {0.f, 0.f, 0.f, 0.f}, dv[4] = {0.f, 0.f, 0.f, 0.f};
-  float dl_sum = 0.f;
+  for (int q = 0; q < KW; ++q) {
+    const bool key_live = j0 + q < k;
+    float hs = 0.f;
+    for (int c = lane; c < d; c += 32) {
+      const float x = key_live ? Kp[(size_t)(j0 + q) * d + c] : 0.f;
+      ks[warp * KW + q][c] = x;
+      vs[warp * KW + q][c] = key_live ? Vp[(size_t)(j0 + q) * d + c] : 0.f;
+      hs = fmaf(x, x, hs);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
+    half_sq[q] = 0.5f * hs;
+  }
+  float dk[KW][4], dv[KW][4], dl_sum[KW];
+#pragma unroll
+  for (int q = 0; q < KW; ++q) {
+    dl_sum[q] = 0.f;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) dk[q][b] = dv[q][b] = 0.f;
+  }
   for (int i0 = 0; i0 < p; i0 += 32) {
     __syncthreads();
     for (int idx = threadIdx.x; idx < 32 * d; idx += 256) {
@@ -264,49 +279,72 @@ simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const
       dbs[threadIdx.x] = in ? db[(size_t)bh * p + i0 + threadIdx.x] : 0.f;
     }
     __syncthreads();
-    const bool live = key_live && (i0 + lane) < p;
-    // A_ij and g_ij for feature i = i0 + lane
-    float A = 0.f, g = 0.f;
-    if (live) {
-      float e1 = 0.f;
-      for (int c = 0; c < d; ++c) e1 = fmaf(Ds[lane * (d + 1) + c], vs[warp][c] - As[lane * (d + 1) + c], e1);
-      g = e1 + dbs[lane];
-      if (kPerformer) {
-        float wk = 0.f;
-        for (int c = 0; c < d; ++c) wk = fmaf(Ws[lane * (d + 1) + c], ks[warp][c], wk);
-        A = expf(wk - half_sq - bs[lane]);               // b_i = log sum_j exp(L_ji): A <= 1
-      } else {
-        A = elu1(ks[warp][i0 + lane]) / bs[lane];        // weight holds z_i for RNN
+    const bool feat_live = (i0 + lane) < p;
+    // A_ij and g_ij for feature i = i0 + lane and the warp's four keys
+    float e1[KW], wk[KW];
+#pragma unroll
+    for (int q = 0; q < KW; ++q) e1[q] = wk[q] = 0.f;
+    for (int c = 0; c < d; ++c) {
+      const float dsv = Ds[lane * (d + 1) + c], asv = As[lane * (d + 1) + c];
+      const float wsv = kPerformer ? Ws[lane * (d + 1) + c] : 0.f;
+#pragma unroll
+      for (int q = 0; q < KW; ++q) {
+        e1[q] = fmaf(dsv, vs[warp * KW + q][c] - asv, e1[q]);
+        if (kPerformer) wk[q] = fmaf(wsv, ks[warp * KW + q][c], wk[q]);
       }
     }
-    const float dL = A * g;
-    dl_sum += dL;
-    if (!kPerformer && live) {
-      const float x = ks[warp][i0 + lane];
-      dKpVp[((size_t)bh * k + j) * d + i0 + lane] = dL * elu1_slope(x) / elu1(x);
+#pragma unroll
+    for (int q = 0; q < KW; ++q) {
+      const bool live = feat_live && (j0 + q < k);
+      float A = 0.f, g = 0.f;
+      if (live) {
+        g = e1[q] + dbs[lane];
+        if (kPerformer) A = expf(wk[q] - half_sq[q] - bs[lane]);     // b_i = log sum_j exp(L_ji): A <= 1
+        else A = elu1(ks[warp * KW + q][i0 + lane]) / bs[lane];      // weight holds z_i for RNN
+      }
+      const float dL = A * g;
+      dl_sum[q] += dL;
+      if (!kPerformer && live) {
+        const float x = ks[warp * KW + q][i0 + lane];
+        dKpVp[((size_t)bh * k + j0 + q) * d + i0 + lane] = dL * elu1_slope(x) / elu1(x);
+      }
+      sA[warp][lane][q] = A;
+      sdL[warp][lane][q] = dL;
     }
+    __syncwarp();
     for (int ii = 0; ii < 32; ++ii) {
-      const float Ai = __shfl_sync(0xffffffffu, A, ii);
-      const float dLi = __shfl_sync(0xffffffffu, dL, ii);
+      const float4 A4 = *reinterpret_cast<const float4*>(&sA[warp][ii][0]);
+      const float4 L4 = *reinterpret_cast<const float4*>(&sdL[warp][ii][0]);
+      const float Aq[KW] = {A4.x, A4.y, A4.z, A4.w}, Lq[KW] = {L4.x, L4.y, L4.z, L4.w};
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         const int c = lane + 32 * b;
         if (c < d) {
-          dv[b] = fmaf(Ai, Ds[ii * (d + 1) + c], dv[b]);
-          if (kPerformer) dk[b] = fmaf(dLi, Ws[ii * (d + 1) + c], dk[b]);
+          const float dsv = Ds[ii * (d + 1) + c];
+          const float wsv = kPerformer ? Ws[ii * (d + 1) + c] : 0.f;
+#pragma unroll
+          for (int q = 0; q < KW; ++q) {
+            dv[q][b] = fmaf(Aq[q], dsv, dv[q][b]);
+            if (kPerformer) dk[q][b] = fmaf(Lq[q], wsv, dk[q][b]);
+          }
         }
       }
     }
+    __syncwarp();
   }
-  if (!key_live) return;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) dl_sum += __shfl_xor_sync(0xffffffffu, dl_sum, o);
+  for (int q = 0; q < KW; ++q) {
+    if (j0 + q >= k) continue;
+    float ds = dl_sum[q];
 #pragma unroll
-  for (int b = 0; b < 4; ++b) {
-    const int c = lane + 32 * b;
-    if (c < d) {
-      if (kPerformer) dKpVp[((size_t)bh * k + j) * d + c] = dk[b] - ks[warp][c] * dl_sum;
-      dKpVp[(((size_t)BH + bh) * k + j) * d + c] = dv[b];
+    for (int o = 16; o > 0; o >>= 1) ds += __shfl_xor_sync(0xffffffffu, ds, o);
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int c = lane + 32 * b;
+      if (c < d) {
+        if (kPerformer) dKpVp[((size_t)bh * k + j0 + q) * d + c] = dk[q][b] - ks[warp * KW + q][c] * ds;
+        dKpVp[(((size_t)BH + bh) * k + j0 + q) * d + c] = dv[q][b];
+      }
     }
   }
 }

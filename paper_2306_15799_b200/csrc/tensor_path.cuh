@@ -506,9 +506,10 @@ inline int launch_k5(TensorContext& tc, const void* E, const void* F, const void
     return -6;
   }
   if (!tc.k5_attr) {
-    cudaError_t e = cudaFuncSetAttribute(k5_bwd_projections<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kK5SmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(k5_bwd_projections<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         K5Shape<0>::kSmemBytes);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(k5_bwd_projections<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kK5SmemBytes);
+      e = cudaFuncSetAttribute(k5_bwd_projections<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, K5Shape<1>::kSmemBytes);
     if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
     tc.k5_attr = true;
   }
@@ -520,13 +521,13 @@ inline int launch_k5(TensorContext& tc, const void* E, const void* F, const void
   }
   K5Params p;
   p.N = N; p.k = k; p.d = d; p.BH = BH; p.H = H; p.status = status;
-  p.row_blocks = (N + 255) / 256;
+  p.row_blocks = (N + K5Shape<0>::kRows - 1) / K5Shape<0>::kRows;
   p.col_groups = (int)((hd + 255) / 256);
-  k5_bwd_projections<0><<<2 * p.row_blocks * p.col_groups, kK5Threads, kK5SmemBytes, st>>>(
+  k5_bwd_projections<0><<<2 * p.row_blocks * p.col_groups, kK5Threads, K5Shape<0>::kSmemBytes, st>>>(
       tm.bE.map, tm.bF.map, tm.split64.map, tm.gK.map, tm.gV.map, p);
   p.row_blocks = (k + 255) / 256;
   p.col_groups = (N + 255) / 256;
-  k5_bwd_projections<1><<<2 * p.row_blocks * p.col_groups, kK5Threads, kK5SmemBytes, st>>>(
+  k5_bwd_projections<1><<<2 * p.row_blocks * p.col_groups, kK5Threads, K5Shape<1>::kSmemBytes, st>>>(
       tm.bK.map, tm.bV.map, tm.split128.map, tm.gE.map, tm.gF.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
