@@ -14,7 +14,8 @@
 // delta_n (running maximum, sum and P-weighted sum of g), the second forms P and c.  da and P^T delta
 // stay in TMEM over all the tiles a CTA has of one head and are added to global memory (atomics) when
 // the head changes; db comes from them there.  Two threads per query row (8 warps; each takes 64 of the 128
-// features of a step), one MMA issuer, one TMA thread; the phases of a tile follow one another (block barriers), nothing here waits for another CTA.
+// features of a step), one MMA issuer, one TMA thread; the phases of a tile follow one another (block
+// barriers), nothing here waits for another CTA.
 #pragma once
 
 #include <cuda_bf16.h>

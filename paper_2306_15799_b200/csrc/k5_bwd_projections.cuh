@@ -7,9 +7,9 @@
 // out as one matrix per projection, `split` = [2][k][2 BH d] (term-major along the row), which is the
 // K-major A operand of kMode 1 and, seen through a tensor map with 64-row boxes, the MN-major B operand of
 // kMode 0.  E, F are read as they lie ([k][N]: an MN-major A operand for kMode 0), K, V as they lie
-// ([.., N, d]: a K-major B operand for kMode 1).  One CTA owns 256 x 256 outputs and the whole
-// contraction: a three-stage TMA ring, one thread issuing tcgen05.mma (M = 128, N = 256, K = 16) into
-// TMEM, four warps storing bf16 through swizzled slabs and TMA stores of whole lines.
+// ([.., N, d]: a K-major B operand for kMode 1).  One CTA owns a tile of outputs (K5Shape below) and the
+// whole contraction: a TMA ring, one thread issuing tcgen05.mma (M = 128, N = 256, K = 16) into TMEM, four
+// warps storing bf16 through swizzled slabs and TMA stores of whole lines.
 #pragma once
 
 #include <cuda_bf16.h>
