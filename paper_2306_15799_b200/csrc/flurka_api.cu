@@ -813,9 +813,10 @@ struct BackwardLayout {
   size_t da, dab_bytes, db, dkpvp, abf, split, total;
 };
 
-// the query side of the backward has a tensor-core kernel for PERFORMER with d = 64 and 128 or 256 features
+// the query side of the backward has a tensor-core kernel for PERFORMER with d = 64 (any feature count the
+// forward's tensor path takes: 64, 128, 192, 256)
 bool backward_tensor_ok(const Problem& pr) {
-  return tensor_path_ok(pr) && pr.kernel == FLURKA_PERFORMER && pr.d == 64 && (pr.m == 128 || pr.m == 256);
+  return tensor_path_ok(pr) && pr.kernel == FLURKA_PERFORMER && pr.d == 64;
 }
 
 BackwardLayout make_backward_layout(const Problem& pr) {

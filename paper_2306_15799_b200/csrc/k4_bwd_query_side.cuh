@@ -1,4 +1,5 @@
-// Backward of the query side on tensor cores (PERFORMER, bf16, d = 64, p = 128 or 256 features).
+// Backward of the query side on tensor cores (PERFORMER, bf16, d = 64, p = 64, 128, 192 or 256 features;
+// a last tile of 64 features is padded to 128 with weights that are exactly zero).
 //
 // The forward's query side (arxiv 2306.15799, Eq. (2) with the normalised weights of Appendix D) is
 //     O_n = sum_i P_ni a_i,    P_n. = softmax_i(l_n.),    l_ni = w_i . q_n + b_i.
@@ -85,7 +86,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   __shared__ float stat[2][3][128];             // sweep 1: (maximum, sum, weighted sum) of the two threads of a row
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int p = prm.p, nh = p >> 7;
+  const int p = prm.p, nh = (p + 127) >> 7;   // feature tiles of 128; rows of W, a past p are zero-filled by TMA
   const bool owner = warp >= 2;
   const int q4 = warp & 3, row = q4 * 32 + lane;
   const int fh = (warp - 2) >> 2;              // which 64 of a step's 128 features this row owner takes
@@ -161,8 +162,9 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       tmem_ld32(tmem + lane_off + kK4ColDD + hh * 16, dd);
       tmem_wait_ld(dd);
       const int feat = hh * 128 + row;
-      const float* arow = prm.a32 + ((size_t)head * p + feat) * 64;
-      float* darow = prm.da + ((size_t)head * p + feat) * 64;
+      const bool live = feat < p;            // (the TMEM loads below are warp-wide: every lane takes them)
+      const float* arow = prm.a32 + ((size_t)head * p + (live ? feat : 0)) * 64;
+      float* darow = prm.da + ((size_t)head * p + (live ? feat : 0)) * 64;
       float dot = 0.f;
 #pragma unroll 1
       for (int c = 0; c < 64; c += 32) {
@@ -178,10 +180,11 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           dot = fmaf(av.w, __uint_as_float(r[e + 3]), dot);
         }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) atomicAdd(darow + c + e, __uint_as_float(r[e]));
+        for (int e = 0; e < 32; ++e)
+          if (live) atomicAdd(darow + c + e, __uint_as_float(r[e]));
       }
       const float pd = __uint_as_float(dd[0]) + __uint_as_float(dd[1]) + __uint_as_float(dd[2]);
-      atomicAdd(prm.db + (size_t)head * p + feat, dot - pd);
+      if (live) atomicAdd(prm.db + (size_t)head * p + feat, dot - pd);
     }
     tcgen05_fence_before();
   };
@@ -201,7 +204,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     prefetch_tmap(&tmDO);
     prefetch_tmap(&tmW);
     prefetch_tmap(&tmA);
-    mbar_arrive_expect_tx(bar_w, (uint32_t)p * 128u);
+    mbar_arrive_expect_tx(bar_w, (uint32_t)nh * 16384u);
     tma_load_2d(base + kK4W, &tmW, bar_w, 0, 0);
     load_tile(0);
   }
@@ -223,7 +226,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if (head_prev >= 0) flush(head_prev);
       __syncthreads();
       if (tid == 0) {
-        mbar_arrive_expect_tx(bar_head, 2u * (uint32_t)p * 128u);
+        mbar_arrive_expect_tx(bar_head, 2u * (uint32_t)nh * 16384u);
         tma_load_3d(base + kK4AHi, &tmA, bar_head, 0, 0, head * 2);
         tma_load_3d(base + kK4ALo, &tmA, bar_head, 0, 0, head * 2 + 1);
       }
@@ -287,7 +290,8 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       bool mine = true;
       if (owner) {
         mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
-        if (mine) {
+        // (this thread's 64 features of the step lie past p: padding, weight zero; the same for the whole warp)
+        if (mine && h * 128 + fh * 64 < p) {
           tcgen05_fence_after();
 #pragma unroll 1
           for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
@@ -358,14 +362,16 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             tmem_wait_ld(rs);
             tmem_wait_ld(rg);
             const uint32_t slab = prow + (uint32_t)(c >> 6) * 16384u;
+            // features past p (padding of the last tile): P and c exactly zero
+            const float keep = (h * 128 + fh * 64 < p) ? 1.f : 0.f;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               uint32_t pw[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const int j = 8 * g + 2 * e;
-                const float p0 = k4_ex2(fmaf(__uint_as_float(rs[j]), kLog2e, -lse2));
-                const float p1 = k4_ex2(fmaf(__uint_as_float(rs[j + 1]), kLog2e, -lse2));
+                const float p0 = keep * k4_ex2(fmaf(__uint_as_float(rs[j]), kLog2e, -lse2));
+                const float p1 = keep * k4_ex2(fmaf(__uint_as_float(rs[j + 1]), kLog2e, -lse2));
                 pw[e] = k4_bf16x2(p0, p1);
                 cw[4 * g + e] = k4_bf16x2(p0 * (__uint_as_float(rg[j]) - delta), p1 * (__uint_as_float(rg[j + 1]) - delta));
               }

@@ -438,7 +438,7 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
   return 0;
 }
 
-// ---- backward of the query side (PERFORMER, d = 64, p = 128 or 256): dQ, and da, db added to ---------
+// ---- backward of the query side (PERFORMER, d = 64, p = 64, 128, 192 or 256): dQ, and da, db added to --
 // abf: scratch for the two bf16 terms of a, [BH][2][p][64]
 inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const void* W, const float* a32,
                      const float* weight, __nv_bfloat16* abf, void* dQ, float* da, float* db, int BH, int H, int N,
@@ -449,9 +449,10 @@ inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const voi
                                      (unsigned long long)(H > 0 ? BH / H : BH)};
   const unsigned bQ[3] = {64, 128, 1};
   const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
-  const unsigned bW[2] = {64, (unsigned)p};
+  const unsigned prows = (unsigned)((p + 127) / 128) * 128;      // whole 128-feature tiles; rows past p read as zero
+  const unsigned bW[2] = {64, prows};
   const unsigned long long dA[3] = {(unsigned long long)d, (unsigned long long)p, (unsigned long long)BH * 2};
-  const unsigned bA[3] = {64, (unsigned)p, 1};
+  const unsigned bA[3] = {64, prows, 1};
   if (!encode_map(&tm.Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Q, dQd, bQ) ||
       !encode_map(&tm.dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, dO, dQd, bQ) ||
       !encode_map(&tm.W, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW) ||

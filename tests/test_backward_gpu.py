@@ -83,6 +83,9 @@ TENSOR_CASES = [
     Workload("bwd_tc_m256", PERFORMER, "bf16", 1, 3, 520, 64, 64, 256, 311),
     Workload("bwd_tc_m128", PERFORMER, "bf16", 2, 2, 384, 64, 128, 128, 312),
     Workload("bwd_tc_m256_k256", PERFORMER, "bf16", 1, 2, 1000, 64, 256, 256, 313),
+    # a last feature tile of 64: padded to 128 inside the kernel with weights that are exactly zero
+    Workload("bwd_tc_m64", PERFORMER, "bf16", 1, 3, 392, 64, 128, 64, 320),
+    Workload("bwd_tc_m192", PERFORMER, "bf16", 2, 2, 264, 64, 64, 192, 321),
 ]
 
 
@@ -96,7 +99,7 @@ def test_backward_tensor_stage1_and_projection_gradients_only():
     """Shapes whose query side has no tensor-core backward still take stage 1 and dK, dV, dE, dF from the
     tensor-core kernels: RNN, d = 128 (two 64-column blocks per head), 64 features, ragged N and k = 64."""
     for w, layout in ((Workload("bwd_tc1_rnn_d128", RNN, "bf16", 1, 3, 200, 128, 64, 0, 317), "bhnd"),
-                      (Workload("bwd_tc1_perf_m64", PERFORMER, "bf16", 2, 2, 328, 64, 192, 64, 318), "bnhd"),
+                      (Workload("bwd_tc1_rnn_d64", RNN, "bf16", 2, 2, 328, 64, 192, 0, 318), "bnhd"),
                       (Workload("bwd_tc1_perf_d128", PERFORMER, "bf16", 1, 2, 520, 128, 320, 128, 319), "bhnd")):
         _check(w, layout=layout)
         assert binding.flurka_last_path() == binding.PATH_TENSOR_STAGE1

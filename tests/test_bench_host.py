@@ -52,3 +52,22 @@ def test_dominant_kernel_follows_the_stage_times():
     w = configs.C4
     roof, _ = bench.rooflines(w, _res([0.21, 0.03, 0.15], [0.4]), PEAKS, steps=1, world=1, exp_rate=None)
     assert roof["kernel"] == "down_projection" and roof["bound"] == "tensor" and "exp" not in roof
+
+
+def test_backward_block_counts_the_backward_work():
+    """The backward's FLOPs: stage 1 again, the four products with E, F, K, V and, for PERFORMER, the
+    four N x m x d products of the query side and the four k x m x d ones of the key side."""
+    w = configs.C3
+    flops, byts = bench.backward_work(w)
+    BH = w.B * w.H
+    assert flops == BH * (12 * w.N * w.k * w.d + 8 * w.N * w.m * w.d + 12 * w.k * w.m * w.d)
+    assert byts == 7 * w.tokens * w.d * w.elem_bytes + 4 * w.k * w.N * w.elem_bytes
+    rb = {"total_ms": 2.2, "step_ms": [1.0, 1.2], "path": "tensor", "launches": 20, "status": 0, "flushed": False}
+    blk = bench.backward_block(w, rb, PEAKS, steps=2, world=1)
+    assert abs(blk["ms_per_step"] - 1.1) < 1e-12
+    assert abs(blk["value"] - w.tokens / 1.1e-3) < 1e-3
+    want = max(flops / (PEAKS["bf16_tflops"] * 1e12), byts / (PEAKS["hbm_gbs"] * 1e9)) / 1.1e-3
+    assert abs(blk["path_roofline"]["frac"] - want) < 1e-12
+    # RNN: no feature products on either side beyond the d x d ones the forward counts
+    f2, _ = bench.backward_work(configs.C2)
+    assert f2 == configs.C2.B * configs.C2.H * 12 * configs.C2.N * configs.C2.k * configs.C2.d
