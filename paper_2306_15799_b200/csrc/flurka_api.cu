@@ -813,10 +813,10 @@ struct BackwardLayout {
   size_t da, dab_bytes, db, dkpvp, abf, split, total;
 };
 
-// the query side of the backward has a tensor-core kernel for PERFORMER with d = 64 (any feature count the
-// forward's tensor path takes: 64, 128, 192, 256)
+// the query side of the backward has a tensor-core kernel for d = 64 (PERFORMER: any feature count the
+// forward's tensor path takes, 64 to 256; RNN: its 64 features are the head dimension)
 bool backward_tensor_ok(const Problem& pr) {
-  return tensor_path_ok(pr) && pr.kernel == FLURKA_PERFORMER && pr.d == 64;
+  return tensor_path_ok(pr) && pr.d == 64;
 }
 
 BackwardLayout make_backward_layout(const Problem& pr) {
@@ -876,7 +876,7 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
     if (rc) return rc;
   }
   if (tc && tcq) {
-    rc = launch_k4(*tc, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.p(),
+    rc = launch_k4(*tc, P, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.p(),
                    (int*)(ws + L.status), st, &cuda_err);
     if (rc) { g_last_cuda_error = cuda_err; return rc; }
     *launches += 2;
@@ -972,7 +972,7 @@ int flurka_backward(const void* Q, const void* K, const void* V, const void* E, 
   else
     rc = perf ? backward_pipeline<__nv_bfloat16, true>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st, &launches, tc, tcq)
               : backward_pipeline<__nv_bfloat16, false>(pr, BL, ws, Q, K, V, E, F, W, dO, dQ, dK, dV, dE, dF, st,
-                                                        &launches, tc, false);
+                                                        &launches, tc, tcq);
   if (rc) return rc;
   ds.partial_pending = false;
   ds.timer.have = false;

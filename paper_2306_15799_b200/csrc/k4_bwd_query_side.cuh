@@ -70,6 +70,7 @@ __global__ void k4_split_a(const float* __restrict__ a32, __nv_bfloat16* __restr
   }
 }
 
+template <bool kPerformer>
 __global__ void __launch_bounds__(kK4Threads, 1)
 k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
                   const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
@@ -204,11 +205,13 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     prefetch_tmap(&tmDO);
     prefetch_tmap(&tmW);
     prefetch_tmap(&tmA);
-    mbar_arrive_expect_tx(bar_w, (uint32_t)nh * 16384u);
-    tma_load_2d(base + kK4W, &tmW, bar_w, 0, 0);
+    if (kPerformer) {
+      mbar_arrive_expect_tx(bar_w, (uint32_t)nh * 16384u);
+      tma_load_2d(base + kK4W, &tmW, bar_w, 0, 0);
+    }
     load_tile(0);
   }
-  if (ntiles > 0) {
+  if (kPerformer && ntiles > 0) {
     const bool mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
     ok = __syncthreads_and(mine) != 0;
   }
@@ -230,7 +233,18 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tma_load_3d(base + kK4AHi, &tmA, bar_head, 0, 0, head * 2);
         tma_load_3d(base + kK4ALo, &tmA, bar_head, 0, 0, head * 2 + 1);
       }
-      if (warp == 1) {
+      if (!kPerformer && warp == 1) {
+        // RNN: the weight of feature i is (elu(q_ni) + 1) z_i; z_i / max z as floats where the bias operand would be
+        const float* wv = prm.weight + (size_t)head * p;
+        float mxz = 0.f;
+        for (int f = lane; f < p; f += 32) mxz = fmaxf(mxz, wv[f]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mxz = fmaxf(mxz, __shfl_xor_sync(0xffffffffu, mxz, o));
+        float* zs = reinterpret_cast<float*>(base_ptr + kK4Bias);
+        const float inv = 1.f / mxz;
+        for (int f = lane; f < 128; f += 32) zs[f] = f < p ? wv[f] * inv : 0.f;
+      }
+      if (kPerformer && warp == 1) {
         // bias[f][c], c < 16, no swizzle: b_f - max b as three bf16 terms in columns 0..2
         const float* wv = prm.weight + (size_t)head * p;
         float mx = -INFINITY;
@@ -269,12 +283,14 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     auto issue_sg = [&](int h) {
       tcgen05_fence_after();
-      const uint64_t aq = make_sdesc(sm_q, 16, 1024, kSwizzle128);
-      const uint64_t bw = make_sdesc(base + kK4W + h * 16384, 16, 1024, kSwizzle128);
-      mma_ss_x4(tmem, aq, bw, 2, 2, idescS, 0u);
-      const uint64_t a1 = make_sdesc(base + kK4Ones, 128, 256, kSwizzleNone);
-      const uint64_t b1 = make_sdesc(base + kK4Bias + h * 4096, 128, 256, kSwizzleNone);
-      mma_ss(tmem, a1, b1, idescS, 1u);
+      if (kPerformer) {
+        const uint64_t aq = make_sdesc(sm_q, 16, 1024, kSwizzle128);
+        const uint64_t bw = make_sdesc(base + kK4W + h * 16384, 16, 1024, kSwizzle128);
+        mma_ss_x4(tmem, aq, bw, 2, 2, idescS, 0u);
+        const uint64_t a1 = make_sdesc(base + kK4Ones, 128, 256, kSwizzleNone);
+        const uint64_t b1 = make_sdesc(base + kK4Bias + h * 4096, 128, 256, kSwizzleNone);
+        mma_ss(tmem, a1, b1, idescS, 1u);
+      }
       const uint64_t ag = make_sdesc(sm_do, 16, 1024, kSwizzle128);
       const uint64_t bh = make_sdesc(base + kK4AHi + h * 16384, 16, 1024, kSwizzle128);
       const uint64_t bl = make_sdesc(base + kK4ALo + h * 16384, 16, 1024, kSwizzle128);
@@ -283,6 +299,27 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       mma_commit(bar_mma);
     };
 
+    // RNN: the un-normalised weights (elu(q_ni) + 1) z_i / max z of 32 features (i = c .. c + 31 = columns of
+    // this thread's row of the Q tile, which is 128-byte swizzled) and the factor elu'(q) / (elu(q) + 1)
+    auto rnn_weights = [&](int c, float (&pv)[32], float (&ratio)[32]) {
+      const float* zs = reinterpret_cast<const float*>(base_ptr + kK4Bias);
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        const uint32_t ch = (uint32_t)((c >> 3) + g);
+        uint32_t w4[4];
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w4[0]), "=r"(w4[1]), "=r"(w4[2]), "=r"(w4[3])
+                     : "r"(sm_q + (uint32_t)row * 128u + ((ch ^ (uint32_t)(row & 7)) << 4)));
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float x0 = __uint_as_float(w4[e] << 16), x1 = __uint_as_float(w4[e] & 0xffff0000u);
+          const int f = 8 * g + 2 * e;
+          pv[f] = (x0 > 0.f ? x0 + 1.f : __expf(x0)) * zs[c + f];
+          pv[f + 1] = (x1 > 0.f ? x1 + 1.f : __expf(x1)) * zs[c + f + 1];
+          ratio[f] = x0 > 0.f ? 1.f / (x0 + 1.f) : 1.f;
+          ratio[f + 1] = x1 > 0.f ? 1.f / (x1 + 1.f) : 1.f;
+        }
+      }
+    };
     // ------------------------------------------------------------ sweep 1: log-sum-exp and delta of each row
     float mx = -INFINITY, den = 0.f, num = 0.f;     // mx in the base-2 domain
     for (int h = 0; h < nh && ok; ++h) {
@@ -296,6 +333,20 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll 1
           for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
             uint32_t rs[32], rg[32];
+            if (!kPerformer) {
+              // no exponent to stabilise: the weights are products of bounded factors
+              float pv[32], ratio[32];
+              tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
+              rnn_weights(c, pv, ratio);
+              tmem_wait_ld(rg);
+              mx = 0.f;
+#pragma unroll
+              for (int e = 0; e < 32; ++e) {
+                den += pv[e];
+                num = fmaf(pv[e], __uint_as_float(rg[e]), num);
+              }
+              continue;
+            }
             tmem_ld32(tmem + lane_off + c, rs);
             tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
             tmem_wait_ld(rs);
@@ -357,13 +408,43 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll 1
           for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
             uint32_t rs[32], rg[32], cw[16];
+            const uint32_t slab = prow + (uint32_t)(c >> 6) * 16384u;
+            // features past p (padding of the last tile): P and c exactly zero
+            const float keep = (h * 128 + fh * 64 < p) ? 1.f : 0.f;
+            if (!kPerformer) {
+              // RNN (p = d = 64): P = weights / their sum; dq_ni = c_ni elu'(q_ni) / (elu(q_ni) + 1) needs no
+              // product, so this thread stores its 32 columns of the dQ row here
+              float pv[32], ratio[32];
+              tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
+              rnn_weights(c & 63, pv, ratio);
+              tmem_wait_ld(rg);
+              const float sc = keep / den;
+              const bool store = keep != 0.f && row0 + row < prm.N;
+              __nv_bfloat16* orow = prm.H > 0
+                  ? prm.dQ + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * 64
+                  : prm.dQ + ((size_t)head * prm.N + row0 + row) * 64;
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                uint32_t pw[4], dq[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const int j = 8 * g + 2 * e;
+                  const float p0 = pv[j] * sc, p1 = pv[j + 1] * sc;
+                  pw[e] = k4_bf16x2(p0, p1);
+                  dq[e] = k4_bf16x2(p0 * (__uint_as_float(rg[j]) - delta) * ratio[j],
+                                    p1 * (__uint_as_float(rg[j + 1]) - delta) * ratio[j + 1]);
+                }
+                const uint32_t chunk = (uint32_t)(((c & 32) >> 3) + g);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab + ((chunk ^ (uint32_t)(row & 7)) << 4)),
+                             "r"(pw[0]), "r"(pw[1]), "r"(pw[2]), "r"(pw[3]) : "memory");
+                if (store) *reinterpret_cast<uint4*>(orow + (c & 63) + 8 * g) = make_uint4(dq[0], dq[1], dq[2], dq[3]);
+              }
+              continue;
+            }
             tmem_ld32(tmem + lane_off + c, rs);
             tmem_ld32(tmem + lane_off + kK4ColG + c, rg);
             tmem_wait_ld(rs);
             tmem_wait_ld(rg);
-            const uint32_t slab = prow + (uint32_t)(c >> 6) * 16384u;
-            // features past p (padding of the last tile): P and c exactly zero
-            const float keep = (h * 128 + fh * 64 < p) ? 1.f : 0.f;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               uint32_t pw[4];
@@ -382,7 +463,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             // over this thread's own (already read) part of S: features 0..63 at columns 0..31, 64..127 at 64..95
             tmem_st16(tmem + lane_off + fh * 64 + ((c & 63) >> 1), cw);
           }
-          tmem_wait_st();
+          if (kPerformer) tmem_wait_st();
           fence_proxy_async_smem();
           tcgen05_fence_before();
         }
@@ -393,7 +474,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if (warp == 1 && elect_one()) {
         tcgen05_fence_after();
         // dQ (+)= c W: 128 features = 8 steps of 16, A 8 columns per step, B 16 rows of W per step
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; kPerformer && j < 2; ++j) {
           const uint64_t bw = make_sdesc(base + kK4W + h * 16384 + j * 8192, 8192, 1024, kSwizzle128);
           mma_ts_x4(tmem + kK4ColDQ, tmem + j * 64, bw, 128, idescQ, (h > 0 || j > 0) ? 1u : 0u);
         }
@@ -416,7 +497,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     first_of_head = false;
 
     // ------------------------------------------------------------ dQ rows (32 columns per thread)
-    if (owner) {
+    if (kPerformer && owner) {
       tcgen05_fence_after();
       uint32_t ra[32];
       tmem_ld32(tmem + lane_off + kK4ColDQ + fh * 32, ra);

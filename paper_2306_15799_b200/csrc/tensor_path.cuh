@@ -440,7 +440,7 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
 
 // ---- backward of the query side (PERFORMER, d = 64, p = 64, 128, 192 or 256): dQ, and da, db added to --
 // abf: scratch for the two bf16 terms of a, [BH][2][p][64]
-inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const void* W, const float* a32,
+inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const void* dO, const void* W, const float* a32,
                      const float* weight, __nv_bfloat16* abf, void* dQ, float* da, float* db, int BH, int H, int N,
                      int p, int* status, cudaStream_t st, int* cuda_err) {
   TensorMaps& tm = tc.maps;
@@ -455,7 +455,7 @@ inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const voi
   const unsigned bA[3] = {64, prows, 1};
   if (!encode_map(&tm.Q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, Q, dQd, bQ) ||
       !encode_map(&tm.dO, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, dO, dQd, bQ) ||
-      !encode_map(&tm.W, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW) ||
+      (performer && !encode_map(&tm.W, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW)) ||
       !encode_map(&tm.abf, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 3, abf, dA, bA)) {
     *cuda_err = (int)cudaErrorInvalidValue;
     return -6;
@@ -473,11 +473,13 @@ inline int launch_k4(TensorContext& tc, const void* Q, const void* dO, const voi
   prm.weight = weight; prm.a32 = a32;
   prm.dQ = reinterpret_cast<__nv_bfloat16*>(dQ);
   prm.da = da; prm.db = db; prm.status = status;
-  cudaError_t e = cudaFuncSetAttribute(k4_bwd_query_side, cudaFuncAttributeMaxDynamicSharedMemorySize, kK4SmemBytes);
+  auto fn = performer ? k4_bwd_query_side<true> : k4_bwd_query_side<false>;
+  cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK4SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   int grid = tc.sm_count();
   if (grid > prm.total_tiles) grid = prm.total_tiles;
-  k4_bwd_query_side<<<grid, kK4Threads, kK4SmemBytes, st>>>(tm.Q.map, tm.dO.map, tm.W.map, tm.abf.map, prm);
+  // the RNN kernel ignores tmW; pass any valid map
+  fn<<<grid, kK4Threads, kK4SmemBytes, st>>>(tm.Q.map, tm.dO.map, performer ? tm.W.map : tm.Q.map, tm.abf.map, prm);
   e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
