@@ -121,6 +121,23 @@ def test_backward_tensor_path_with_few_ctas(limit):
         binding.flurka_set_cta_limit(prev)
 
 
+def test_backward_full_length_sequences():
+    """c3's and c2's sequence lengths and projection sizes with two heads: every gradient against the oracle;
+    with few CTAs each one accumulates da, db over 64 tiles of a head before they leave TMEM."""
+    from paper_2306_15799_b200 import configs
+    w3 = configs.shrink(configs.C3, name="bwd_c3_two_heads", B=1, H=2)
+    w2 = configs.shrink(configs.C2, name="bwd_c2_two_heads", B=1, H=2)
+    _check(w3)
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    prev = binding.flurka_set_cta_limit(4)
+    try:
+        _check(w3)
+        _check(w2)
+        assert binding.flurka_last_path() == binding.PATH_TENSOR
+    finally:
+        binding.flurka_set_cta_limit(prev)
+
+
 def test_backward_cuda_core_path_on_a_tensor_shape():
     prev = binding.flurka_set_path(binding.PATH_SIMT)
     try:
