@@ -814,9 +814,10 @@ struct BackwardLayout {
 };
 
 // the query side of the backward has a tensor-core kernel for d = 64 (PERFORMER: any feature count the
-// forward's tensor path takes, 64 to 256; RNN: its 64 features are the head dimension)
+// forward's tensor path takes, 64 to 256; RNN: its 64 features are the head dimension) and for PERFORMER
+// with d = 128
 bool backward_tensor_ok(const Problem& pr) {
-  return tensor_path_ok(pr) && pr.d == 64;
+  return tensor_path_ok(pr) && (pr.d == 64 || pr.kernel == FLURKA_PERFORMER);
 }
 
 BackwardLayout make_backward_layout(const Problem& pr) {
@@ -876,7 +877,7 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
     if (rc) return rc;
   }
   if (tc && tcq) {
-    rc = launch_k4(*tc, P, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.p(),
+    rc = launch_k4(*tc, P, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.d, pr.p(),
                    (int*)(ws + L.status), st, &cuda_err);
     if (rc) { g_last_cuda_error = cuda_err; return rc; }
     *launches += 2;

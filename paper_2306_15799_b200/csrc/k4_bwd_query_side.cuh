@@ -26,12 +26,13 @@
 namespace flurka {
 
 struct K4Params {
-  int N, p, BH, H;              // H > 0: Q, dO, dQ are [B,N,H,64]; H == 0: [BH,N,64]
+  int N, p, BH, H;              // H > 0: Q, dO, dQ are [B,N,H,d]; H == 0: [BH,N,d]
+  int d;                        // 64, or 128 (PERFORMER only: see the kernel's header)
   int tiles_per_head, total_tiles;
   const float* weight;          // [BH][p]      b_i
-  const float* a32;             // [BH][p][64]  a_i (fp32)
+  const float* a32;             // [BH][p][d]   a_i (fp32)
   __nv_bfloat16* dQ;
-  float* da;                    // [BH][p][64]  added to
+  float* da;                    // [BH][p][d]   added to
   float* db;                    // [BH][p]      added to
   int* status;
 };
@@ -57,9 +58,9 @@ __device__ __forceinline__ float k4_ex2(float x) {
   return y;
 }
 
-// a [BH][p][64] fp32 -> two bf16 terms, [BH][2][p][64]
-__global__ void k4_split_a(const float* __restrict__ a32, __nv_bfloat16* __restrict__ abf, int BH, int p) {
-  const long long per_head = (long long)p * 64;
+// a [BH][p][d] fp32 -> two bf16 terms, [BH][2][p][d]
+__global__ void k4_split_a(const float* __restrict__ a32, __nv_bfloat16* __restrict__ abf, int BH, int p, int d) {
+  const long long per_head = (long long)p * d;
   const long long total = (long long)BH * per_head;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long h = i / per_head, r = i % per_head;
@@ -88,13 +89,18 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = prm.p, nh = (p + 127) >> 7;   // feature tiles of 128; rows of W, a past p are zero-filled by TMA
+  const int d = prm.d, kd = d >> 6;           // 64-column blocks of the head dimension
+  const bool stream = kd == 2;                // d = 128: see the header
+  const uint32_t bar_step = bars + 56;        // d = 128: W, a of the step's 128 features have landed
   const bool owner = warp >= 2;
   const int q4 = warp & 3, row = q4 * 32 + lane;
   const int fh = (warp - 2) >> 2;              // which 64 of a step's 128 features this row owner takes
   const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
 
-  const int t_begin = (int)(((long long)blockIdx.x * prm.total_tiles) / gridDim.x);
-  const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.total_tiles) / gridDim.x);
+  // d = 128: every tile is visited twice, once per 64-column half of dQ and da (index = half * total_tiles + tile)
+  const long long units = (long long)prm.total_tiles * kd;
+  const int t_begin = (int)(((long long)blockIdx.x * units) / gridDim.x);
+  const int t_end = (int)(((long long)(blockIdx.x + 1) * units) / gridDim.x);
   const int ntiles = t_end - t_begin;
 
   if (tid == 0) {
@@ -105,6 +111,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     mbar_init(bar_in + 8, 1);
     mbar_init(bar_mma, 1);
     mbar_init(bar_mma2, 1);
+    mbar_init(bar_step, 1);
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -138,9 +145,20 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const uint32_t tmem = tmem_base_shared;
 
   auto load_tile = [&](int i) {
-    const int tile = t_begin + i;
+    const int tile = (t_begin + i) % prm.total_tiles;
     const int head = tile / prm.tiles_per_head;
     const int row0 = (tile % prm.tiles_per_head) * 128;
+    if (stream) {
+      // one stage: Q as two 64-column slabs, then dO as two
+      const uint32_t dst = base + kK4In;
+      mbar_arrive_expect_tx(bar_in, 65536u);
+      for (int kb = 0; kb < 2; ++kb) {
+        const int x = (prm.H > 0 ? (head % prm.H) * 128 : 0) + kb * 64, z = prm.H > 0 ? head / prm.H : head;
+        tma_load_3d(dst + kb * 16384, &tmQ, bar_in, x, row0, z);
+        tma_load_3d(dst + 32768 + kb * 16384, &tmDO, bar_in, x, row0, z);
+      }
+      return;
+    }
     const uint32_t st = (uint32_t)(i & 1);
     const uint32_t dst = base + kK4In + st * 32768u;
     mbar_arrive_expect_tx(bar_in + 8 * st, 32768u);
@@ -154,7 +172,8 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   };
 
   // da, P^T delta of one head leave TMEM: thread = feature; db from the identity in the header
-  auto flush = [&](int head) {
+  auto flush = [&](int hkey) {
+    const int head = hkey % prm.BH, dh = hkey / prm.BH;     // dh: which 64 columns of da these accumulators are
     if (!owner || fh >= nh) return;
     tcgen05_fence_after();
     {
@@ -164,8 +183,8 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       tmem_wait_ld(dd);
       const int feat = hh * 128 + row;
       const bool live = feat < p;            // (the TMEM loads below are warp-wide: every lane takes them)
-      const float* arow = prm.a32 + ((size_t)head * p + (live ? feat : 0)) * 64;
-      float* darow = prm.da + ((size_t)head * p + (live ? feat : 0)) * 64;
+      const float* arow = prm.a32 + ((size_t)head * p + (live ? feat : 0)) * d + dh * 64;
+      float* darow = prm.da + ((size_t)head * p + (live ? feat : 0)) * d + dh * 64;
       float dot = 0.f;
 #pragma unroll 1
       for (int c = 0; c < 64; c += 32) {
@@ -184,14 +203,15 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int e = 0; e < 32; ++e)
           if (live) atomicAdd(darow + c + e, __uint_as_float(r[e]));
       }
-      const float pd = __uint_as_float(dd[0]) + __uint_as_float(dd[1]) + __uint_as_float(dd[2]);
+      // (both column halves accumulate P^T delta; it is subtracted once)
+      const float pd = dh == 0 ? __uint_as_float(dd[0]) + __uint_as_float(dd[1]) + __uint_as_float(dd[2]) : 0.f;
       if (live) atomicAdd(prm.db + (size_t)head * p + feat, dot - pd);
     }
     tcgen05_fence_before();
   };
 
   bool ok = true;
-  uint32_t ph_mma = 0, ph_mma2 = 0, ph_head = 0;
+  uint32_t ph_mma = 0, ph_mma2 = 0, ph_head = 0, ph_step = 0;
   int head_prev = -1;
   bool first_of_head = true;
   const float kLog2e = 1.4426950408889634f;
@@ -205,30 +225,32 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     prefetch_tmap(&tmDO);
     prefetch_tmap(&tmW);
     prefetch_tmap(&tmA);
-    if (kPerformer) {
+    if (kPerformer && !stream) {
       mbar_arrive_expect_tx(bar_w, (uint32_t)nh * 16384u);
       tma_load_2d(base + kK4W, &tmW, bar_w, 0, 0);
     }
-    load_tile(0);
+    if (!stream) load_tile(0);
   }
-  if (kPerformer && ntiles > 0) {
+  if (kPerformer && !stream && ntiles > 0) {
     const bool mine = mbar_wait(bar_w, 0, prm.status, &abort_flag);
     ok = __syncthreads_and(mine) != 0;
   }
 
   for (int i = 0; i < ntiles && ok; ++i) {
-    const int tile = t_begin + i;
+    const int dh = (t_begin + i) / prm.total_tiles;           // which 64 columns of dQ, da this visit is for (d = 128)
+    const int tile = (t_begin + i) % prm.total_tiles;
     const int head = tile / prm.tiles_per_head;
+    const int hkey = dh * prm.BH + head;
     const int row0 = (tile % prm.tiles_per_head) * 128;
-    const uint32_t st = (uint32_t)(i & 1);
-    const uint32_t sm_q = base + kK4In + st * 32768u, sm_do = sm_q + 16384u;
+    const uint32_t st = stream ? 0u : (uint32_t)(i & 1);
+    const uint32_t sm_q = base + kK4In + st * 32768u, sm_do = sm_q + (stream ? 32768u : 16384u);
 
-    if (head != head_prev) {
+    if (hkey != head_prev) {
       // every MMA issued so far has completed (the last wait of the previous tile), so the accumulators
       // of the old head can leave and its operands can be replaced
       if (head_prev >= 0) flush(head_prev);
       __syncthreads();
-      if (tid == 0) {
+      if (tid == 0 && !stream) {
         mbar_arrive_expect_tx(bar_head, 2u * (uint32_t)nh * 16384u);
         tma_load_3d(base + kK4AHi, &tmA, bar_head, 0, 0, head * 2);
         tma_load_3d(base + kK4ALo, &tmA, bar_head, 0, 0, head * 2 + 1);
@@ -266,36 +288,60 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         fence_proxy_async_smem();
       }
-      const bool mine = mbar_wait(bar_head, ph_head, prm.status, &abort_flag);
-      ph_head ^= 1;
+      const bool mine = stream ? true : mbar_wait(bar_head, ph_head, prm.status, &abort_flag);
+      if (!stream) ph_head ^= 1;
       ok = __syncthreads_and(mine) != 0;
       if (!ok) break;
-      head_prev = head;
+      head_prev = hkey;
       first_of_head = true;
     }
-    // the other stage held tile i-1, which is complete: fetch tile i+1 into it
-    if (tid == 0 && i + 1 < ntiles) load_tile(i + 1);
+    // the other stage held tile i-1, which is complete: fetch tile i+1 into it (d = 128: one stage, this tile now)
+    if (tid == 0 && !stream && i + 1 < ntiles) load_tile(i + 1);
+    if (tid == 0 && stream) load_tile(i);
     {
-      const bool mine = mbar_wait(bar_in + 8 * st, (uint32_t)(i >> 1) & 1u, prm.status, &abort_flag);
+      const bool mine = mbar_wait(bar_in + 8 * st, (stream ? (uint32_t)i : (uint32_t)(i >> 1)) & 1u, prm.status, &abort_flag);
       ok = __syncthreads_and(mine) != 0;
       if (!ok) break;
     }
 
+    // d = 128: W and the two terms of a for the step's 128 features (96 KB) come in before every step; every
+    // product that read the previous step's is complete by then
+    uint32_t step_ok = 1;
+    auto load_step = [&](int h) {
+      if (tid == 0) {
+        mbar_arrive_expect_tx(bar_step, 98304u);
+        for (int kb = 0; kb < 2; ++kb) {
+          tma_load_2d(base + kK4W + kb * 16384, &tmW, bar_step, kb * 64, h * 128);
+          tma_load_3d(base + kK4AHi + kb * 16384, &tmA, bar_step, kb * 64, h * 128, head * 2);
+          tma_load_3d(base + kK4ALo + kb * 16384, &tmA, bar_step, kb * 64, h * 128, head * 2 + 1);
+        }
+      }
+      const bool mine = mbar_wait(bar_step, ph_step, prm.status, &abort_flag);
+      ph_step ^= 1;
+      step_ok = __syncthreads_and(mine) != 0;
+    };
     auto issue_sg = [&](int h) {
       tcgen05_fence_after();
+      // rows of the step's features: at h * 16384 in the resident tiles (d = 64), at 0 in the step's own (d = 128);
+      // 64-column blocks of the head dimension 16384 B apart
+      const uint32_t fo = stream ? 0u : (uint32_t)h * 16384u;
       if (kPerformer) {
-        const uint64_t aq = make_sdesc(sm_q, 16, 1024, kSwizzle128);
-        const uint64_t bw = make_sdesc(base + kK4W + h * 16384, 16, 1024, kSwizzle128);
-        mma_ss_x4(tmem, aq, bw, 2, 2, idescS, 0u);
+        for (int kb = 0; kb < kd; ++kb) {
+          const uint64_t aq = make_sdesc(sm_q + kb * 16384, 16, 1024, kSwizzle128);
+          const uint64_t bw = make_sdesc(base + kK4W + fo + kb * 16384, 16, 1024, kSwizzle128);
+          mma_ss_x4(tmem, aq, bw, 2, 2, idescS, kb > 0 ? 1u : 0u);
+        }
         const uint64_t a1 = make_sdesc(base + kK4Ones, 128, 256, kSwizzleNone);
         const uint64_t b1 = make_sdesc(base + kK4Bias + h * 4096, 128, 256, kSwizzleNone);
         mma_ss(tmem, a1, b1, idescS, 1u);
       }
-      const uint64_t ag = make_sdesc(sm_do, 16, 1024, kSwizzle128);
-      const uint64_t bh = make_sdesc(base + kK4AHi + h * 16384, 16, 1024, kSwizzle128);
-      const uint64_t bl = make_sdesc(base + kK4ALo + h * 16384, 16, 1024, kSwizzle128);
-      mma_ss_x4(tmem + kK4ColG, ag, bh, 2, 2, idescS, 0u);
-      mma_ss_x4(tmem + kK4ColG, ag, bl, 2, 2, idescS, 1u);
+      for (int kb = 0; kb < kd; ++kb) {
+        const uint64_t ag = make_sdesc(sm_do + kb * 16384, 16, 1024, kSwizzle128);
+        const uint64_t bh = make_sdesc(base + kK4AHi + fo + kb * 16384, 16, 1024, kSwizzle128);
+        const uint64_t bl = make_sdesc(base + kK4ALo + fo + kb * 16384, 16, 1024, kSwizzle128);
+        mma_ss_x4(tmem + kK4ColG, ag, bh, 2, 2, idescS, kb > 0 ? 1u : 0u);
+        mma_ss_x4(tmem + kK4ColG, ag, bl, 2, 2, idescS, 1u);
+      }
       mma_commit(bar_mma);
     };
 
@@ -323,6 +369,10 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // ------------------------------------------------------------ sweep 1: log-sum-exp and delta of each row
     float mx = -INFINITY, den = 0.f, num = 0.f;     // mx in the base-2 domain
     for (int h = 0; h < nh && ok; ++h) {
+      if (stream) {
+        load_step(h);
+        if (!step_ok) { ok = false; break; }
+      }
       if (warp == 1 && elect_one()) issue_sg(h);
       bool mine = true;
       if (owner) {
@@ -398,6 +448,10 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
     // ------------------------------------------------------------ sweep 2: P, c and the three products they feed
     for (int h = 0; h < nh && ok; ++h) {
+      if (stream) {
+        load_step(h);
+        if (!step_ok) { ok = false; break; }
+      }
       if (warp == 1 && elect_one()) issue_sg(h);
       bool mine = true;
       if (owner) {
@@ -475,13 +529,14 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tcgen05_fence_after();
         // dQ (+)= c W: 128 features = 8 steps of 16, A 8 columns per step, B 16 rows of W per step
         for (int j = 0; kPerformer && j < 2; ++j) {
-          const uint64_t bw = make_sdesc(base + kK4W + h * 16384 + j * 8192, 8192, 1024, kSwizzle128);
+          // W rows of the step's features, the 64 columns this visit owns
+          const uint64_t bw = make_sdesc(base + kK4W + (stream ? dh : h) * 16384 + j * 8192, 8192, 1024, kSwizzle128);
           mma_ts_x4(tmem + kK4ColDQ, tmem + j * 64, bw, 128, idescQ, (h > 0 || j > 0) ? 1u : 0u);
         }
         // da_h (+)= P_h^T dO and (P^T delta)_h: 128 rows = 8 steps of 16 rows (2048 B of P and of dO, 256 B of delta)
         for (int j = 0; j < 2; ++j) {
           const uint64_t ap = make_sdesc(base + kK4P + j * 8192, 16384, 1024, kSwizzle128);
-          const uint64_t bo = make_sdesc(sm_do + j * 8192, 8192, 1024, kSwizzle128);
+          const uint64_t bo = make_sdesc(sm_do + (stream ? dh * 16384 : 0) + j * 8192, 8192, 1024, kSwizzle128);
           mma_ss_x4(tmem + kK4ColDA + h * 64, ap, bo, 128, 128, idescA, (!first_of_head || j > 0) ? 1u : 0u);
           const uint64_t bd = make_sdesc(base + kK4Delta + j * 1024, 128, 2048, kSwizzleNone);
           mma_ss_x4(tmem + kK4ColDD + h * 16, ap, bd, 128, 16, idescD, (!first_of_head || j > 0) ? 1u : 0u);
@@ -505,9 +560,9 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       tcgen05_fence_before();
       if (row0 + row < prm.N) {
         __nv_bfloat16* orow = prm.H > 0
-            ? prm.dQ + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * 64
-            : prm.dQ + ((size_t)head * prm.N + row0 + row) * 64;
-        orow += fh * 32;
+            ? prm.dQ + (((size_t)(head / prm.H) * prm.N + row0 + row) * prm.H + (size_t)(head % prm.H)) * d
+            : prm.dQ + ((size_t)head * prm.N + row0 + row) * d;
+        orow += dh * 64 + fh * 32;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint4 v;

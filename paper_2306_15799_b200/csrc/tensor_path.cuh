@@ -442,14 +442,14 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
 // abf: scratch for the two bf16 terms of a, [BH][2][p][64]
 inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const void* dO, const void* W, const float* a32,
                      const float* weight, __nv_bfloat16* abf, void* dQ, float* da, float* db, int BH, int H, int N,
-                     int p, int* status, cudaStream_t st, int* cuda_err) {
+                     int d, int p, int* status, cudaStream_t st, int* cuda_err) {
   TensorMaps& tm = tc.maps;
-  const int d = 64;
+  const bool stream = d == 128;      // W and a come in per step of 128 features (boxes of 128 rows)
   const unsigned long long dQd[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
                                      (unsigned long long)(H > 0 ? BH / H : BH)};
   const unsigned bQ[3] = {64, 128, 1};
   const unsigned long long dW[2] = {(unsigned long long)d, (unsigned long long)p};
-  const unsigned prows = (unsigned)((p + 127) / 128) * 128;      // whole 128-feature tiles; rows past p read as zero
+  const unsigned prows = stream ? 128u : (unsigned)((p + 127) / 128) * 128;   // whole 128-feature tiles; rows past p read as zero
   const unsigned bW[2] = {64, prows};
   const unsigned long long dA[3] = {(unsigned long long)d, (unsigned long long)p, (unsigned long long)BH * 2};
   const unsigned bA[3] = {64, prows, 1};
@@ -461,13 +461,13 @@ inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const voi
     return -6;
   }
   {
-    const long long total = (long long)BH * p * 64;
+    const long long total = (long long)BH * p * d;
     int grid = (int)((total + 255) / 256);
     if (grid > 148 * 8) grid = 148 * 8;
-    k4_split_a<<<grid, 256, 0, st>>>(a32, abf, BH, p);
+    k4_split_a<<<grid, 256, 0, st>>>(a32, abf, BH, p, d);
   }
   K4Params prm;
-  prm.N = N; prm.p = p; prm.BH = BH; prm.H = H;
+  prm.N = N; prm.p = p; prm.BH = BH; prm.H = H; prm.d = d;
   prm.tiles_per_head = (N + 127) / 128;
   prm.total_tiles = prm.tiles_per_head * BH;
   prm.weight = weight; prm.a32 = a32;
@@ -477,7 +477,7 @@ inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const voi
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK4SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   int grid = tc.sm_count();
-  if (grid > prm.total_tiles) grid = prm.total_tiles;
+  if (grid > prm.total_tiles * (d / 64)) grid = prm.total_tiles * (d / 64);
   // the RNN kernel ignores tmW; pass any valid map
   fn<<<grid, kK4Threads, kK4SmemBytes, st>>>(tm.Q.map, tm.dO.map, performer ? tm.W.map : tm.Q.map, tm.abf.map, prm);
   e = cudaGetLastError();

@@ -89,6 +89,10 @@ TENSOR_CASES = [
     # RNN with d = 64: its 64 features are the head dimension, the weights need no product and no exponent
     Workload("bwd_tc_rnn", RNN, "bf16", 2, 2, 392, 64, 192, 0, 322),
     Workload("bwd_tc_rnn_k256", RNN, "bf16", 1, 3, 1000, 64, 256, 0, 323),
+    # d = 128 (PERFORMER): W and a arrive per step of 128 features, every tile is visited once per 64-column half
+    Workload("bwd_tc_d128_m128", PERFORMER, "bf16", 1, 2, 520, 128, 320, 128, 319),
+    Workload("bwd_tc_d128_m256", PERFORMER, "bf16", 2, 2, 392, 128, 64, 256, 325),
+    Workload("bwd_tc_d128_m64", PERFORMER, "bf16", 1, 3, 264, 128, 128, 64, 326),
 ]
 
 
@@ -100,10 +104,10 @@ def test_backward_tensor_path_matches_oracle(w):
 
 def test_backward_tensor_stage1_and_projection_gradients_only():
     """Shapes whose query side has no tensor-core backward still take stage 1 and dK, dV, dE, dF from the
-    tensor-core kernels: d = 128 (two 64-column blocks per head), RNN and PERFORMER, ragged N and k = 64."""
+    tensor-core kernels: RNN with d = 128 (two 64-column blocks per head), ragged N, k = 64 and 320."""
     for w, layout in ((Workload("bwd_tc1_rnn_d128", RNN, "bf16", 1, 3, 200, 128, 64, 0, 317), "bhnd"),
                       (Workload("bwd_tc1_rnn_d128_bnhd", RNN, "bf16", 2, 2, 328, 128, 192, 0, 318), "bnhd"),
-                      (Workload("bwd_tc1_perf_d128", PERFORMER, "bf16", 1, 2, 520, 128, 320, 128, 319), "bhnd")):
+                      (Workload("bwd_tc1_rnn_d128_k320", RNN, "bf16", 1, 2, 520, 128, 320, 0, 327), "bhnd")):
         _check(w, layout=layout)
         assert binding.flurka_last_path() == binding.PATH_TENSOR_STAGE1
 
@@ -116,6 +120,7 @@ def test_backward_tensor_path_with_few_ctas(limit):
         _check(Workload("bwd_tc_few_ctas", PERFORMER, "bf16", 1, 3, 520, 64, 64, 256, 314))
         _check(Workload("bwd_tc_few_ctas_bnhd", PERFORMER, "bf16", 2, 2, 264, 64, 64, 128, 315), layout="bnhd")
         _check(Workload("bwd_tc_few_ctas_rnn", RNN, "bf16", 1, 3, 392, 64, 64, 0, 324), layout="bnhd")
+        _check(Workload("bwd_tc_few_ctas_d128", PERFORMER, "bf16", 2, 2, 264, 128, 64, 256, 328), layout="bnhd")
         assert binding.flurka_last_path() == binding.PATH_TENSOR
     finally:
         binding.flurka_set_cta_limit(prev)
