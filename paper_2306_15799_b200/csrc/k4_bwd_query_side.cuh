@@ -1,5 +1,5 @@
-// Backward of the query side on tensor cores (PERFORMER, bf16, d = 64, p = 64, 128, 192 or 256 features;
-// a last tile of 64 features is padded to 128 with weights that are exactly zero).
+// Backward of the query side on tensor cores (bf16; PERFORMER with p = 64, 128, 192 or 256 features and
+// d = 64 or 128, RNN with d = 64; a last tile of 64 features is padded to 128 with weights that are exactly zero).
 //
 // The forward's query side (arxiv 2306.15799, Eq. (2) with the normalised weights of Appendix D) is
 //     O_n = sum_i P_ni a_i,    P_n. = softmax_i(l_n.),    l_ni = w_i . q_n + b_i.
@@ -17,6 +17,11 @@
 // the head changes; db comes from them there.  Two threads per query row (8 warps; each takes 64 of the 128
 // features of a step), one MMA issuer, one TMA thread; the phases of a tile follow one another (block
 // barriers), nothing here waits for another CTA.
+// RNN (kPerformer = false): l_ni = log((elu(q_ni) + 1) z_i), so the weights come from the Q tile in shared
+// memory without a product or an exponent, and dq_ni = c_ni elu'(q_ni) / (elu(q_ni) + 1) is stored by the row owner.
+// d = 128: TMEM cannot hold dQ and da at full width beside S and G, nor shared memory W and both terms of a
+// for 256 features, so every tile is visited twice, once per 64-column half of dQ and da (S, G and the weights
+// are formed again), and W, a arrive per step of 128 features.
 #pragma once
 
 #include <cuda_bf16.h>
