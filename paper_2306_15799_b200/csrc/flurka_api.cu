@@ -810,7 +810,7 @@ namespace {
 // memset), then dK', dV' [2][BH][k][d]; all fp32.
 struct BackwardLayout {
   Layout L;
-  size_t da, dab_bytes, db, dkpvp, abf, split, total;
+  size_t da, dab_bytes, db, dkpvp, abf, split, rowstat, total;
 };
 
 // the query side of the backward has a tensor-core kernel for d = 64 (PERFORMER: any feature count the
@@ -832,6 +832,9 @@ BackwardLayout make_backward_layout(const Problem& pr) {
   b.dkpvp = off; off = align256(off + (size_t)2 * pr.BH() * pr.k * pr.d * 4);
   b.abf = off;
   if (backward_tensor_ok(pr)) off = align256(off + (size_t)2 * pr.BH() * pr.p() * pr.d * 2);   // a as two bf16 terms
+  b.rowstat = off;
+  if (backward_tensor_ok(pr) && pr.d == 128)             // (log-sum-exp, delta) of every row of every 128-row tile
+    off = align256(off + (size_t)pr.BH() * ((pr.N + 127) / 128) * 128 * 8);
   b.split = off;
   if (tensor_path_ok(pr)) off = align256(off + (size_t)2 * pr.k * 2 * pr.BH() * pr.d * 2);      // dK', dV' as two bf16 terms
   b.total = off;
@@ -878,7 +881,7 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
   }
   if (tc && tcq) {
     rc = launch_k4(*tc, P, Q, dO, W, a32, weight, (__nv_bfloat16*)(ws + BL.abf), dQ, da, db, pr.BH(), smh, pr.N, pr.d, pr.p(),
-                   (int*)(ws + L.status), st, &cuda_err);
+                   (int*)(ws + L.status), st, &cuda_err, ws + BL.rowstat);
     if (rc) { g_last_cuda_error = cuda_err; return rc; }
     *launches += 2;
   } else {

@@ -39,6 +39,8 @@ struct K4Params {
   __nv_bfloat16* dQ;
   float* da;                    // [BH][p][d]   added to
   float* db;                    // [BH][p]      added to
+  float2* rowstat;              // d = 128: [total_tiles * 128] (log-sum-exp, delta) of every row, kept from a
+                                // tile's first visit for its second
   int* status;
 };
 
@@ -102,11 +104,11 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int fh = (warp - 2) >> 2;              // which 64 of a step's 128 features this row owner takes
   const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
 
-  // d = 128: every tile is visited twice, once per 64-column half of dQ and da (index = half * total_tiles + tile)
-  const long long units = (long long)prm.total_tiles * kd;
-  const int t_begin = (int)(((long long)blockIdx.x * units) / gridDim.x);
-  const int t_end = (int)(((long long)(blockIdx.x + 1) * units) / gridDim.x);
-  const int ntiles = t_end - t_begin;
+  // d = 128: a CTA walks its tiles twice, once per 64-column half of dQ and da (visit i: half i / nt, tile i % nt)
+  const int t_begin = (int)(((long long)blockIdx.x * prm.total_tiles) / gridDim.x);
+  const int t_end = (int)(((long long)(blockIdx.x + 1) * prm.total_tiles) / gridDim.x);
+  const int nt = t_end - t_begin;
+  const int ntiles = nt * kd;
 
   if (tid == 0) {
     abort_flag = 0;
@@ -150,7 +152,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const uint32_t tmem = tmem_base_shared;
 
   auto load_tile = [&](int i) {
-    const int tile = (t_begin + i) % prm.total_tiles;
+    const int tile = t_begin + i % nt;
     const int head = tile / prm.tiles_per_head;
     const int row0 = (tile % prm.tiles_per_head) * 128;
     if (stream) {
@@ -242,8 +244,10 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   }
 
   for (int i = 0; i < ntiles && ok; ++i) {
-    const int dh = (t_begin + i) / prm.total_tiles;           // which 64 columns of dQ, da this visit is for (d = 128)
-    const int tile = (t_begin + i) % prm.total_tiles;
+    const int dh = i / nt;                                    // which 64 columns of dQ, da this visit is for (d = 128)
+    const int tile = t_begin + i % nt;
+    // second visit of a tile: its rows' log-sum-exp and delta are on record, sweep 1 is not done again
+    const bool have_stats = stream && dh == 1;
     const int head = tile / prm.tiles_per_head;
     const int hkey = dh * prm.BH + head;
     const int row0 = (tile % prm.tiles_per_head) * 128;
@@ -373,7 +377,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     };
     // ------------------------------------------------------------ sweep 1: log-sum-exp and delta of each row
     float mx = -INFINITY, den = 0.f, num = 0.f;     // mx in the base-2 domain
-    for (int h = 0; h < nh && ok; ++h) {
+    for (int h = 0; h < nh && ok && !have_stats; ++h) {
       if (stream) {
         load_step(h);
         if (!step_ok) { ok = false; break; }
@@ -429,9 +433,9 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
     if (!ok) break;
     // the two threads of a row put their parts together (both in the same order, so they agree to the bit)
-    if (owner) { stat[fh][0][row] = mx; stat[fh][1][row] = den; stat[fh][2][row] = num; }
+    if (owner && !have_stats) { stat[fh][0][row] = mx; stat[fh][1][row] = den; stat[fh][2][row] = num; }
     __syncthreads();
-    if (owner) {
+    if (owner && !have_stats) {
       const float m0 = stat[0][0][row], m1 = stat[1][0][row];
       const float nm = fmaxf(m0, m1);
       const float s0 = k4_ex2(m0 - nm), s1 = k4_ex2(m1 - nm);
@@ -439,8 +443,18 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       den = fmaf(stat[0][1][row], s0, stat[1][1][row] * s1);
       num = fmaf(stat[0][2][row], s0, stat[1][2][row] * s1);
     }
-    const float lse2 = mx + __log2f(den);
-    const float delta = num / den;
+    float lse2 = mx + __log2f(den);
+    float delta = num / den;
+    if (stream && owner) {
+      float2* rs2 = prm.rowstat + (size_t)tile * 128 + row;
+      if (have_stats) {
+        const float2 v = *rs2;
+        lse2 = v.x;
+        delta = v.y;
+      } else if (fh == 0) {
+        *rs2 = make_float2(lse2, delta);
+      }
+    }
     if (owner && fh == 0) {
       // delta_n as three bf16 terms: element (c, n) of the [16 x 128] operand at (n/8)*128 + c*16 + (n%8)*2 bytes
       __nv_bfloat16* dt = reinterpret_cast<__nv_bfloat16*>(base_ptr + kK4Delta) + (row >> 3) * 64 + (row & 7);

@@ -442,7 +442,8 @@ inline int launch_k3(TensorContext& tc, bool performer, const void* Q, const voi
 // abf: scratch for the two bf16 terms of a, [BH][2][p][64]
 inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const void* dO, const void* W, const float* a32,
                      const float* weight, __nv_bfloat16* abf, void* dQ, float* da, float* db, int BH, int H, int N,
-                     int d, int p, int* status, cudaStream_t st, int* cuda_err) {
+                     int d, int p, int* status, cudaStream_t st, int* cuda_err, void* rowstat = nullptr) {
+  // rowstat: d = 128 only, 8 bytes per query row of every 128-row tile (BH * ceil(N / 128) * 128 rows)
   TensorMaps& tm = tc.maps;
   const bool stream = d == 128;      // W and a come in per step of 128 features (boxes of 128 rows)
   const unsigned long long dQd[3] = {(unsigned long long)(H > 0 ? H * d : d), (unsigned long long)N,
@@ -473,11 +474,12 @@ inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const voi
   prm.weight = weight; prm.a32 = a32;
   prm.dQ = reinterpret_cast<__nv_bfloat16*>(dQ);
   prm.da = da; prm.db = db; prm.status = status;
+  prm.rowstat = reinterpret_cast<float2*>(rowstat);
   auto fn = performer ? k4_bwd_query_side<true> : k4_bwd_query_side<false>;
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK4SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   int grid = tc.sm_count();
-  if (grid > prm.total_tiles * (d / 64)) grid = prm.total_tiles * (d / 64);
+  if (grid > prm.total_tiles) grid = prm.total_tiles;
   // the RNN kernel ignores tmW; pass any valid map
   fn<<<grid, kK4Threads, kK4SmemBytes, st>>>(tm.Q.map, tm.dO.map, performer ? tm.W.map : tm.Q.map, tm.abf.map, prm);
   e = cudaGetLastError();
