@@ -26,10 +26,12 @@ struct K5Params {
 
 // kMode 0 has a short contraction (2 k / 64 chunks) and a long epilogue: 128 x 256 outputs per CTA and two
 // 48 KB stages, so that two CTAs share an SM and one's epilogue runs under the other's MMAs; kMode 1 has a
-// long contraction: 256 x 256 outputs and three 64 KB stages
+// long contraction: 256 x 256 outputs and three 64 KB stages; kMode 2 is kMode 1 with 128 x 256 outputs and four
+// 48 KB stages, for shapes whose dE, dF have too few 256 x 256 tiles to occupy the SMs (each CTA is then bound
+// by the latency of its ring, so more CTAs with more, smaller stages in flight go faster)
 template <int kMode> struct K5Shape {
-  static constexpr int kRows = kMode == 0 ? 128 : 256;
-  static constexpr int kStages = kMode == 0 ? 2 : 3;
+  static constexpr int kRows = kMode == 1 ? 256 : 128;
+  static constexpr int kStages = kMode == 0 ? 2 : (kMode == 1 ? 3 : 4);
   static constexpr int kABytes = kRows * 128;                       // 64 contraction elements per row
   static constexpr int kStageBytes = kABytes + 32768;
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
@@ -75,10 +77,10 @@ k5_bwd_projections(const __grid_constant__ CUtensorMap tmP0, const __grid_consta
   constexpr int kK5Stages = K5Shape<kMode>::kStages, kK5StageBytes = K5Shape<kMode>::kStageBytes;
   constexpr int kRows = K5Shape<kMode>::kRows, kABytes = K5Shape<kMode>::kABytes;
   const uint32_t bar_base = smem_base + kK5Stages * kK5StageBytes;
-  const uint32_t bar_full = bar_base;                 // [3]
-  const uint32_t bar_empty = bar_base + 24;           // [3]
-  const uint32_t bar_accum = bar_base + 48;
-  const uint32_t tmem_slot = bar_base + 64;
+  const uint32_t bar_full = bar_base;                 // [<= 4]
+  const uint32_t bar_empty = bar_base + 32;           // [<= 4]
+  const uint32_t bar_accum = bar_base + 64;
+  const uint32_t tmem_slot = bar_base + 80;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
 

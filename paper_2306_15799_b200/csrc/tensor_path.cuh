@@ -515,6 +515,8 @@ inline int launch_k5(TensorContext& tc, const void* E, const void* F, const void
                                          K5Shape<0>::kSmemBytes);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(k5_bwd_projections<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, K5Shape<1>::kSmemBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(k5_bwd_projections<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, K5Shape<2>::kSmemBytes);
     if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
     tc.k5_attr = true;
   }
@@ -532,8 +534,15 @@ inline int launch_k5(TensorContext& tc, const void* E, const void* F, const void
       tm.bE.map, tm.bF.map, tm.split64.map, tm.gK.map, tm.gV.map, p);
   p.row_blocks = (k + 255) / 256;
   p.col_groups = (N + 255) / 256;
-  k5_bwd_projections<1><<<2 * p.row_blocks * p.col_groups, kK5Threads, K5Shape<1>::kSmemBytes, st>>>(
-      tm.bK.map, tm.bV.map, tm.split128.map, tm.gE.map, tm.gF.map, p);
+  if (2 * p.row_blocks * p.col_groups >= 100) {
+    k5_bwd_projections<1><<<2 * p.row_blocks * p.col_groups, kK5Threads, K5Shape<1>::kSmemBytes, st>>>(
+        tm.bK.map, tm.bV.map, tm.split128.map, tm.gE.map, tm.gF.map, p);
+  } else {
+    // few tiles: 128-row tiles put twice as many CTAs to work, each with four smaller stages in flight
+    p.row_blocks = (k + 127) / 128;
+    k5_bwd_projections<2><<<2 * p.row_blocks * p.col_groups, kK5Threads, K5Shape<2>::kSmemBytes, st>>>(
+        tm.bK.map, tm.bV.map, tm.split128.map, tm.gE.map, tm.gF.map, p);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
