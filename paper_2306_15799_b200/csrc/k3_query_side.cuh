@@ -100,6 +100,10 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
   const uint32_t tmem_slot = bars + 320;
   __shared__ int abort_flag;
   __shared__ uint32_t tmem_base_shared;
+  // RNN: how many heads' scale vectors have been built so far.  A count, not an mbarrier: a row-owner group
+  // whose first tile already belongs to the CTA's second head has never waited for the first head's phase, and a
+  // parity wait cannot tell "phase 1 complete" from "nothing complete yet".
+  __shared__ volatile int scale_epoch;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -110,6 +114,7 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
+    scale_epoch = 0;
     for (int i = 0; i < kK3MaxQStages; ++i) {
       mbar_init(bar_qfull + 8 * i, 1);
       mbar_init(bar_qempty + 8 * i, kPerformer ? 1 : 128);
@@ -323,6 +328,11 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           float* sc = reinterpret_cast<float*>(base_ptr + L.scale);
           const float inv = 1.f / mx;
           for (int f = lane; f < p; f += 32) sc[f] = wv[f] * inv;
+          __syncwarp();
+          if (lane == 0) {
+            __threadfence_block();
+            scale_epoch = events + 1;
+          }
         }
         mbar_arrive(bar_biasready);
         head_prev = head;
@@ -510,7 +520,24 @@ k3_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
           // RNN: p_f = (elu(q_f) + 1) * z_f / max z, features = the d entries of the Q row
           // (no wait for the buffer: this thread has itself read out the tile that used it before, and
           // the second product starts only when all 128 owners have said so)
-          ok = mbar_wait(bar_biasready, (events - 1) & 1, prm.status, &abort_flag);
+          // this head's scale vector is in place (it is replaced only after every product of this head, hence
+          // every row owner's use of it, is complete)
+          if (scale_epoch < events) {
+            const uint64_t t0 = global_timer_ns();
+            uint32_t spins = 0;
+            while (scale_epoch < events) {
+              if ((++spins & 63u) == 0) {
+                if (abort_flag) { ok = false; break; }
+                if (global_timer_ns() - t0 > kWaitLimitNs) {
+                  atomicOr(prm.status, 1);
+                  abort_flag = 1;
+                  ok = false;
+                  break;
+                }
+              }
+            }
+          }
+          __threadfence_block();
           if (ok) ok = mbar_wait(bar_qfull + 8 * st, (i >> ns_shift) & 1, prm.status, &abort_flag);
           if (!ok) break;
           const uint32_t qb = base + L.q + st * q_stage_bytes;

@@ -58,7 +58,8 @@ def _check_full(w, heads, n_rows, seed=0):
 
 
 def test_c2_full_size():
-    _check_full(configs.C2, heads=[(0, 0), (3, 7), (7, 11)], n_rows=512)
+    # (1, 1): with 148 CTAs its first tile is the second tile of a CTA whose first tile is head (1, 0)'s last
+    _check_full(configs.C2, heads=[(0, 0), (1, 1), (3, 7), (7, 11)], n_rows=512)
 
 
 def test_c3_full_size():

@@ -256,6 +256,21 @@ def test_tensor_path_matches_oracle(w, limit):
         binding.flurka_set_cta_limit(prev)
 
 
+@pytest.mark.parametrize("limit,tiles", [(1, 1), (2, 3), (3, 1)])
+def test_rnn_head_change_at_a_ctas_second_tile(limit, tiles):
+    """RNN query side: a row-owner group whose first tile already belongs to the CTA's second head must still
+    get that head's scale vector (tiles of one head per CTA: 1 or 3, so the odd group starts in a later head).
+    Repeated, because a stale vector shows only when the group runs ahead of the operand builder."""
+    from paper_2306_15799_b200.configs import Workload
+    w = Workload("rnn_head_change_t%d" % tiles, RNN, "bf16", 2, 5, 128 * tiles, 64, 64, 0, 417 + tiles)
+    prev = binding.flurka_set_cta_limit(limit)
+    try:
+        for _ in range(6):
+            pu.check_all_heads(w, path=binding.PATH_TENSOR)
+    finally:
+        binding.flurka_set_cta_limit(prev)
+
+
 def test_auto_picks_tensor_path_when_the_shape_allows():
     w = TENSOR_CASES[0]
     pu.check_all_heads(w)
