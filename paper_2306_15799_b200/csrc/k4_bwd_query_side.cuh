@@ -78,7 +78,7 @@ __global__ void k4_split_a(const float* __restrict__ a32, __nv_bfloat16* __restr
   }
 }
 
-template <bool kPerformer>
+template <bool kPerformer, bool kStream>
 __global__ void __launch_bounds__(kK4Threads, 1)
 k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmDO,
                   const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
@@ -96,8 +96,9 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = prm.p, nh = (p + 127) >> 7;   // feature tiles of 128; rows of W, a past p are zero-filled by TMA
-  const int d = prm.d, kd = d >> 6;           // 64-column blocks of the head dimension
-  const bool stream = kd == 2;                // d = 128: see the header
+  constexpr int kd = kStream ? 2 : 1;         // 64-column blocks of the head dimension
+  constexpr int d = 64 * kd;
+  constexpr bool stream = kStream;            // d = 128: see the header
   const uint32_t bar_step = bars + 56;        // d = 128: W, a of the step's 128 features have landed
   const bool owner = warp >= 2;
   const int q4 = warp & 3, row = q4 * 32 + lane;

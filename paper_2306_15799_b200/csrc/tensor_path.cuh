@@ -475,7 +475,7 @@ inline int launch_k4(TensorContext& tc, bool performer, const void* Q, const voi
   prm.dQ = reinterpret_cast<__nv_bfloat16*>(dQ);
   prm.da = da; prm.db = db; prm.status = status;
   prm.rowstat = reinterpret_cast<float2*>(rowstat);
-  auto fn = performer ? k4_bwd_query_side<true> : k4_bwd_query_side<false>;
+  auto fn = stream ? k4_bwd_query_side<true, true> : (performer ? k4_bwd_query_side<true, false> : k4_bwd_query_side<false, false>);
   cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kK4SmemBytes);
   if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
   int grid = tc.sm_count();
