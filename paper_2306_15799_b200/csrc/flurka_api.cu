@@ -896,7 +896,7 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
   }
   {
     auto fn = simt_bwd_key_side<T, P>;
-    const size_t smem = (size_t)3 * 32 * (pr.d + 1) * 4;
+    const size_t smem = ((size_t)3 * 32 * (pr.d + 1) + (size_t)2 * 8 * kBwdKeysPerWarp * pr.d) * 4;
     if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
       return cuda_fail(e);
     dim3 grid((pr.k + 8 * kBwdKeysPerWarp - 1) / (8 * kBwdKeysPerWarp), pr.BH());

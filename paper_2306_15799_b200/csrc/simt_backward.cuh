@@ -219,11 +219,11 @@ simt_bwd_query_side(const T* __restrict__ Q, const T* __restrict__ W, const T* _
 // lane = column for the sums over features; A and dL of a chunk go through shared memory so that the
 // column loop reads the four keys' values of a feature with one 16-byte broadcast load each.
 // Inputs: K', V' (KpVp), W, a, b (weight), da, db.  Outputs: dKpVp [2][B*H][k][d] fp32 (dK' then dV').
-// Dynamic shared memory: 3 * 32 * (d+1) floats (W, a, da chunks).
+// Dynamic shared memory: 3 * 32 * (d+1) floats (W, a, da chunks) + 2 * 32 * d floats (the block's keys, values).
 // ---------------------------------------------------------------------------------------------
 constexpr int kBwdKeysPerWarp = 4;
 template <typename T, bool kPerformer>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const float* __restrict__ weight,
                   const float* __restrict__ a32, const float* __restrict__ da, const float* __restrict__ db,
                   float* __restrict__ dKpVp, int BH, int d, int k, int p) {
@@ -232,7 +232,9 @@ simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const
   float* Ws = smem;                          // [32][d+1]
   float* As = Ws + 32 * (d + 1);             // [32][d+1]
   float* Ds = As + 32 * (d + 1);             // [32][d+1]  da chunk
-  __shared__ float ks[8 * KW][128], vs[8 * KW][128];
+  // the block's 8 * KW keys and values, rows of d floats (dynamic: d = 64 leaves room for a fourth block per SM)
+  float* ks = Ds + 32 * (d + 1);             // [8 * KW][d]
+  float* vs = ks + 8 * KW * d;               // [8 * KW][d]
   __shared__ __align__(16) float sA[8][32][KW], sdL[8][32][KW];
   __shared__ float bs[32], dbs[32];
 
@@ -248,8 +250,8 @@ simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const
     float hs = 0.f;
     for (int c = lane; c < d; c += 32) {
       const float x = key_live ? Kp[(size_t)(j0 + q) * d + c] : 0.f;
-      ks[warp * KW + q][c] = x;
-      vs[warp * KW + q][c] = key_live ? Vp[(size_t)(j0 + q) * d + c] : 0.f;
+      ks[(warp * KW + q) * d + c] = x;
+      vs[(warp * KW + q) * d + c] = key_live ? Vp[(size_t)(j0 + q) * d + c] : 0.f;
       hs = fmaf(x, x, hs);
     }
 #pragma unroll
@@ -289,8 +291,8 @@ simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const
       const float wsv = kPerformer ? Ws[lane * (d + 1) + c] : 0.f;
 #pragma unroll
       for (int q = 0; q < KW; ++q) {
-        e1[q] = fmaf(dsv, vs[warp * KW + q][c] - asv, e1[q]);
-        if (kPerformer) wk[q] = fmaf(wsv, ks[warp * KW + q][c], wk[q]);
+        e1[q] = fmaf(dsv, vs[(warp * KW + q) * d + c] - asv, e1[q]);
+        if (kPerformer) wk[q] = fmaf(wsv, ks[(warp * KW + q) * d + c], wk[q]);
       }
     }
 #pragma unroll
@@ -300,12 +302,12 @@ simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const
       if (live) {
         g = e1[q] + dbs[lane];
         if (kPerformer) A = expf(wk[q] - half_sq[q] - bs[lane]);     // b_i = log sum_j exp(L_ji): A <= 1
-        else A = elu1(ks[warp * KW + q][i0 + lane]) / bs[lane];      // weight holds z_i for RNN
+        else A = elu1(ks[(warp * KW + q) * d + i0 + lane]) / bs[lane];      // weight holds z_i for RNN
       }
       const float dL = A * g;
       dl_sum[q] += dL;
       if (!kPerformer && live) {
-        const float x = ks[warp * KW + q][i0 + lane];
+        const float x = ks[(warp * KW + q) * d + i0 + lane];
         dKpVp[((size_t)bh * k + j0 + q) * d + i0 + lane] = dL * elu1_slope(x) / elu1(x);
       }
       sA[warp][lane][q] = A;
@@ -342,7 +344,7 @@ simt_bwd_key_side(const float* __restrict__ KpVp, const T* __restrict__ W, const
     for (int b = 0; b < 4; ++b) {
       const int c = lane + 32 * b;
       if (c < d) {
-        if (kPerformer) dKpVp[((size_t)bh * k + j0 + q) * d + c] = dk[q][b] - ks[warp * KW + q][c] * ds;
+        if (kPerformer) dKpVp[((size_t)bh * k + j0 + q) * d + c] = dk[q][b] - ks[(warp * KW + q) * d + c] * ds;
         dKpVp[(((size_t)BH + bh) * k + j0 + q) * d + c] = dv[q][b];
       }
     }
