@@ -103,6 +103,8 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const bool owner = warp >= 2;
   const int q4 = warp & 3, row = q4 * 32 + lane;
   const int fh = (warp - 2) >> 2;              // which 64 of a step's 128 features this row owner takes
+  // (RNN: 64 features in all, 32 per thread of a row)
+  const int c_lo = kPerformer ? fh * 64 : fh * 32, c_hi = kPerformer ? fh * 64 + 64 : fh * 32 + 32;
   const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
 
   // d = 128: a CTA walks its tiles twice, once per 64-column half of dQ and da (visit i: half i / nt, tile i % nt)
@@ -139,6 +141,11 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // the delta operand [16 x 128] (K-major, no swizzle): rows 0..2 are rewritten per tile, the rest stays zero
     uint32_t* dz = reinterpret_cast<uint32_t*>(base_ptr + kK4Delta);
     for (int e = lane; e < 1024; e += 32) dz[e] = 0u;
+  }
+  if (!kPerformer && warp >= 4) {
+    // RNN: features 64..127 of the P tile (its second slab) do not exist: zero, once
+    uint32_t* pz = reinterpret_cast<uint32_t*>(base_ptr + kK4P + 16384);
+    for (int e = threadIdx.x - 128; e < 4096; e += kK4Threads - 128) pz[e] = 0u;
   }
   fence_proxy_async_smem();
   tcgen05_fence_before();
@@ -345,12 +352,13 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const uint64_t b1 = make_sdesc(base + kK4Bias + h * 4096, 128, 256, kSwizzleNone);
         mma_ss(tmem, a1, b1, idescS, 1u);
       }
+      const uint32_t idescG = kPerformer ? idescS : make_idesc(kFmtBF16, 0, 0, 128, 64);   // RNN: 64 features
       for (int kb = 0; kb < kd; ++kb) {
         const uint64_t ag = make_sdesc(sm_do + kb * 16384, 16, 1024, kSwizzle128);
         const uint64_t bh = make_sdesc(base + kK4AHi + fo + kb * 16384, 16, 1024, kSwizzle128);
         const uint64_t bl = make_sdesc(base + kK4ALo + fo + kb * 16384, 16, 1024, kSwizzle128);
-        mma_ss_x4(tmem + kK4ColG, ag, bh, 2, 2, idescS, kb > 0 ? 1u : 0u);
-        mma_ss_x4(tmem + kK4ColG, ag, bl, 2, 2, idescS, 1u);
+        mma_ss_x4(tmem + kK4ColG, ag, bh, 2, 2, idescG, kb > 0 ? 1u : 0u);
+        mma_ss_x4(tmem + kK4ColG, ag, bl, 2, 2, idescG, 1u);
       }
       mma_commit(bar_mma);
     };
@@ -388,10 +396,10 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       if (owner) {
         mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
         // (this thread's 64 features of the step lie past p: padding, weight zero; the same for the whole warp)
-        if (mine && h * 128 + fh * 64 < p) {
+        if (mine && (!kPerformer || h * 128 + fh * 64 < p)) {
           tcgen05_fence_after();
 #pragma unroll 1
-          for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
+          for (int c = c_lo; c < c_hi; c += 32) {
             uint32_t rs[32], rg[32];
             if (!kPerformer) {
               // no exponent to stabilise: the weights are products of bounded factors
@@ -480,11 +488,11 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tcgen05_fence_after();
           const uint32_t prow = base + kK4P + (uint32_t)row * 128u;
 #pragma unroll 1
-          for (int c = fh * 64; c < fh * 64 + 64; c += 32) {
+          for (int c = c_lo; c < c_hi; c += 32) {
             uint32_t rs[32], rg[32], cw[16];
             const uint32_t slab = prow + (uint32_t)(c >> 6) * 16384u;
             // features past p (padding of the last tile): P and c exactly zero
-            const float keep = (h * 128 + fh * 64 < p) ? 1.f : 0.f;
+            const float keep = (!kPerformer || h * 128 + fh * 64 < p) ? 1.f : 0.f;
             if (!kPerformer) {
               // RNN (p = d = 64): P = weights / their sum; dq_ni = c_ni elu'(q_ni) / (elu(q_ni) + 1) needs no
               // product, so this thread stores its 32 columns of the dQ row here
