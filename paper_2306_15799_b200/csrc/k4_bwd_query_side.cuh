@@ -12,7 +12,8 @@
 //     da += P^T dO  and  (P^T delta) += P^T [delta_hi delta_mid delta_lo]  (P = bf16, written to shared memory
 //     by the row owners in the canonical 128-byte-swizzled layout, used as an MN-major A operand),
 // in two sweeps over the features, 128 at a time: the first gives each row its log-sum-exp and
-// delta_n (running maximum, sum and P-weighted sum of g), the second forms P and c.  da and P^T delta
+// delta_n (running maximum, sum and P-weighted sum of g), the second forms P and c, starting with the step
+// whose S and G sweep 1 left in TMEM.  da and P^T delta
 // stay in TMEM over all the tiles a CTA has of one head and are added to global memory (atomics) when
 // the head changes; db comes from them there.  Two threads per query row (8 warps; each takes 64 of the 128
 // features of a step), one MMA issuer, one TMA thread; the phases of a tile follow one another (block
@@ -475,15 +476,18 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
 
     // ------------------------------------------------------------ sweep 2: P, c and the three products they feed
-    for (int h = 0; h < nh && ok; ++h) {
-      if (stream) {
+    // (last step first: its S and G are still in TMEM from sweep 1, and at d = 128 its W is still in shared memory)
+    for (int hi = 0; hi < nh && ok; ++hi) {
+      const int h = nh - 1 - hi;
+      const bool reuse = hi == 0 && !have_stats;
+      if (stream && !reuse) {
         load_step(h);
         if (!step_ok) { ok = false; break; }
       }
-      if (warp == 1 && elect_one()) issue_sg(h);
+      if (!reuse && warp == 1 && elect_one()) issue_sg(h);
       bool mine = true;
       if (owner) {
-        mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
+        if (!reuse) mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
         if (mine) {
           tcgen05_fence_after();
           const uint32_t prow = base + kK4P + (uint32_t)row * 128u;
@@ -550,7 +554,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tcgen05_fence_before();
         }
       }
-      ph_mma ^= 1;
+      if (!reuse) ph_mma ^= 1;
       ok = __syncthreads_and(mine) != 0;
       if (!ok) break;
       if (warp == 1 && elect_one()) {
@@ -559,7 +563,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int j = 0; kPerformer && j < 2; ++j) {
           // W rows of the step's features, the 64 columns this visit owns
           const uint64_t bw = make_sdesc(base + kK4W + (stream ? dh : h) * 16384 + j * 8192, 8192, 1024, kSwizzle128);
-          mma_ts_x4(tmem + kK4ColDQ, tmem + j * 64, bw, 128, idescQ, (h > 0 || j > 0) ? 1u : 0u);
+          mma_ts_x4(tmem + kK4ColDQ, tmem + j * 64, bw, 128, idescQ, (hi > 0 || j > 0) ? 1u : 0u);
         }
         // da_h (+)= P_h^T dO and (P^T delta)_h: 128 rows = 8 steps of 16 rows (2048 B of P and of dO, 256 B of delta)
         for (int j = 0; j < 2; ++j) {
