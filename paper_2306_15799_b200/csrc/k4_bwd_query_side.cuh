@@ -230,6 +230,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint32_t ph_mma = 0, ph_mma2 = 0, ph_head = 0, ph_step = 0;
   int head_prev = -1;
   bool first_of_head = true;
+  bool pre_issued = false;        // this tile's first S and G were issued at the end of the previous tile
   const float kLog2e = 1.4426950408889634f;
   const uint32_t idescS = make_idesc(kFmtBF16, 0, 0, 128, 128);   // S, G: both operands K-major
   const uint32_t idescQ = make_idesc(kFmtBF16, 0, 1, 128, 64);    // dQ: A from TMEM, W as an MN-major B
@@ -338,7 +339,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       ph_step ^= 1;
       step_ok = __syncthreads_and(mine) != 0;
     };
-    auto issue_sg = [&](int h) {
+    auto issue_sg_from = [&](int h, uint32_t sm_q, uint32_t sm_do) {
       tcgen05_fence_after();
       // rows of the step's features: at h * 16384 in the resident tiles (d = 64), at 0 in the step's own (d = 128);
       // 64-column blocks of the head dimension 16384 B apart
@@ -363,6 +364,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       mma_commit(bar_mma);
     };
+    auto issue_sg = [&](int h) { issue_sg_from(h, sm_q, sm_do); };
 
     // RNN: the un-normalised weights (elu(q_ni) + 1) z_i / max z of 32 features (i = c .. c + 31 = columns of
     // this thread's row of the Q tile, which is 128-byte swizzled) and the factor elu'(q) / (elu(q) + 1)
@@ -392,7 +394,7 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         load_step(h);
         if (!step_ok) { ok = false; break; }
       }
-      if (warp == 1 && elect_one()) issue_sg(h);
+      if (!(pre_issued && h == 0) && warp == 1 && elect_one()) issue_sg(h);
       bool mine = true;
       if (owner) {
         mine = mbar_wait(bar_mma, ph_mma, prm.status, &abort_flag);
@@ -582,6 +584,20 @@ k4_bwd_query_side(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
     if (!ok) break;
     first_of_head = false;
+    // the next tile's first S and G (same head, its Q and dO already fetched) can run under this tile's dQ read-out:
+    // every product that used the S and G columns is complete
+    pre_issued = false;
+    if (!stream && i + 1 < ntiles && (t_begin + i + 1) / prm.tiles_per_head == head) {
+      pre_issued = true;
+      if (warp == 1) {
+        const uint32_t nst = (uint32_t)((i + 1) & 1);
+        const bool landed = mbar_wait(bar_in + 8 * nst, (uint32_t)((i + 1) >> 1) & 1u, prm.status, &abort_flag);
+        if (__all_sync(0xffffffffu, landed ? 1 : 0) && elect_one()) {
+          const uint32_t nq = base + kK4In + nst * 32768u;
+          issue_sg_from(0, nq, nq + 16384u);
+        }
+      }
+    }
 
     // ------------------------------------------------------------ dQ rows (32 columns per thread)
     if (kPerformer && owner) {
