@@ -271,6 +271,24 @@ def test_rnn_head_change_at_a_ctas_second_tile(limit, tiles):
         binding.flurka_set_cta_limit(prev)
 
 
+def test_rnn_forward_is_repeatable_with_every_sm_busy():
+    """Twelve runs of an RNN forward with 148 CTAs whose tile ranges cross heads at every position: apart from the
+    order of stage 1's fp32 partial sums (which RNN features do not amplify) nothing may differ from run to run.
+    A stale per-head operand shows here as a difference of many units in the last place."""
+    w = Workload("rnn_repeatable", RNN, "bf16", 2, 12, 4096, 64, 256, 0, 431)
+    dev = pu.to_device(synth.make_inputs(w))
+    first = None
+    for _ in range(12):
+        out = binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant).float()
+        torch.cuda.synchronize()
+        assert binding.flurka_last_status() == 0 and binding.flurka_last_path() == binding.PATH_TENSOR
+        if first is None:
+            first = out.clone()
+            continue
+        spacing = torch.clamp(first.abs(), min=1e-2) * 2.0 ** -7          # bf16 spacing of the first run's values
+        assert float(((out - first).abs() / spacing).max()) <= 2.0
+
+
 def test_auto_picks_tensor_path_when_the_shape_allows():
     w = TENSOR_CASES[0]
     pu.check_all_heads(w)
