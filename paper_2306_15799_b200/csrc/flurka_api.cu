@@ -894,7 +894,11 @@ int backward_pipeline(const Problem& pr, const BackwardLayout& BL, char* ws, con
                                 pr.p(), smh);
     ++*launches;
   }
-  {
+  if (tc && P && pr.d == 64) {
+    rc = launch_k6(*tc, W, kpvp, weight, a32, da, db, dkpvp, pr.BH(), pr.k, pr.p(), (int*)(ws + L.status), st, &cuda_err);
+    if (rc) { g_last_cuda_error = cuda_err; return rc; }
+    ++*launches;
+  } else {
     auto fn = simt_bwd_key_side<T, P>;
     const size_t smem = ((size_t)3 * 32 * (pr.d + 1) + (size_t)2 * 8 * kBwdKeysPerWarp * pr.d) * 4;
     if ((e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)

@@ -13,6 +13,7 @@
 #include "k3_query_side.cuh"
 #include "k4_bwd_query_side.cuh"
 #include "k5_bwd_projections.cuh"
+#include "k6_bwd_key_side.cuh"
 
 namespace flurka {
 
@@ -544,6 +545,28 @@ inline int launch_k5(TensorContext& tc, const void* E, const void* F, const void
         tm.bK.map, tm.bV.map, tm.split128.map, tm.gE.map, tm.gF.map, p);
   }
   cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
+  return 0;
+}
+
+// ---- backward of the key side (PERFORMER, d = 64): dK', dV' from da, db ---------------------------------
+inline int launch_k6(TensorContext& tc, const void* W, const float* kpvp, const float* weight, const float* a32,
+                     const float* da, const float* db, float* dkpvp, int BH, int k, int p, int* status, cudaStream_t st,
+                     int* cuda_err) {
+  TensorMaps& tm = tc.maps;
+  const unsigned long long dW[2] = {64ull, (unsigned long long)p};
+  const unsigned bW[2] = {64, 128};
+  if (!encode_map(&tm.W2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, 2, W, dW, bW)) {
+    *cuda_err = (int)cudaErrorInvalidValue;
+    return -6;
+  }
+  K6Params prm;
+  prm.k = k; prm.p = p; prm.BH = BH;
+  prm.kpvp = kpvp; prm.weight = weight; prm.a32 = a32; prm.da = da; prm.db = db; prm.dkpvp = dkpvp; prm.status = status;
+  cudaError_t e = cudaFuncSetAttribute(k6_bwd_key_side, cudaFuncAttributeMaxDynamicSharedMemorySize, kK6SmemBytes);
+  if (e != cudaSuccess) { *cuda_err = (int)e; (void)cudaGetLastError(); return -6; }
+  k6_bwd_key_side<<<BH * ((k + 127) / 128), kK6Threads, kK6SmemBytes, st>>>(tm.W2.map, prm);
+  e = cudaGetLastError();
   if (e != cudaSuccess) { *cuda_err = (int)e; return -6; }
   return 0;
 }
