@@ -178,7 +178,8 @@ int flurka_forward_finish(const void* Q, const void* W, int variant, int B, int 
  * Kernels: where flurka_forward's tensor-core path takes the shape (bf16, the rules below) the two
  * down-projections, the key-side summaries and, with E, F shared by the heads, the gradients dK, dV, dE, dF
  * (products with E, F, K, V: dK', dV' enter as two bf16 terms) run on tcgen05 kernels; so does the query side
- * (dQ and the gradients of the key-side summaries) for d = 64 and, PERFORMER only, d = 128.
+ * (dQ and the gradients of the key-side summaries) for d = 64 and, PERFORMER only, d = 128, and the key side's
+ * backward half (dK', dV' from those gradients) for PERFORMER with d = 64.
  * flurka_last_path() then reports FLURKA_PATH_TENSOR (query side included) or FLURKA_PATH_TENSOR_STAGE1.
  * Everything else, and every shape under FLURKA_PATH_SIMT, runs on CUDA cores with fp32 arithmetic;
  * FLURKA_PATH_TENSOR forced on a shape without a tensor-core query side returns FLURKA_ERR_SHAPE.

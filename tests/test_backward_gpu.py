@@ -93,6 +93,9 @@ TENSOR_CASES = [
     Workload("bwd_tc_d128_m128", PERFORMER, "bf16", 1, 2, 520, 128, 320, 128, 319),
     Workload("bwd_tc_d128_m256", PERFORMER, "bf16", 2, 2, 392, 128, 64, 256, 325),
     Workload("bwd_tc_d128_m64", PERFORMER, "bf16", 1, 3, 264, 128, 128, 64, 326),
+    # key side on its tensor-core kernel with a last chunk of 64 keys (k = 320) and with four chunks (k = 512)
+    Workload("bwd_tc_k320", PERFORMER, "bf16", 1, 2, 264, 64, 320, 128, 329),
+    Workload("bwd_tc_k512_m64", PERFORMER, "bf16", 2, 1, 392, 64, 512, 64, 330),
 ]
 
 
