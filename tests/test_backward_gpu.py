@@ -146,6 +146,15 @@ def test_backward_full_length_sequences():
         binding.flurka_set_cta_limit(prev)
 
 
+def test_backward_tensor_path_with_per_head_projections():
+    """One pair E_i, F_i per head on a tensor-core shape: stage 1, the key side and the query side on their
+    tcgen05 kernels, the products with E, F, K, V on CUDA cores (the tensor-core ones need shared E, F)."""
+    _check(Workload("bwd_tc_per_head", PERFORMER, "bf16", 2, 3, 392, 64, 128, 128, 331), per_head=True)
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+    _check(Workload("bwd_tc_per_head_rnn_bnhd", RNN, "bf16", 2, 2, 264, 64, 64, 0, 332), layout="bnhd", per_head=True)
+    assert binding.flurka_last_path() == binding.PATH_TENSOR
+
+
 def test_backward_cuda_core_path_on_a_tensor_shape():
     prev = binding.flurka_set_path(binding.PATH_SIMT)
     try:
