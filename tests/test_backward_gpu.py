@@ -155,6 +155,31 @@ def test_backward_tensor_path_with_per_head_projections():
     assert binding.flurka_last_path() == binding.PATH_TENSOR
 
 
+@pytest.mark.parametrize("d,m", [(64, 256), (128, 256)])
+def test_backward_in_a_caller_workspace_of_exactly_the_stated_size(d, m):
+    """flurka_backward_workspace_bytes covers every scratch area of the tensor-core kernels (the bf16 terms of a
+    and of dK', dV', the per-row statistics at d = 128): a caller's block of exactly that size works, a smaller
+    one is refused."""
+    w = Workload("bwd_ws_d%d" % d, PERFORMER, "bf16", 1, 2, 392, d, 128, m, 340 + d)
+    need = binding.flurka_backward_workspace_bytes(w.variant, torch.bfloat16, w.B, w.H, w.N, w.d, w.k, w.m)
+    assert need > binding.flurka_workspace_bytes(w.variant, torch.bfloat16, w.B, w.H, w.N, w.d, w.k, w.m)
+    x = pu.to_device(synth.make_inputs(w))
+    dO = torch.randn_like(x["Q"])
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    binding.flurka_set_workspace(small)
+    try:
+        with pytest.raises(binding.FlurkaError) as ei:
+            binding.flurka_backward(x["Q"], x["K"], x["V"], x["E"], x["F"], x["W"], dO, w.variant)
+        assert ei.value.code == -5
+        # poisoned, so that anything the kernels read without having written it shows
+        buf = torch.full((need,), 0xFF, dtype=torch.uint8, device="cuda")
+        binding.flurka_set_workspace(buf)
+        _check(w)
+        assert binding.flurka_last_path() == binding.PATH_TENSOR
+    finally:
+        binding.flurka_set_workspace(None)
+
+
 def test_backward_cuda_core_path_on_a_tensor_shape():
     prev = binding.flurka_set_path(binding.PATH_SIMT)
     try:
