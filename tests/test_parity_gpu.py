@@ -148,7 +148,7 @@ def test_caller_workspace_and_too_small_workspace():
         with pytest.raises(binding.FlurkaError) as ei:
             binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], None, w.variant)
         assert ei.value.code == -5
-        buf = torch.empty(need, dtype=torch.uint8, device="cuda")
+        buf = torch.full((need,), 0xFF, dtype=torch.uint8, device="cuda")     # poisoned: nothing may be read unwritten
         binding.flurka_set_workspace(buf)
         out = binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], None, w.variant)
         torch.cuda.synchronize()
@@ -156,6 +156,25 @@ def test_caller_workspace_and_too_small_workspace():
         binding.flurka_set_workspace(None)
     ref = pu.oracle_head(inputs, w, 0, 1)
     pu.assert_close(out[0, 1].cpu().double().numpy(), ref, "bf16", "caller workspace")
+
+
+def test_performer_tensor_path_in_a_poisoned_caller_workspace():
+    """The PERFORMER tensor path (key split included: k = 256, two heads) in a caller's block of exactly the
+    stated size that was filled with 0xFF: every scratch area is written before it is read."""
+    w = _wl("ws_perf_bf16", PERFORMER, "bf16", 1, 2, 520, 64, 256, 256, 52)
+    inputs = synth.make_inputs(w)
+    need = binding.flurka_workspace_bytes(w.variant, torch.bfloat16, w.B, w.H, w.N, w.d, w.k, w.m)
+    dev = pu.to_device(inputs)
+    buf = torch.full((need,), 0xFF, dtype=torch.uint8, device="cuda")
+    binding.flurka_set_workspace(buf)
+    try:
+        out = binding.flurka_forward(dev["Q"], dev["K"], dev["V"], dev["E"], dev["F"], dev["W"], w.variant)
+        torch.cuda.synchronize()
+        assert binding.flurka_last_status() == 0 and binding.flurka_last_path() == binding.PATH_TENSOR
+    finally:
+        binding.flurka_set_workspace(None)
+    for h in range(2):
+        pu.assert_close(out[0, h].cpu().double().numpy(), pu.oracle_head(inputs, w, 0, h), "bf16", "poisoned workspace head %d" % h)
 
 
 def test_repeated_calls_are_independent():
